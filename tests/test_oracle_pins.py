@@ -1,0 +1,439 @@
+"""Pins for the fp64 oracle: closed forms, statistics the Gaussian sketch must
+obey, SVD leverage scores, invariants and brute force.  CPU only.
+
+Each test is chosen so that one plausible mistake in the oracle (a dropped
+term, a transposed G, a wrong index base, a wrong tie rule) makes it fail.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import curdkv_oracle as orc
+from paper_2509_15038_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_bits(x):
+    return synth.f64_to_bf16_u16(np.asarray(x, dtype=np.float64))
+
+
+def rand_kv(rng, B, H, n, d, scale=1.0):
+    K = bf16_bits(rng.standard_normal((B, H, n, d)) * scale)
+    V = bf16_bits(rng.standard_normal((B, H, n, d)) * scale)
+    return K, V
+
+
+# ---------------------------------------------------------------- sketch + norms
+
+def test_hand_worked_example():
+    """Alg. 1 lines 2-9 on the exact-arithmetic example in tests/golden/hand_example.txt."""
+    vals = {}
+    with open(os.path.join(GOLDEN, "hand_example.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, *nums = line.split()
+            vals[name] = np.array([float(x) for x in nums])
+    K = bf16_bits([[[[1, 0], [0, 2], [1, 1], [3, -1]]]])
+    V = bf16_bits([[[[2, 0], [1, 1], [0, 1], [1, 0]]]])
+    G = np.array([[1, 1], [0, 2]], dtype=np.float32)
+    sc, S, lK, lV = orc.score(K, V, G, return_factors=True)
+    np.testing.assert_allclose(lK[0, 0], vals["lK"], rtol=0, atol=0)
+    np.testing.assert_allclose(lV[0, 0], vals["lV"], rtol=0, atol=0)
+    assert S[0, 0] == vals["sum"][0]
+    np.testing.assert_allclose(sc[0, 0], vals["lKV"] / vals["sum"][0], rtol=1e-15)
+    sck, Sk = orc.score(K, V, G, score_mode=1)
+    scv, Sv = orc.score(K, V, G, score_mode=2)
+    np.testing.assert_allclose(sck[0, 0], vals["lK"] / 38.0, rtol=1e-15)
+    np.testing.assert_allclose(scv[0, 0], vals["lV"] / 24.0, rtol=1e-15)
+    idx, cnt = orc.select_fixed(sc, budget=2, num_sink=1)
+    assert idx[0, 0].tolist() == vals["select_s1_k2"].astype(int).tolist() and cnt[0, 0] == 2
+    idx, cnt = orc.select_fixed(sc, budget=3, num_sink=1)
+    assert idx[0, 0].tolist() == vals["select_s1_k3"].astype(int).tolist() and cnt[0, 0] == 3
+
+
+def test_orthogonal_G_gives_exact_row_norms():
+    """G orthogonal (r = d) => ||a G||^2 = ||a||^2 exactly (up to fp64 rounding)."""
+    rng = np.random.default_rng(1)
+    B, H, n, d = 2, 3, 17, 16
+    K, V = rand_kv(rng, B, H, n, d)
+    Q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    # fp32 G: orthogonal to ~1e-7, so the identity holds to ~1e-6 relative
+    for G in (np.eye(d, dtype=np.float32), Q.astype(np.float32)):
+        _, _, lK, lV = orc.score(K, V, G, return_factors=True)
+        nk = (synth.u16_to_f64(K) ** 2).sum(-1)
+        nv = (synth.u16_to_f64(V) ** 2).sum(-1)
+        np.testing.assert_allclose(lK, nk, rtol=2e-6)
+        np.testing.assert_allclose(lV, nv, rtol=2e-6)
+
+
+def test_selector_G_catches_transposed_or_misindexed_G():
+    """G = [I_r; 0] picks the first r coordinates; one-hot G[t0][c0] = 2 gives 4 a[t0]^2.
+    A transposed or mis-strided G changes both closed forms."""
+    rng = np.random.default_rng(2)
+    B, H, n, d, r = 1, 2, 9, 12, 5
+    K, V = rand_kv(rng, B, H, n, d)
+    Kd, Vd = synth.u16_to_f64(K), synth.u16_to_f64(V)
+    G = np.zeros((d, r), dtype=np.float32)
+    G[:r, :r] = np.eye(r)
+    _, _, lK, lV = orc.score(K, V, G, return_factors=True)
+    np.testing.assert_allclose(lK, (Kd[..., :r] ** 2).sum(-1), rtol=1e-14)
+    np.testing.assert_allclose(lV, (Vd[..., :r] ** 2).sum(-1), rtol=1e-14)
+    G = np.zeros((d, r), dtype=np.float32)
+    G[7, 3] = 2.0
+    _, _, lK, lV = orc.score(K, V, G, return_factors=True)
+    np.testing.assert_allclose(lK, 4 * Kd[..., 7] ** 2, rtol=1e-14)
+    np.testing.assert_allclose(lV, 4 * Vd[..., 7] ** 2, rtol=1e-14)
+
+
+def test_per_head_G():
+    """A [H, d, r] G applies head h's matrix to head h only."""
+    rng = np.random.default_rng(3)
+    B, H, n, d, r = 2, 3, 5, 8, 4
+    K, V = rand_kv(rng, B, H, n, d)
+    G = synth.make_G(d, r, seed=5, heads=H)
+    sc, S = orc.score(K, V, G)
+    for h in range(H):
+        sh, Sh = orc.score(K[:, h:h + 1], V[:, h:h + 1], G[h])
+        np.testing.assert_array_equal(sc[:, h], sh[:, 0])
+        np.testing.assert_array_equal(S[:, h], Sh[:, 0])
+
+
+def test_gaussian_sketch_moments():
+    """G_ij ~ N(0,1/r) => l_j / ||a_j||^2 ~ chi2_r / r: mean 1, variance 2/r (Sec. 3.2)."""
+    rng = np.random.default_rng(4)
+    d, r, n, trials = 16, 8, 4, 2000
+    K, V = rand_kv(rng, 1, 1, n, d)
+    norms = (synth.u16_to_f64(K)[0, 0] ** 2).sum(-1)
+    ratios = np.empty((trials, n))
+    for t in range(trials):
+        G = synth.make_G(d, r, seed=1000 + t)
+        _, _, lK, _ = orc.score(K, V, G, return_factors=True)
+        ratios[t] = lK[0, 0] / norms
+    mean, var = ratios.mean(0), ratios.var(0)
+    se_mean = np.sqrt(2.0 / r / trials)
+    assert np.all(np.abs(mean - 1.0) < 4 * se_mean)
+    # Var of the sample variance of chi2_r/r: (m4 - s^4)/T with m4 = 12(r+4)/r^3 + 4/r^2
+    s2 = 2.0 / r
+    m4 = 12.0 * (r + 4) / r ** 3 + s2 ** 2
+    se_var = np.sqrt((m4 - s2 ** 2) / trials)
+    assert np.all(np.abs(var - s2) < 4 * se_var)
+
+
+def test_sketch_error_shrinks_like_inverse_sqrt_r():
+    rng = np.random.default_rng(5)
+    d, n = 32, 64
+    K, V = rand_kv(rng, 1, 1, n, d)
+    norms = (synth.u16_to_f64(K)[0, 0] ** 2).sum(-1)
+    rs = [8, 32, 128, 512, 2048]
+    errs = []
+    for r in rs:
+        e = []
+        for seed in range(6):
+            _, _, lK, _ = orc.score(K, V, synth.make_G(d, r, seed=seed), return_factors=True)
+            e.append(np.sqrt(np.mean((lK[0, 0] / norms - 1.0) ** 2)))
+        errs.append(np.mean(e))
+    slope = np.polyfit(np.log(rs), np.log(errs), 1)[0]
+    assert -0.62 < slope < -0.38, (slope, errs)
+    np.testing.assert_allclose(errs, np.sqrt(2.0 / np.array(rs)), rtol=0.25)
+
+
+def test_flat_spectrum_matches_svd_leverage():
+    """On A = c U W^T (equal singular values) normalised sketch scores converge to the
+    SVD row leverage ||U(j,:)||^2 / rank (Eq. row leverage score); sum of squared
+    leverages equals rank(A)."""
+    rng = np.random.default_rng(6)
+    n, d, q = 48, 16, 16
+    U, _ = np.linalg.qr(rng.standard_normal((n, q)))
+    W, _ = np.linalg.qr(rng.standard_normal((d, q)))
+    A = 3.0 * U @ W.T
+    K = bf16_bits(A[None, None])
+    Ad = synth.u16_to_f64(K)[0, 0]
+    Us, sv, _ = np.linalg.svd(Ad, full_matrices=False)
+    rank = int((sv > 1e-8 * sv[0]).sum())
+    lev = (Us[:, :rank] ** 2).sum(-1)
+    assert rank == q and abs(lev.sum() - rank) < 1e-9
+    assert sv.max() / sv.min() < 1.02            # bf16 rounding keeps the spectrum ~flat
+    errs = []
+    for r in (16, 256, 4096):
+        sc, _ = orc.score(K, K, synth.make_G(d, r, seed=r), score_mode=1)
+        errs.append(np.abs(sc[0, 0] - lev / rank).max() / (lev / rank).max())
+    assert errs[0] > errs[1] > errs[2] and errs[2] < 0.06, errs
+    # exact limit: orthogonal G
+    sc, _ = orc.score(K, K, np.eye(d, dtype=np.float32), score_mode=1)
+    np.testing.assert_allclose(sc[0, 0], lev / rank, rtol=0.03)
+
+
+def test_general_matrix_converges_to_row_norms_not_leverage():
+    """Without whitening the sketch estimates squared row norms; on a matrix with a
+    decaying spectrum these differ from SVD leverage (recorded, not a defect)."""
+    rng = np.random.default_rng(7)
+    n, d = 40, 8
+    A = rng.standard_normal((n, d)) * np.array([8, 4, 2, 1, 1, 0.5, 0.25, 0.1])
+    K = bf16_bits(A[None, None])
+    Ad = synth.u16_to_f64(K)[0, 0]
+    sc, _ = orc.score(K, K, synth.make_G(d, 8192, seed=0), score_mode=1)
+    rown = (Ad ** 2).sum(-1)
+    np.testing.assert_allclose(sc[0, 0], rown / rown.sum(), rtol=0.1)
+    Us, _, _ = np.linalg.svd(Ad, full_matrices=False)
+    lev = (Us ** 2).sum(-1) / d
+    assert np.abs(sc[0, 0] - lev).max() > 0.2 * lev.max()
+
+
+# ---------------------------------------------------------------- combine + normalise
+
+def test_scores_sum_to_one_and_are_product_of_factors():
+    rng = np.random.default_rng(8)
+    B, H, n, d, r = 2, 4, 33, 16, 8
+    K, V = rand_kv(rng, B, H, n, d)
+    G = synth.make_G(d, r)
+    sc, S, lK, lV = orc.score(K, V, G, return_factors=True)
+    np.testing.assert_allclose(sc.sum(-1), 1.0, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(sc * S[..., None], lK * lV, rtol=1e-13)
+    np.testing.assert_allclose(S, (lK * lV).sum(-1), rtol=1e-13)
+
+
+def test_scale_invariance_and_permutation_equivariance():
+    rng = np.random.default_rng(9)
+    B, H, n, d, r = 1, 2, 21, 16, 8
+    K, V = rand_kv(rng, B, H, n, d)
+    G = synth.make_G(d, r)
+    sc, S = orc.score(K, V, G)
+    # powers of two scale bf16 values exactly
+    K4 = bf16_bits(synth.u16_to_f64(K) * 4.0)
+    Vh = bf16_bits(synth.u16_to_f64(V) * 0.5)
+    sc2, S2 = orc.score(K4, Vh, G)
+    np.testing.assert_allclose(sc2, sc, rtol=1e-13)
+    np.testing.assert_allclose(S2, S * 16.0 * 0.25, rtol=1e-13)
+    perm = rng.permutation(n)
+    sc3, _ = orc.score(K[:, :, perm], V[:, :, perm], G)
+    np.testing.assert_allclose(sc3, sc[:, :, perm], rtol=1e-12)
+    i0, _ = orc.select_fixed(sc, budget=7)
+    i3, _ = orc.select_fixed(sc3, budget=7)
+    for h in range(H):
+        assert sorted(perm[i3[0, h]].tolist()) == i0[0, h].tolist()
+
+
+def test_ragged_lengths_ignore_padding_rows():
+    rng = np.random.default_rng(10)
+    B, H, n, d, r = 3, 2, 20, 8, 4
+    K, V = rand_kv(rng, B, H, n, d)
+    G = synth.make_G(d, r)
+    lens = np.array([20, 7, 0], dtype=np.int32)
+    sc, S = orc.score(K, V, G, seqlens=lens)
+    for b in range(B):
+        nb = lens[b]
+        assert np.all(sc[b, :, nb:] == 0)
+        if nb:
+            ref, Sr = orc.score(K[b:b + 1, :, :nb], V[b:b + 1, :, :nb], G)
+            np.testing.assert_array_equal(sc[b, :, :nb], ref[0])
+        else:
+            assert np.all(S[b] == 0)
+    idx, cnt = orc.select_fixed(sc, budget=9, window=2, seqlens=lens)
+    assert cnt[:, 0].tolist() == [9, 7, 0]
+    assert idx[1, 0, :7].tolist() == list(range(7)) and np.all(idx[1, 0, 7:] == -1)
+    assert np.all(idx[2] == -1)
+
+
+def test_no_projection_ablation_is_plain_row_norms():
+    rng = np.random.default_rng(11)
+    K, V = rand_kv(rng, 1, 2, 10, 8)
+    _, _, lK, lV = orc.score(K, V, synth.make_G(8, 4), use_projection=0, return_factors=True)
+    np.testing.assert_allclose(lK, (synth.u16_to_f64(K) ** 2).sum(-1), rtol=1e-14)
+    np.testing.assert_allclose(lV, (synth.u16_to_f64(V) ** 2).sum(-1), rtol=1e-14)
+
+
+def test_planted_tokens_are_selected_cfg1_recipe():
+    """Rows scaled x20 in K and V score ~1.6e5x typical, so every planted token outside
+    the window is kept for any k >= 8 + window."""
+    w = synth.shrink(synth.CONFIGS["cfg1"], n_max=256)
+    K, V = synth.make_kv_element(w, 0)
+    Ku, Vu = synth.to_u16(K)[None], synth.to_u16(V)[None]
+    sc, _ = orc.score(Ku, Vu, synth.make_G(w.d, w.r))
+    idx, cnt = orc.select_fixed(sc, budget=8 + 32, window=32)
+    rown = (synth.u16_to_f64(Ku) ** 2).sum(-1)[0]
+    for h in range(w.kv_heads):
+        planted = np.argsort(rown[h])[-8:]
+        assert rown[h][planted].min() > 100 * np.median(rown[h])
+        assert set(planted.tolist()) <= set(idx[0, h].tolist())
+        assert set(range(256 - 32, 256)) <= set(idx[0, h].tolist())
+
+
+# ---------------------------------------------------------------- top-k
+
+def brute_fixed(sc, k, s, w):
+    n = len(sc)
+    k_eff = min(k, n)
+    forced = []
+    for j in range(n - 1, max(n - w, 0) - 1, -1):
+        if len(forced) < k_eff:
+            forced.append(j)
+    for j in range(min(s, n)):
+        if j not in forced and len(forced) < k_eff:
+            forced.append(j)
+    cand = sorted((j for j in range(n) if j not in forced), key=lambda j: (-sc[j], j))
+    return sorted(forced + cand[: k_eff - len(forced)])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_select_fixed_matches_brute_force(seed):
+    rng = np.random.default_rng(100 + seed)
+    B, H, n = 2, 3, int(rng.integers(1, 40))
+    sc = rng.random((B, H, n))
+    if seed % 2:                                  # heavy ties
+        sc = np.round(sc * 4) / 4
+    k, s, w = int(rng.integers(0, n + 3)), int(rng.integers(0, 4)), int(rng.integers(0, 5))
+    idx, cnt = orc.select_fixed(sc, budget=k, num_sink=s, window=w)
+    for b in range(B):
+        for h in range(H):
+            want = brute_fixed(sc[b, h], k, s, w)
+            c = cnt[b, h]
+            assert c == len(want) == min(k, n)
+            assert idx[b, h, :c].tolist() == want
+            assert np.all(idx[b, h, c:] == -1)
+
+
+def test_select_tie_rule_lower_index_wins():
+    sc = np.array([[[0.1, 0.3, 0.3, 0.3, 0.0, 0.0]]])
+    idx, _ = orc.select_fixed(sc, budget=2)
+    assert idx[0, 0].tolist() == [1, 2]
+    idx, _ = orc.select_fixed(sc, budget=5)
+    assert idx[0, 0].tolist() == [0, 1, 2, 3, 4]
+    idx, _ = orc.select_fixed(np.zeros((1, 1, 6)), budget=3, window=1)
+    assert idx[0, 0].tolist() == [0, 1, 5]
+    nan = np.array([[[np.nan, 0.5, np.nan, 0.25]]])
+    idx, _ = orc.select_fixed(nan, budget=3)
+    assert idx[0, 0].tolist() == [0, 1, 3]
+
+
+def test_select_forced_set_and_budget_edges():
+    rng = np.random.default_rng(12)
+    sc = rng.random((1, 1, 30))
+    idx, cnt = orc.select_fixed(sc, budget=10, num_sink=4, window=3)
+    got = idx[0, 0].tolist()
+    assert cnt[0, 0] == 10 and got == sorted(set(got))
+    assert {0, 1, 2, 3, 27, 28, 29} <= set(got)
+    # budget == |F|: nothing but forced tokens
+    idx, _ = orc.select_fixed(sc, budget=7, num_sink=4, window=3)
+    assert idx[0, 0].tolist() == [0, 1, 2, 3, 27, 28, 29]
+    # budget < |F|: window first, then sinks
+    idx, _ = orc.select_fixed(sc, budget=4, num_sink=4, window=3)
+    assert idx[0, 0].tolist() == [0, 27, 28, 29]
+    # budget >= n keeps everything
+    idx, cnt = orc.select_fixed(sc, budget=64)
+    assert cnt[0, 0] == 30 and idx[0, 0, :30].tolist() == list(range(30))
+    # per-head budgets
+    sc2 = rng.random((1, 3, 30))
+    hb = np.array([[5, 0, 9]], dtype=np.int32)
+    idx, cnt = orc.select_fixed(sc2, budget=9, head_budgets=hb)
+    assert cnt[0].tolist() == [5, 0, 9]
+    for h in range(3):
+        assert idx[0, h, : hb[0, h]].tolist() == brute_fixed(sc2[0, h], hb[0, h], 0, 0)
+
+
+# ---------------------------------------------------------------- AdaCurDKV
+
+def brute_adaptive(sc, k, s, w, alpha):
+    H, n = sc.shape
+    k_eff = min(k, n)
+    forced = brute_fixed(np.zeros(n), 0, 0, 0)
+    forced = []
+    for j in range(n - 1, max(n - w, 0) - 1, -1):
+        if len(forced) < k_eff:
+            forced.append(j)
+    for j in range(min(s, n)):
+        if j not in forced and len(forced) < k_eff:
+            forced.append(j)
+    p = min(max(int(np.floor(alpha * k)), len(forced)), k_eff)
+    keep = [set(forced) for _ in range(H)]
+    pool = []
+    for h in range(H):
+        cand = sorted((j for j in range(n) if j not in forced), key=lambda j: (-sc[h, j], j))
+        keep[h] |= set(cand[: p - len(forced)])
+        pool += [(-sc[h, j], h, j) for j in cand[p - len(forced):]]
+    pool.sort()
+    for _, h, j in pool[: H * (k_eff - p)]:
+        keep[h].add(j)
+    return [sorted(x) for x in keep]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_select_adaptive_matches_brute_force(seed):
+    rng = np.random.default_rng(200 + seed)
+    B, H, n = 2, int(rng.integers(1, 5)), int(rng.integers(2, 40))
+    sc = rng.random((B, H, n)) * rng.random((B, H, 1))      # heads with different mass
+    if seed % 2:
+        sc = np.round(sc * 8) / 8
+    k, s, w = int(rng.integers(1, n + 2)), int(rng.integers(0, 3)), int(rng.integers(0, 4))
+    alpha = float(rng.choice([0.0, 0.2, 0.5, 1.0]))
+    idx, cnt, off = orc.select_adaptive(sc, budget=k, num_sink=s, window=w, alpha=alpha)
+    assert off[0] == 0 and off[-1] == len(idx) == B * H * min(k, n)
+    for b in range(B):
+        want = brute_adaptive(sc[b], k, s, w, alpha)
+        for h in range(H):
+            o = off[b * H + h]
+            assert cnt[b, h] == len(want[h]) == off[b * H + h + 1] - o
+            assert idx[o:o + cnt[b, h]].tolist() == want[h]
+
+
+def test_adaptive_invariants_and_special_cases():
+    rng = np.random.default_rng(13)
+    B, H, n, k, w = 2, 4, 64, 16, 3
+    sc = rng.random((B, H, n)) * np.array([1.0, 0.1, 5.0, 0.01])[None, :, None]
+    idx, cnt, off = orc.select_adaptive(sc, budget=k, window=w, alpha=0.2)
+    assert np.all(cnt.sum(-1) == H * k)
+    assert np.all(cnt >= max(int(np.floor(0.2 * k)), w))
+    assert cnt[0, 2] > cnt[0, 0] > cnt[0, 1] >= cnt[0, 3]
+    # alpha = 1 and H = 1 reduce to the fixed-budget selection
+    fidx, fcnt = orc.select_fixed(sc, budget=k, window=w)
+    idx1, cnt1, off1 = orc.select_adaptive(sc, budget=k, window=w, alpha=1.0)
+    assert np.all(cnt1 == k) and idx1.tolist() == fidx.reshape(-1).tolist()
+    one = sc[:, :1]
+    fidx, _ = orc.select_fixed(one, budget=k, window=w)
+    idx2, cnt2, _ = orc.select_adaptive(one, budget=k, window=w, alpha=0.2)
+    assert idx2.tolist() == fidx.reshape(-1).tolist()
+    # all the score mass in one head: it receives the whole pooled remainder
+    sc3 = np.zeros((1, H, n))
+    sc3[0, 1] = rng.random(n) + 1.0
+    _, cnt3, _ = orc.select_adaptive(sc3, budget=k, window=w, alpha=0.25)
+    p = max(int(np.floor(0.25 * k)), w)
+    assert cnt3[0].tolist() == [p, p + H * (k - p), p, p]
+
+
+# ---------------------------------------------------------------- gather, GQA, bytes
+
+def test_compact_is_byte_exact_indexing():
+    rng = np.random.default_rng(14)
+    B, H, n, d = 2, 3, 25, 8
+    K, V = rand_kv(rng, B, H, n, d)
+    sc = rng.random((B, H, n))
+    idx, cnt = orc.select_fixed(sc, budget=6, window=2)
+    Ko, Vo = orc.compact(K, V, idx, cnt)
+    for b in range(B):
+        for h in range(H):
+            np.testing.assert_array_equal(Ko[b, h], K[b, h, idx[b, h]])
+            np.testing.assert_array_equal(Vo[b, h], V[b, h, idx[b, h]])
+    pidx, pcnt, poff = orc.select_adaptive(sc, budget=6, window=2, alpha=0.2)
+    Kp, Vp = orc.compact(K, V, pidx, pcnt, poff)
+    for b in range(B):
+        for h in range(H):
+            o, c = poff[b * H + h], pcnt[b, h]
+            np.testing.assert_array_equal(Kp[o:o + c], K[b, h, pidx[o:o + c]])
+            np.testing.assert_array_equal(Vp[o:o + c], V[b, h, pidx[o:o + c]])
+
+
+def test_gqa_group_map():
+    assert [orc.kv_head_of_query(q, 32, 8) for q in (0, 3, 4, 31)] == [0, 0, 1, 7]
+    assert [orc.kv_head_of_query(q, 8, 8) for q in range(8)] == list(range(8))
+
+
+def test_cache_byte_accounting_matches_paper_128k_figure():
+    """A 131072-token LLaMA-3.1-8B cache in bf16 is 16 GiB (the appendix's "approximately
+    16 GB"); at 128,000 tokens the same formula gives 15.6 GiB (the main text's figure,
+    Sec. 4.4)."""
+    w = synth.CONFIGS["cfg4"]
+    per_token = w.layers * w.batch * w.kv_heads * w.d * 2 * 2      # K and V, 2 bytes each
+    assert per_token * w.n_max == 16 * 2 ** 30
+    assert round(per_token * 128_000 / 2 ** 30, 1) == 15.6
