@@ -1,0 +1,153 @@
+/*
+ * curdkv.h -- C ABI of the B200 (sm_100a) implementation of CurDKV / AdaCurDKV
+ * prefill-time KV-cache selection ("Value-Guided KV Compression for LLMs via
+ * Approximated CUR Decomposition", Algorithm 1 and Sec. 3.2).
+ *
+ * For every (batch element, KV head) the library
+ *   1. sketches the bf16 key and value matrices with a caller-supplied Gaussian
+ *      matrix G and takes squared sketch-row norms (Alg. 1 lines 2-4),
+ *   2. multiplies key and value scores and normalises them per head (lines 5-6),
+ *   3. keeps the sink and recent-window tokens and the top-scoring rest
+ *      (lines 7-9), with a fixed budget per head or AdaCurDKV's layer-wide
+ *      adaptive budgets (Sec. 3.2, "Adaptive budget allocation"),
+ *   4. gathers the surviving rows into a compacted cache (line 10).
+ *
+ * General conventions
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned
+ *     by the caller.  The library never allocates or frees device memory and
+ *     never retains a pointer after a call returns.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     All work is enqueued on it; calls return without synchronising unless
+ *     stated otherwise.
+ *   - Return codes report errors the host can see (bad arguments, unsupported
+ *     shapes, small workspace, launch failure).  Anomalies seen on the device
+ *     (an out-of-range index, a bounded wait that ran out) are OR-ed into a
+ *     status word at the start of the workspace; read it with
+ *     curdkv_device_status().  No kernel traps or spins without limit.
+ *   - Layers of a model may be folded into the batch axis: every batch element
+ *     is an independent group of `kv_heads` problems.
+ *   - Results are deterministic: identical inputs give bit-identical outputs.
+ */
+#ifndef CURDKV_H_
+#define CURDKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum curdkv_status {
+  CURDKV_OK = 0,
+  CURDKV_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, budget < 0, alpha outside [0,1] ... */
+  CURDKV_ERR_UNSUPPORTED = 2, /* shape outside what the kernels handle (see curdkv_score)       */
+  CURDKV_ERR_WORKSPACE = 3,   /* workspace smaller than curdkv_workspace_bytes()                 */
+  CURDKV_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed                               */
+  CURDKV_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (from the status word)       */
+} curdkv_status;
+
+/* Bits of the device status word (workspace[0], int32). */
+#define CURDKV_DEV_TIMEOUT 0x1u   /* a pipeline wait gave up; results of that launch are invalid */
+#define CURDKV_DEV_BAD_INDEX 0x2u /* an index outside [0, n) was skipped by the gather           */
+
+/* Shape of one call: K and V are bf16 tensors addressed as
+ *   K[b][h][j][c] = K_base[b*k_stride_b + h*k_stride_h + j*k_stride_n + c]
+ * with strides in ELEMENTS, c contiguous; b < batch, h < kv_heads, j < n_max,
+ * c < d.  Base addresses and all strides times 2 bytes must be multiples of 16.
+ * (K in R^{g x n x d} of Alg. 1 with g = kv_heads, one such group per batch
+ * element.) */
+typedef struct curdkv_desc {
+  int32_t batch;          /* independent (layer, sequence) groups                           */
+  int32_t kv_heads;       /* g: KV groups per batch element                                 */
+  int32_t q_heads;        /* query heads; a multiple of kv_heads (GQA), informational       */
+  int32_t n_max;          /* rows allocated per (b, h)                                      */
+  int32_t d;              /* head dimension                                                 */
+  int32_t r;              /* sketch dimension (columns of G)                                */
+  int64_t k_stride_b, k_stride_h, k_stride_n;
+  int64_t v_stride_b, v_stride_h, v_stride_n;
+  const int32_t* seqlens; /* device int32 [batch]: valid rows n_b (clamped to [0, n_max]),
+                             or NULL when every sequence has n_max rows                     */
+  int32_t score_mode;     /* 0: l = lK * lV (Alg. 1 line 5)  1: key only  2: value only
+                             (ablation of App. C.3)                                         */
+  int32_t use_projection; /* 1: sketch with G (Alg. 1 lines 2-3); 0: raw squared row norms  */
+} curdkv_desc;
+
+/* Bytes of device workspace the calls below need for this shape (256-byte
+ * aligned base required).  `max_budget` and `adaptive` describe the largest
+ * selection that will be requested.  Returns 0 for an invalid descriptor. */
+size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32_t adaptive);
+
+/* Alg. 1 lines 2-6: scores[b][h][j] = lK_j * lV_j / sum_j(lK_j * lV_j) with
+ * lK_j = ||K[b][h][j] G||^2, lV_j = ||V[b][h][j] G||^2 (fp32 accumulation).
+ *   G          fp32 [d][r] row-major shared by all heads (g_per_head = 0) or
+ *              [kv_heads][d][r] (g_per_head = 1); the same G for K and V.
+ *              Entries are expected ~N(0, 1/r) but any finite values work.
+ *   scores     fp32 [batch][kv_heads][n_max]; entries j >= n_b are set to 0.
+ *   head_sums  fp32 [batch][kv_heads]: the normaliser sum_j lK_j*lV_j.
+ * Clears the device status word first.  Supported: d = 128, 1 <= r <= 64 with
+ * projection; d % 8 == 0, d <= 1024 without.  Anything else returns
+ * CURDKV_ERR_UNSUPPORTED and enqueues nothing. */
+curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
+                           const curdkv_desc* desc, float* scores, float* head_sums,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Alg. 1 lines 7-9 (adaptive = 0) or AdaCurDKV (adaptive = 1).
+ * Forced set of a sequence of n_b rows: the last `window` rows and the first
+ * `num_sink` rows; if the budget cannot hold them all, the most recent window
+ * rows come first, then sinks in index order.  Ties between equal scores go
+ * to the lower token index (adaptive: lower head first, then lower index).
+ * NaN or non-positive scores rank as 0.
+ *   budget        k: rows kept per head, forced rows included; min(k, n_b) are kept
+ *   head_budgets  adaptive = 0 only: NULL, or int32 [batch][kv_heads] per-head k
+ *                 (each clamped to [0, budget])
+ *   alpha         adaptive = 1 only: safeguard in [0,1]; every head keeps at least
+ *                 min(max(floor(alpha*k), forced), min(k, n_b)) rows, the rest of the
+ *                 layer total kv_heads*min(k, n_b) goes to the globally best rows
+ *   idx           adaptive = 0: int32 [batch][kv_heads][budget], ascending token
+ *                 index, unused tail = -1.  adaptive = 1: packed, head (b,h)
+ *                 occupies idx[head_offsets[b*kv_heads+h] ...], ascending; capacity
+ *                 batch*kv_heads*min(budget, n_max) entries.
+ *   head_counts   int32 [batch][kv_heads]: rows kept per head
+ *   head_offsets  int32 [batch*kv_heads + 1]: row of idx where each head starts.
+ *                 adaptive = 1: exclusive prefix sums of head_counts (required);
+ *                 adaptive = 0: p*budget, written only if not NULL
+ * adaptive = 1 supports kv_heads <= 16. */
+curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_t budget,
+                            const int32_t* head_budgets, int32_t num_sink, int32_t window,
+                            int32_t adaptive, double alpha, int32_t* idx, int32_t* head_counts,
+                            int32_t* head_offsets, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream);
+
+/* Alg. 1 line 10: K_out[row] = K[b][h][idx[...]], V_out likewise (byte copies).
+ *   out_stride_h > 0  fixed layout: idx is [batch][kv_heads][idx_stride]; row t of
+ *                     head (b,h) goes to output row (b*kv_heads+h)*out_stride_h + t
+ *   out_stride_h = 0  packed layout: head (b,h) starts at row head_offsets[b*kv_heads+h]
+ *                     of both idx and the outputs
+ * Output rows are d contiguous bf16.  Rows beyond head_counts are left
+ * untouched.  An index outside [0, n_b) is skipped and flagged in the status
+ * word (workspace may be NULL: then it is only skipped). */
+curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* desc,
+                             const int32_t* idx, int64_t idx_stride, const int32_t* head_counts,
+                             const int32_t* head_offsets, void* K_out, void* V_out,
+                             int64_t out_stride_h, void* workspace, void* cuda_stream);
+
+/* GQA (Sec. 3.2): query head q uses KV head q / (q_heads / kv_heads).  Writes
+ * kv_head_of_q int32 [q_heads] (device) so that attention consumers can index
+ * the shared selection without replicating the compacted cache. */
+curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, void* cuda_stream);
+
+/* Copies the device status word to *host_flags (host pointer) after
+ * synchronising the stream.  Returns CURDKV_ERR_TIMEOUT if the timeout bit is
+ * set, CURDKV_OK otherwise (other bits are reported through *host_flags). */
+curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, void* cuda_stream);
+
+/* Number of kernels this library has launched in this process so far. */
+uint64_t curdkv_launch_count(void);
+
+const char* curdkv_status_string(curdkv_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CURDKV_H_ */

@@ -1,0 +1,207 @@
+"""Thin ctypes binding of ``libcurdkv.so`` (declared in ``include/curdkv.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch supplies device memory and the current stream.  There is no
+CPU or eager fallback: if the library is missing or a call fails, an exception
+is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libcurdkv.so"
+_lib = None
+
+STATUS_OK = 0
+DEV_TIMEOUT = 0x1
+DEV_BAD_INDEX = 0x2
+
+EXPORTS = (
+    "curdkv_workspace_bytes", "curdkv_score", "curdkv_select", "curdkv_compact",
+    "curdkv_gqa_map", "curdkv_device_status", "curdkv_launch_count", "curdkv_status_string",
+)
+
+
+class CurdkvError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {status_string(code)} (status {code})")
+        self.code = code
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("kv_heads", ctypes.c_int32), ("q_heads", ctypes.c_int32),
+        ("n_max", ctypes.c_int32), ("d", ctypes.c_int32), ("r", ctypes.c_int32),
+        ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_n", ctypes.c_int64),
+        ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_n", ctypes.c_int64),
+        ("seqlens", ctypes.c_void_p),
+        ("score_mode", ctypes.c_int32), ("use_projection", ctypes.c_int32),
+    ]
+
+
+def load():
+    """Load the CUDA library (built by ``python -m paper_2509_15038_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2509_15038_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    dp = ctypes.POINTER(Desc)
+    lib.curdkv_workspace_bytes.restype = ctypes.c_size_t
+    lib.curdkv_workspace_bytes.argtypes = [dp, i32, i32]
+    lib.curdkv_score.restype = ctypes.c_int
+    lib.curdkv_score.argtypes = [vp, vp, vp, i32, dp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.curdkv_select.restype = ctypes.c_int
+    lib.curdkv_select.argtypes = [vp, dp, i32, vp, i32, i32, i32, ctypes.c_double, vp, vp, vp, vp,
+                                  ctypes.c_size_t, vp]
+    lib.curdkv_compact.restype = ctypes.c_int
+    lib.curdkv_compact.argtypes = [vp, vp, dp, vp, i64, vp, vp, vp, vp, i64, vp, vp]
+    lib.curdkv_gqa_map.restype = ctypes.c_int
+    lib.curdkv_gqa_map.argtypes = [dp, vp, vp]
+    lib.curdkv_device_status.restype = ctypes.c_int
+    lib.curdkv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.curdkv_launch_count.restype = ctypes.c_uint64
+    lib.curdkv_launch_count.argtypes = []
+    lib.curdkv_status_string.restype = ctypes.c_char_p
+    lib.curdkv_status_string.argtypes = [ctypes.c_int]
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().curdkv_status_string(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(load().curdkv_launch_count())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    # an empty view of a live allocation still has a valid base address
+    return ctypes.c_void_p(t.data_ptr() if t.numel() else t.untyped_storage().data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, what: str):
+    if code != STATUS_OK:
+        raise CurdkvError(code, what)
+
+
+def make_desc(K: torch.Tensor, V: torch.Tensor, r: int, *, q_heads: Optional[int] = None,
+              seqlens: Optional[torch.Tensor] = None, score_mode: int = 0,
+              use_projection: int = 1) -> Desc:
+    """Descriptor of bf16 K, V ``[B, Hkv, n_max, d]`` (any strides with d contiguous)."""
+    if K.dtype != torch.bfloat16 or V.dtype != torch.bfloat16:
+        raise TypeError("K and V must be bf16")
+    if K.dim() != 4 or K.shape != V.shape or K.stride(3) != 1 or V.stride(3) != 1:
+        raise ValueError("K and V must be [B, Hkv, n, d] with a contiguous last axis")
+    if seqlens is not None and (seqlens.dtype != torch.int32 or seqlens.numel() != K.shape[0]
+                                or not seqlens.is_contiguous()):
+        raise ValueError("seqlens must be a contiguous int32 tensor of length B")
+    B, H, n, d = K.shape
+    return Desc(B, H, q_heads or H, n, d, int(r),
+                K.stride(0), K.stride(1), K.stride(2), V.stride(0), V.stride(1), V.stride(2),
+                seqlens.data_ptr() if seqlens is not None else None,
+                int(score_mode), int(use_projection))
+
+
+def workspace_bytes(desc: Desc, max_budget: int = 0, adaptive: bool = False) -> int:
+    return int(load().curdkv_workspace_bytes(ctypes.byref(desc), int(max_budget), int(adaptive)))
+
+
+def alloc_workspace(desc: Desc, max_budget: int = 0, adaptive: bool = False, device=None) -> torch.Tensor:
+    nbytes = workspace_bytes(desc, max_budget, adaptive)
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device or "cuda")
+
+
+def curdkv_score(K, V, G, desc: Desc, workspace: torch.Tensor, scores=None, head_sums=None):
+    """Alg. 1 lines 2-6.  G: fp32 device tensor [d, r] or [Hkv, d, r].  Returns (scores, head_sums)."""
+    dev = K.device
+    if scores is None:
+        scores = torch.empty((desc.batch, desc.kv_heads, desc.n_max), dtype=torch.float32, device=dev)
+    if head_sums is None:
+        head_sums = torch.empty((desc.batch, desc.kv_heads), dtype=torch.float32, device=dev)
+    g_per_head = int(G is not None and G.dim() == 3)
+    if G is not None and (G.dtype != torch.float32 or not G.is_contiguous()):
+        raise TypeError("G must be a contiguous fp32 tensor")
+    code = load().curdkv_score(_ptr(K), _ptr(V), _ptr(G), g_per_head, ctypes.byref(desc),
+                               _ptr(scores), _ptr(head_sums), _ptr(workspace),
+                               workspace.numel(), _stream())
+    _check(code, "curdkv_score")
+    return scores, head_sums
+
+
+def curdkv_select(scores, desc: Desc, budget: int, *, num_sink: int = 0, window: int = 0,
+                  head_budgets=None, adaptive: bool = False, alpha: float = 0.2,
+                  workspace: Optional[torch.Tensor] = None, idx=None, head_counts=None,
+                  head_offsets=None):
+    """Alg. 1 lines 7-9 / AdaCurDKV.  Returns (idx, head_counts, head_offsets)."""
+    dev = scores.device
+    P = desc.batch * desc.kv_heads
+    if idx is None:
+        if adaptive:
+            idx = torch.empty((P * max(min(budget, desc.n_max), 0) + 1,), dtype=torch.int32, device=dev)[:-1]
+        else:
+            idx = torch.empty((P * max(budget, 0) + 1,), dtype=torch.int32, device=dev)
+            idx = idx[: P * max(budget, 0)].view(desc.batch, desc.kv_heads, max(budget, 0))
+    if head_counts is None:
+        head_counts = torch.empty((desc.batch, desc.kv_heads), dtype=torch.int32, device=dev)
+    if head_offsets is None:
+        head_offsets = torch.empty((P + 1,), dtype=torch.int32, device=dev)
+    code = load().curdkv_select(_ptr(scores), ctypes.byref(desc), int(budget), _ptr(head_budgets),
+                                int(num_sink), int(window), int(adaptive), float(alpha),
+                                _ptr(idx), _ptr(head_counts), _ptr(head_offsets), _ptr(workspace),
+                                0 if workspace is None else workspace.numel(), _stream())
+    _check(code, "curdkv_select")
+    return idx, head_counts, head_offsets
+
+
+def curdkv_compact(K, V, desc: Desc, idx, head_counts, head_offsets=None, *, packed: bool = False,
+                   K_out=None, V_out=None, workspace: Optional[torch.Tensor] = None):
+    """Alg. 1 line 10.  Fixed layout -> [B, Hkv, budget, d]; packed -> [capacity, d]."""
+    dev = K.device
+    if packed:
+        rows = idx.numel()
+        shape, out_stride_h, idx_stride = (rows, desc.d), 0, 0
+    else:
+        budget = idx.shape[-1]
+        shape, out_stride_h, idx_stride = (desc.batch, desc.kv_heads, budget, desc.d), budget, budget
+    if K_out is None:
+        K_out = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+    if V_out is None:
+        V_out = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+    if not packed and out_stride_h == 0:
+        return K_out, V_out
+    code = load().curdkv_compact(_ptr(K), _ptr(V), ctypes.byref(desc), _ptr(idx), idx_stride,
+                                 _ptr(head_counts), _ptr(head_offsets), _ptr(K_out), _ptr(V_out),
+                                 out_stride_h, _ptr(workspace), _stream())
+    _check(code, "curdkv_compact")
+    return K_out, V_out
+
+
+def curdkv_gqa_map(desc: Desc, device="cuda") -> torch.Tensor:
+    out = torch.empty((desc.q_heads,), dtype=torch.int32, device=device)
+    _check(load().curdkv_gqa_map(ctypes.byref(desc), _ptr(out), _stream()), "curdkv_gqa_map")
+    return out
+
+
+def curdkv_device_status(workspace: torch.Tensor) -> int:
+    """Synchronises the current stream and returns the device status flags."""
+    flags = ctypes.c_uint32(0)
+    code = load().curdkv_device_status(_ptr(workspace), ctypes.byref(flags), _stream())
+    if code not in (STATUS_OK, 5):
+        raise CurdkvError(code, "curdkv_device_status")
+    return int(flags.value)

@@ -1,0 +1,72 @@
+// Gather of the selected rows into the compacted cache (Alg. 1 line 10):
+// byte copies with 16-byte vectors, a half-warp per row (K in lanes 0-15, V in
+// lanes 16-31), four rows in flight per warp.
+#pragma once
+#include "common.cuh"
+
+namespace curdkv {
+
+struct CompactArgs {
+  KvView K, V;
+  const int32_t* seqlens;
+  int heads, n_max, d;
+  const int32_t* idx;
+  int64_t idx_stride;
+  const int32_t* counts;
+  const int32_t* offsets;
+  __nv_bfloat16* K_out;
+  __nv_bfloat16* V_out;
+  int64_t out_stride_h;     // > 0: fixed layout, 0: packed
+  uint32_t* status;
+};
+
+constexpr int kCompactWarps = 8;
+constexpr int kCompactRowsPerWarp = 4;
+constexpr int kCompactRowsPerCta = kCompactWarps * kCompactRowsPerWarp;
+
+// grid = batch*heads*ctas_per_head; the CTAs of a head stride over its rows.
+__global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const CompactArgs a,
+                                                                     const int ctas_per_head) {
+  const int p = blockIdx.x / ctas_per_head, part = blockIdx.x % ctas_per_head;
+  const int b = p / a.heads, h = p % a.heads;
+  const int n = seq_len_of(a.seqlens, b, a.n_max);
+  const int count = a.counts[p];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+  const bool fixed = a.out_stride_h > 0;
+  const int32_t* ix = fixed ? a.idx + (size_t)p * a.idx_stride : a.idx + a.offsets[p];
+  const size_t out_row0 = fixed ? (size_t)p * a.out_stride_h : (size_t)a.offsets[p];
+  const KvView& T = half ? a.V : a.K;
+  const __nv_bfloat16* src = T.base + b * T.stride_b + h * T.stride_h;
+  __nv_bfloat16* dst = (half ? a.V_out : a.K_out) + out_row0 * a.d;
+  const int chunks = a.d >> 3;
+
+  for (int t0 = (part * kCompactWarps + warp) * kCompactRowsPerWarp; t0 < count;
+       t0 += ctas_per_head * kCompactRowsPerCta) {
+    int j[kCompactRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kCompactRowsPerWarp; ++i) {
+      j[i] = t0 + i < count ? __ldg(ix + t0 + i) : -1;
+      if (t0 + i < count && (j[i] < 0 || j[i] >= n)) {
+        if (lane == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+        j[i] = -1;
+      }
+    }
+    for (int c = l16; c < chunks; c += 16) {
+      uint4 v[kCompactRowsPerWarp];
+#pragma unroll
+      for (int i = 0; i < kCompactRowsPerWarp; ++i)
+        if (j[i] >= 0) v[i] = __ldg(reinterpret_cast<const uint4*>(src + j[i] * T.stride_n) + c);
+#pragma unroll
+      for (int i = 0; i < kCompactRowsPerWarp; ++i)
+        if (j[i] >= 0) __stcs(reinterpret_cast<uint4*>(dst + (size_t)(t0 + i) * a.d) + c, v[i]);
+    }
+  }
+}
+
+// GQA group map (Sec. 3.2): query head q reads KV head q / (q_heads / kv_heads).
+__global__ void gqa_map_kernel(int32_t* kv_head_of_q, int q_heads, int kv_heads) {
+  const int q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q < q_heads) kv_head_of_q[q] = q / (q_heads / kv_heads);
+}
+
+}  // namespace curdkv

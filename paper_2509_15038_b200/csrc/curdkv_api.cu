@@ -1,0 +1,227 @@
+// C ABI of the CurDKV library: argument checks and kernel launches.
+#include <atomic>
+#include <cstdint>
+
+#include "common.cuh"
+#include "compact.cuh"
+#include "score_simt.cuh"
+#include "select.cuh"
+
+namespace {
+
+using namespace curdkv;
+
+std::atomic<uint64_t> g_launches{0};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool launch_ok() {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess;
+}
+
+curdkv_status check_desc(const curdkv_desc* d) {
+  if (d == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (d->batch < 0 || d->kv_heads < 1 || d->n_max < 0 || d->d < 1) return CURDKV_ERR_INVALID_ARG;
+  if (d->q_heads < d->kv_heads || d->q_heads % d->kv_heads != 0) return CURDKV_ERR_INVALID_ARG;
+  if (d->score_mode < 0 || d->score_mode > 2) return CURDKV_ERR_INVALID_ARG;
+  if (d->use_projection != 0 && d->use_projection != 1) return CURDKV_ERR_INVALID_ARG;
+  if ((int64_t)d->batch * d->kv_heads > (int64_t)1 << 24) return CURDKV_ERR_UNSUPPORTED;
+  return CURDKV_OK;
+}
+
+curdkv_status check_kv(const void* K, const void* V, const curdkv_desc* d) {
+  if (K == nullptr || V == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (d->d % 8 != 0 || d->d > 1024) return CURDKV_ERR_UNSUPPORTED;
+  if (!aligned16(K) || !aligned16(V)) return CURDKV_ERR_INVALID_ARG;
+  const int64_t s[6] = {d->k_stride_b, d->k_stride_h, d->k_stride_n,
+                        d->v_stride_b, d->v_stride_h, d->v_stride_n};
+  for (int64_t x : s)
+    if (x < 0 || x % 8 != 0) return CURDKV_ERR_INVALID_ARG;
+  if (d->k_stride_n < d->d || d->v_stride_n < d->d) return CURDKV_ERR_INVALID_ARG;
+  return CURDKV_OK;
+}
+
+inline int tiles_per_head(const curdkv_desc* d) { return (d->n_max + kTileRows - 1) / kTileRows; }
+
+inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
+
+KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
+  return KvView{static_cast<const __nv_bfloat16*>(base), sb, sh, sn};
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32_t adaptive) {
+  (void)max_budget;
+  (void)adaptive;
+  if (check_desc(desc) != CURDKV_OK) return 0;
+  const size_t tiles = (size_t)desc->batch * desc->kv_heads * tiles_per_head(desc);
+  return kStatusBytes + round256(tiles * sizeof(float));
+}
+
+curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
+                           const curdkv_desc* desc, float* scores, float* head_sums,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if ((st = check_kv(K, V, desc)) != CURDKV_OK) return st;
+  if (scores == nullptr || head_sums == nullptr || workspace == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (g_per_head != 0 && g_per_head != 1) return CURDKV_ERR_INVALID_ARG;
+  if (desc->use_projection) {
+    if (G == nullptr || desc->r < 1) return CURDKV_ERR_INVALID_ARG;
+    if (desc->d != 128 || desc->r > 64) return CURDKV_ERR_UNSUPPORTED;
+  }
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  if (workspace_bytes < curdkv_workspace_bytes(desc, 0, 0)) return CURDKV_ERR_WORKSPACE;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  const int tiles = tiles_per_head(desc);
+  if (P == 0 || tiles == 0) return CURDKV_OK;
+  if (P * tiles > 0x7fffffffLL) return CURDKV_ERR_UNSUPPORTED;
+
+  ScoreArgs a;
+  a.K = view_of(K, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n);
+  a.V = view_of(V, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n);
+  a.G = G;
+  a.g_per_head = g_per_head;
+  a.seqlens = desc->seqlens;
+  a.heads = desc->kv_heads;
+  a.n_max = desc->n_max;
+  a.d = desc->d;
+  a.r = desc->r;
+  a.tiles_per_head = tiles;
+  a.score_mode = desc->score_mode;
+  a.scores = scores;
+  a.tile_sums = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
+
+  const unsigned grid = (unsigned)(P * tiles);
+  if (desc->use_projection) {
+    const int r_pad = (desc->r + 31) / 32 * 32;
+    const size_t smem = 2 * (size_t)kTileRows * kFmaD * 2 + (size_t)kFmaD * r_pad * sizeof(float);
+    if (cudaFuncSetAttribute(sketch_fma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem) != cudaSuccess)
+      return CURDKV_ERR_CUDA;
+    sketch_fma_kernel<<<grid, 256, smem, stream>>>(a, r_pad);
+  } else {
+    row_norm_kernel<<<grid, 256, 0, stream>>>(a);
+  }
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+
+  const int chunks = (desc->n_max + kNormChunk - 1) / kNormChunk;
+  normalise_kernel<<<(unsigned)(P * chunks), 256, 0, stream>>>(scores, a.tile_sums, head_sums,
+                                                              desc->n_max, tiles, chunks);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_t budget,
+                            const int32_t* head_budgets, int32_t num_sink, int32_t window,
+                            int32_t adaptive, double alpha, int32_t* idx, int32_t* head_counts,
+                            int32_t* head_offsets, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if (scores == nullptr || idx == nullptr || head_counts == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (budget < 0 || num_sink < 0 || window < 0) return CURDKV_ERR_INVALID_ARG;
+  if (adaptive != 0 && adaptive != 1) return CURDKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  if (P == 0) return CURDKV_OK;
+  if (adaptive) {
+    if (!(alpha >= 0.0 && alpha <= 1.0) || head_offsets == nullptr || head_budgets != nullptr)
+      return CURDKV_ERR_INVALID_ARG;
+    return CURDKV_ERR_UNSUPPORTED;
+  }
+  select_fixed_kernel<<<(unsigned)P, kSelThreads, 0, stream>>>(
+      scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,
+      idx, head_counts, head_offsets);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* desc,
+                             const int32_t* idx, int64_t idx_stride, const int32_t* head_counts,
+                             const int32_t* head_offsets, void* K_out, void* V_out,
+                             int64_t out_stride_h, void* workspace, void* cuda_stream) {
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if ((st = check_kv(K, V, desc)) != CURDKV_OK) return st;
+  if (idx == nullptr || head_counts == nullptr || K_out == nullptr || V_out == nullptr)
+    return CURDKV_ERR_INVALID_ARG;
+  if (!aligned16(K_out) || !aligned16(V_out)) return CURDKV_ERR_INVALID_ARG;
+  if (out_stride_h < 0 || idx_stride < 0) return CURDKV_ERR_INVALID_ARG;
+  if (out_stride_h == 0 && head_offsets == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (out_stride_h > 0 && idx_stride == 0) return CURDKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  if (P == 0) return CURDKV_OK;
+
+  CompactArgs a;
+  a.K = view_of(K, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n);
+  a.V = view_of(V, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n);
+  a.seqlens = desc->seqlens;
+  a.heads = desc->kv_heads;
+  a.n_max = desc->n_max;
+  a.d = desc->d;
+  a.idx = idx;
+  a.idx_stride = idx_stride;
+  a.counts = head_counts;
+  a.offsets = head_offsets;
+  a.K_out = static_cast<__nv_bfloat16*>(K_out);
+  a.V_out = static_cast<__nv_bfloat16*>(V_out);
+  a.out_stride_h = out_stride_h;
+  a.status = static_cast<uint32_t*>(workspace);
+
+  // enough CTAs per head to cover a typical head in one sweep; larger heads loop
+  const int64_t rows_hint = out_stride_h > 0 ? out_stride_h : (idx_stride > 0 ? idx_stride : 1024);
+  int64_t ctas = (rows_hint + kCompactRowsPerCta - 1) / kCompactRowsPerCta;
+  if (ctas < 1) ctas = 1;
+  if (ctas > 256) ctas = 256;
+  while (P * ctas > 0x7fffffffLL) ctas >>= 1;
+  compact_kernel<<<(unsigned)(P * ctas), kCompactWarps * 32, 0, stream>>>(a, (int)ctas);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, void* cuda_stream) {
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if (kv_head_of_q == nullptr) return CURDKV_ERR_INVALID_ARG;
+  gqa_map_kernel<<<(desc->q_heads + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      kv_head_of_q, desc->q_heads, desc->kv_heads);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, void* cuda_stream) {
+  if (workspace == nullptr || host_flags == nullptr) return CURDKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(host_flags, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream) !=
+      cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+  return (*host_flags & CURDKV_DEV_TIMEOUT) ? CURDKV_ERR_TIMEOUT : CURDKV_OK;
+}
+
+uint64_t curdkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* curdkv_status_string(curdkv_status status) {
+  switch (status) {
+    case CURDKV_OK: return "ok";
+    case CURDKV_ERR_INVALID_ARG: return "invalid argument";
+    case CURDKV_ERR_UNSUPPORTED: return "unsupported shape";
+    case CURDKV_ERR_WORKSPACE: return "workspace too small";
+    case CURDKV_ERR_CUDA: return "CUDA call failed";
+    case CURDKV_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,227 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import curdkv_oracle as orc
+from paper_2509_15038_b200 import binding as cur
+from paper_2509_15038_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def gpu_score(K, V, G, seqlens=None, q_heads=None, score_mode=0, use_projection=1):
+    sl = None if seqlens is None else torch.as_tensor(seqlens, dtype=torch.int32, device=DEV)
+    Gd = None if G is None else torch.as_tensor(G, dtype=torch.float32, device=DEV).contiguous()
+    r = 1 if G is None else G.shape[-1]
+    desc = cur.make_desc(K, V, r, q_heads=q_heads, seqlens=sl, score_mode=score_mode,
+                         use_projection=use_projection)
+    ws = cur.alloc_workspace(desc)
+    scores, sums = cur.curdkv_score(K, V, Gd, desc, ws)
+    return desc, ws, scores, sums, sl
+
+
+def full_pipeline_check(K, V, G, budget, s, w, seqlens=None, what="", **kw):
+    desc, ws, scores, sums, sl = gpu_score(K, V, G, seqlens, **kw)
+    idx, cnt, _ = cur.curdkv_select(scores, desc, budget, num_sink=s, window=w, workspace=ws)
+    Ko, Vo = cur.curdkv_compact(K, V, desc, idx, cnt, workspace=ws)
+    assert cur.curdkv_device_status(ws) == 0
+
+    Ku, Vu = synth.to_u16(K), synth.to_u16(V)
+    rs, rS = orc.score(Ku, Vu, G if G is not None else np.zeros((K.shape[-1], 1), np.float32),
+                       seqlens=seqlens, score_mode=kw.get("score_mode", 0),
+                       use_projection=kw.get("use_projection", 1))
+    worst = pu.assert_scores_close(scores.cpu().numpy(), rs, what + " scores")
+    np.testing.assert_allclose(sums.cpu().numpy(), rS, rtol=1e-4)
+    ridx, rcnt = orc.select_fixed(rs, budget, num_sink=s, window=w, seqlens=seqlens)
+    gi, gc = idx.cpu().numpy(), cnt.cpu().numpy()
+    np.testing.assert_array_equal(gc, rcnt)
+    B, H, n_max, _ = K.shape
+    diffs = 0
+    for b in range(B):
+        n = n_max if seqlens is None else int(min(max(seqlens[b], 0), n_max))
+        for h in range(H):
+            c = rcnt[b, h]
+            forced = pu.forced_tokens(n, c, s, w)
+            diffs += pu.assert_selection_within_band(gi[b, h, :c], ridx[b, h, :c], rs[b, h], n, forced,
+                                                     f"{what} b={b} h={h}")
+            assert np.all(gi[b, h, c:] == -1)
+    # gathered bytes: exact copies of the rows the GPU selected
+    Kg, Vg = orc.compact(Ku, Vu, gi, gc)
+    np.testing.assert_array_equal(synth.to_u16(Ko), Kg)
+    np.testing.assert_array_equal(synth.to_u16(Vo), Vg)
+    # selection in the GPU's own precision: the oracle's rule on the fp32 scores is bit-exact
+    eidx, ecnt = orc.select_fixed(scores.cpu().numpy().astype(np.float64), budget, num_sink=s,
+                                  window=w, seqlens=seqlens)
+    np.testing.assert_array_equal(gi, eidx)
+    return worst, diffs
+
+
+def test_cfg1_full():
+    w = synth.CONFIGS["cfg1"]
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, w.r, seed=0)
+    worst, diffs = full_pipeline_check(K, V, G, w.budget, w.num_sink, w.window, what="cfg1")
+    assert worst < 1e-3
+
+
+def test_cfg2_two_layers():
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=2)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, w.r, seed=0)
+    full_pipeline_check(K, V, G, w.budget, w.num_sink, w.window, q_heads=w.q_heads, what="cfg2x2")
+
+
+def test_ragged_tail_and_sinks():
+    """n_max not a multiple of the 128-row tile, ragged lengths incl. 0, paper mode s = 4."""
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=5, n_max=1000)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, 32, seed=0)
+    lens = np.array([1000, 777, 128, 0, 1], dtype=np.int32)
+    for s, win, k in ((4, 0, 100), (4, 16, 100), (0, 32, 300), (4, 8, 10), (4, 8, 2000)):
+        full_pipeline_check(K, V, G, k, s, win, seqlens=lens, what=f"ragged s={s} w={win} k={k}")
+
+
+def test_strided_token_major_layout():
+    """K, V stored [B, n, H, d] (token-major) and viewed as [B, H, n, d]."""
+    B, H, n, d = 2, 4, 640, 128
+    g = torch.Generator(device=DEV).manual_seed(7)
+    Kb = torch.randn((B, n, H, d), generator=g, device=DEV).to(torch.bfloat16)
+    Vb = torch.randn((B, n, H, d), generator=g, device=DEV).to(torch.bfloat16)
+    K, V = Kb.permute(0, 2, 1, 3), Vb.permute(0, 2, 1, 3)
+    full_pipeline_check(K, V, synth.make_G(d, 32), 64, 0, 8, what="strided")
+
+
+@pytest.mark.parametrize("r", [20, 32, 64, 1])
+def test_sketch_dims(r):
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, n_max=1536, kv_heads=3, q_heads=3)
+    K, V, _ = synth.make_kv(w, DEV)
+    full_pipeline_check(K, V, synth.make_G(w.d, r, seed=r), 200, 4, 32, what=f"r={r}")
+
+
+def test_per_head_G():
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=2, n_max=512, kv_heads=4, q_heads=4)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, 32, seed=3, heads=4)
+    full_pipeline_check(K, V, G, 100, 0, 16, what="per-head G")
+
+
+@pytest.mark.parametrize("mode,proj", [(1, 1), (2, 1), (0, 0), (1, 0), (2, 0)])
+def test_ablation_modes(mode, proj):
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, n_max=900, kv_heads=2, q_heads=2)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, 32) if proj else None
+    full_pipeline_check(K, V, G, 90, 4, 16, score_mode=mode, use_projection=proj,
+                        what=f"mode={mode} proj={proj}")
+
+
+def test_orthogonal_G_closed_form_on_gpu():
+    """G = I (r = d... here the first 64 coordinates): scores are partial row norms."""
+    w = synth.shrink(synth.CONFIGS["cfg1"], n_max=384, kv_heads=2, q_heads=2)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = np.zeros((128, 64), dtype=np.float32)
+    G[:64, :64] = np.eye(64)
+    desc, ws, scores, sums, _ = gpu_score(K, V, G, score_mode=1)
+    want = (synth.u16_to_f64(synth.to_u16(K))[..., :64] ** 2).sum(-1)
+    want /= want.sum(-1, keepdims=True)
+    pu.assert_scores_close(scores.cpu().numpy(), want, "selector G")
+
+
+def _select_case(scores_np, budget, s, w, seqlens=None, head_budgets=None):
+    B, H, n = scores_np.shape
+    sc = torch.as_tensor(scores_np, dtype=torch.float32, device=DEV)
+    dummy = torch.empty((B, H, n, 8), dtype=torch.bfloat16, device=DEV)
+    sl = None if seqlens is None else torch.as_tensor(seqlens, dtype=torch.int32, device=DEV)
+    desc = cur.make_desc(dummy, dummy, 1, seqlens=sl)
+    hb = None if head_budgets is None else torch.as_tensor(head_budgets, dtype=torch.int32, device=DEV)
+    idx, cnt, _ = cur.curdkv_select(sc, desc, budget, num_sink=s, window=w, head_budgets=hb)
+    ridx, rcnt = orc.select_fixed(sc.cpu().numpy().astype(np.float64), budget, num_sink=s, window=w,
+                                  seqlens=seqlens, head_budgets=head_budgets)
+    np.testing.assert_array_equal(cnt.cpu().numpy(), rcnt)
+    np.testing.assert_array_equal(idx.cpu().numpy(), ridx)
+
+
+def test_select_edges_and_ties():
+    rng = np.random.default_rng(0)
+    sc = rng.random((2, 3, 5000)).astype(np.float32)
+    for k, s, w in ((0, 0, 0), (1, 0, 0), (7, 4, 3), (6, 4, 3), (4999, 0, 0), (5000, 2, 2), (9000, 0, 0)):
+        _select_case(sc, k, s, w)
+    tied = (np.round(sc * 16) / 16).astype(np.float32)          # heavy ties incl. zeros
+    for k in (10, 1000, 2500):
+        _select_case(tied, k, 2, 5)
+    _select_case(np.zeros((1, 2, 300), np.float32), 17, 0, 4)
+    weird = sc.copy()
+    weird[0, 0, ::7] = np.nan
+    weird[0, 1, ::5] = -1.0
+    weird[1, 2, 3] = np.inf
+    _select_case(weird, 600, 1, 1)
+    _select_case(sc, 800, 3, 9, seqlens=np.array([4097, 33], dtype=np.int32))
+    _select_case(sc, 800, 0, 9, head_budgets=np.array([[800, 0, 13], [5000, 77, 1]], dtype=np.int32))
+    tiny = rng.random((1, 1, 3)).astype(np.float32) * 1e-30      # tiny positive values keep their order
+    _select_case(tiny, 2, 0, 0)
+
+
+def test_select_long_rows():
+    rng = np.random.default_rng(1)
+    sc = (rng.random((1, 2, 131072)) ** 8).astype(np.float32)
+    sc /= sc.sum(-1, keepdims=True)
+    _select_case(sc, 6681, 0, 128)
+    _select_case(sc, 6681, 4, 0)
+
+
+def test_compact_flags_bad_index_without_faulting():
+    B, H, n, d = 1, 2, 64, 128
+    K = torch.randn((B, H, n, d), device=DEV).to(torch.bfloat16)
+    V = torch.randn((B, H, n, d), device=DEV).to(torch.bfloat16)
+    desc = cur.make_desc(K, V, 32)
+    ws = cur.alloc_workspace(desc)
+    ws.zero_()
+    idx = torch.tensor([[[0, 5, -1, 63], [1, 64, 2, 3]]], dtype=torch.int32, device=DEV)
+    cnt = torch.full((B, H), 4, dtype=torch.int32, device=DEV)
+    Ko, Vo = cur.curdkv_compact(K, V, desc, idx, cnt, workspace=ws)
+    assert cur.curdkv_device_status(ws) & cur.DEV_BAD_INDEX
+    assert torch.equal(Ko[0, 0, 1], K[0, 0, 5]) and torch.equal(Vo[0, 1, 3], V[0, 1, 3])
+    assert torch.all(Ko[0, 0, 2] == 0) and torch.all(Vo[0, 1, 1] == 0)
+
+
+def test_invalid_arguments_return_status_codes():
+    K = torch.zeros((1, 2, 256, 128), dtype=torch.bfloat16, device=DEV)
+    G = torch.zeros((128, 32), dtype=torch.float32, device=DEV)
+    desc = cur.make_desc(K, K, 32)
+    ws = cur.alloc_workspace(desc)
+    before = cur.launch_count()
+    with pytest.raises(cur.CurdkvError) as e:
+        cur.curdkv_score(K, K, None, desc, ws)
+    assert e.value.code == 1
+    with pytest.raises(cur.CurdkvError) as e:
+        cur.curdkv_score(K, K, G, desc, ws[:256])
+    assert e.value.code == 3
+    bad = cur.make_desc(K, K, 200)
+    with pytest.raises(cur.CurdkvError) as e:
+        cur.curdkv_score(K, K, G, bad, ws)
+    assert e.value.code == 2
+    scores = torch.zeros((1, 2, 256), device=DEV)
+    with pytest.raises(cur.CurdkvError) as e:
+        cur.curdkv_select(scores, desc, -1)
+    assert e.value.code == 1
+    with pytest.raises(cur.CurdkvError) as e:
+        cur.curdkv_select(scores, desc, 8, adaptive=True, alpha=1.5)
+    assert e.value.code == 1
+    assert cur.launch_count() == before
+
+
+def test_determinism_and_gqa_map():
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=2, n_max=4096)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, w.r)
+    outs = []
+    for _ in range(2):
+        desc, ws, scores, sums, _ = gpu_score(K, V, G, q_heads=w.q_heads)
+        idx, cnt, _ = cur.curdkv_select(scores, desc, 500, window=64)
+        outs.append((scores.clone(), sums.clone(), idx.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    m = cur.curdkv_gqa_map(desc).cpu().tolist()
+    assert m == [orc.kv_head_of_query(q, w.q_heads, w.kv_heads) for q in range(w.q_heads)]
