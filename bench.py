@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Throughput of the CurDKV prefill-time selection path on B200.
+
+One step = the whole hot path (score -> select -> compact) over one synthetic KV
+cache.  Prints ONE JSON line (rank 0).  ``--impl reference`` times the fp64 CPU
+oracle on a bounded sample of the same workload instead.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2509_15038_b200 import synth
+
+METRIC = "kv_head_tokens_compressed_per_s"
+UNIT = "head-tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_bytes(w, seqlens):
+    """Algorithmic bytes of one step: K+V read once + compacted rows written."""
+    P = w.folded_batch * w.kv_heads
+    if seqlens is None:
+        tokens = P * w.n_max
+        kept = P * min(w.budget, w.n_max)
+    else:
+        tokens = int(seqlens.astype(np.int64).sum()) * w.kv_heads
+        kept = int(np.minimum(seqlens, w.budget).astype(np.int64).sum()) * w.kv_heads
+    row_pair = 2 * w.d * 2
+    return tokens, tokens * row_pair, kept * row_pair
+
+
+# --------------------------------------------------------------------------- CUDA arm
+
+def run_cuda(args):
+    from paper_2509_15038_b200 import binding as cur
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    w = synth.CONFIGS[args.workload]
+    # weak scaling: every rank holds one full copy of the workload with its own data seed;
+    # the problems are independent, so there is no data-path collective.
+    w = synth.shrink(w, data_seed=w.data_seed + 100 * rank)
+    K, V, seqlens = synth.make_kv(w, dev)
+    G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
+    sl = None if seqlens is None else torch.as_tensor(seqlens, device=dev)
+    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads, seqlens=sl)
+    ws = cur.alloc_workspace(desc, w.budget, w.adaptive)
+    P = w.folded_batch * w.kv_heads
+    scores = torch.empty((w.folded_batch, w.kv_heads, w.n_max), dtype=torch.float32, device=dev)
+    sums = torch.empty((w.folded_batch, w.kv_heads), dtype=torch.float32, device=dev)
+    cap = min(w.budget, w.n_max)
+    if w.adaptive:
+        idx = torch.empty((P * cap,), dtype=torch.int32, device=dev)
+        Ko = torch.empty((P * cap, w.d), dtype=torch.bfloat16, device=dev)
+    else:
+        idx = torch.empty((w.folded_batch, w.kv_heads, w.budget), dtype=torch.int32, device=dev)
+        Ko = torch.empty((w.folded_batch, w.kv_heads, w.budget, w.d), dtype=torch.bfloat16, device=dev)
+    Vo = torch.empty_like(Ko)
+    cnt = torch.empty((w.folded_batch, w.kv_heads), dtype=torch.int32, device=dev)
+    off = torch.empty((P + 1,), dtype=torch.int32, device=dev)
+
+    def step(events=None):
+        if events is not None:
+            events[0].record()
+        cur.curdkv_score(K, V, G, desc, ws, scores=scores, head_sums=sums)
+        if events is not None:
+            events[1].record()
+        cur.curdkv_select(scores, desc, w.budget, num_sink=w.num_sink, window=w.window,
+                          adaptive=w.adaptive, alpha=w.alpha, workspace=ws, idx=idx,
+                          head_counts=cnt, head_offsets=off)
+        if events is not None:
+            events[2].record()
+        cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=w.adaptive, K_out=Ko, V_out=Vo,
+                           workspace=ws)
+        if events is not None:
+            events[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    flags = cur.curdkv_device_status(ws)
+    if flags:
+        raise RuntimeError(f"device status flags {flags:#x} after warm-up")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    launches0 = cur.launch_count()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        step(ev[i])
+    t1.record()
+    barrier()
+    launches = cur.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t0.elapsed_time(t1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in ev]).mean(0)
+
+    tokens, read_bytes, write_bytes = workload_bytes(w, seqlens)
+    value = world * tokens / (ms_step * 1e-3)
+    gbs = world * (read_bytes + write_bytes) / (ms_step * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    score_gbs = read_bytes / (stage_ms[0] * 1e-3) / 1e9
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": f"{w.name}: {w.layers} layers x batch {w.batch} x {w.kv_heads} KV heads "
+                        f"(GQA {w.q_heads}:{w.kv_heads}), n={w.n_max}, d={w.d}, r={w.r}, "
+                        f"budget {w.budget} incl. window {w.window}, sinks {w.num_sink}, "
+                        + ("AdaCurDKV alpha=%.2f" % w.alpha if w.adaptive else "fixed per-head budget")
+                        + (f", ragged lengths {w.ragged}" if w.ragged else ""),
+            "head_tokens_per_step": tokens, "seq_tokens_per_step": tokens // (w.layers * w.kv_heads),
+            "l2": "inputs (%.1f GB) exceed the 126 MB L2, no flush between steps" % (read_bytes / 1e9),
+            "sharding": "independent replicas per rank, no collective",
+        },
+        "gb_per_s": gbs, "counted_bytes_per_step": read_bytes + write_bytes,
+        "pct_of_nominal_8000": 100 * gbs / world / NOMINAL_HBM_GBS,
+        "pct_of_measured_copy": 100 * gbs / world / peak,
+        "seq_tokens_per_s": value / (w.layers * w.kv_heads),
+        "stage_ms": {"score": float(stage_ms[0]), "select": float(stage_ms[1]),
+                     "compact": float(stage_ms[2])},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "roofline": {
+            "bound": "hbm", "kernel": "curdkv_score (sketch + normalise)",
+            "achieved": score_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
+            "unit": "GB/s", "frac": score_gbs / peak, "traffic": None,
+            "algorithmic_bytes_per_launch": read_bytes,
+        },
+    }
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            out["cpu_baseline"] = cpu_baseline(w, core_seconds=20.0)
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- oracle arm
+
+def oracle_sample(w, elements):
+    """K, V bits of `elements` folded-batch elements of workload w, generated on the CPU."""
+    Ks, Vs = [], []
+    for lb in range(elements):
+        k, v = synth.make_kv_element(w, lb, "cpu")
+        Ks.append(synth.to_u16(k))
+        Vs.append(synth.to_u16(v))
+    seqlens = synth.make_seqlens(w)
+    sl = None if seqlens is None else seqlens[:elements].copy()
+    return np.stack(Ks), np.stack(Vs), sl
+
+
+def oracle_step(w, Ku, Vu, sl, G):
+    from oracle import curdkv_oracle as orc
+
+    sc, _ = orc.score(Ku, Vu, G, seqlens=sl)
+    if w.adaptive:
+        idx, cnt, off = orc.select_adaptive(sc, w.budget, w.num_sink, w.window, w.alpha, seqlens=sl)
+        orc.compact(Ku, Vu, idx, cnt, off)
+    else:
+        idx, cnt = orc.select_fixed(sc, w.budget, w.num_sink, w.window, seqlens=sl)
+        orc.compact(Ku, Vu, idx, cnt)
+
+
+def sample_elements(w, core_seconds):
+    """Folded-batch elements whose oracle run costs about `core_seconds` of CPU work
+    (the naive fp64 loops manage roughly 7e8 multiply-adds per core-second)."""
+    macs_per_elem = 2.0 * w.kv_heads * w.n_max * w.d * w.r
+    return int(min(max(1, round(core_seconds * 7e8 / macs_per_elem)), w.folded_batch))
+
+
+def cpu_baseline(w, core_seconds=20.0):
+    from oracle import curdkv_oracle as orc
+
+    elems = sample_elements(w, core_seconds)
+    Ku, Vu, sl = oracle_sample(w, elems)
+    G = synth.make_G(w.d, w.r, seed=0)
+    t0 = time.perf_counter()
+    oracle_step(w, Ku, Vu, sl, G)
+    dt = time.perf_counter() - t0
+    tokens = (elems * w.n_max if sl is None else int(sl.sum())) * w.kv_heads
+    return {"value": tokens / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{elems} of {w.folded_batch} (layer, sequence) groups of {w.name} "
+                      f"({elems * w.kv_heads} problems, {tokens} head-tokens), {dt:.2f} s wall",
+            "seconds": dt}
+
+
+def run_reference(args):
+    from oracle import curdkv_oracle as orc
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = synth.CONFIGS[args.workload]
+    elems = sample_elements(w, core_seconds=20.0)
+    Ku, Vu, sl = oracle_sample(w, elems)
+    G = synth.make_G(w.d, w.r, seed=0)
+    for _ in range(args.warmup):
+        oracle_step(w, Ku, Vu, sl, G)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(w, Ku, Vu, sl, G)
+    dt = (time.perf_counter() - t0) / args.steps
+    tokens = (elems * w.n_max if sl is None else int(sl.sum())) * w.kv_heads
+    value = tokens / dt
+    sample = (f"each step = {elems} of {w.folded_batch} (layer, sequence) groups of {w.name} "
+              f"({tokens} head-tokens)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name + " (bounded sample)", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

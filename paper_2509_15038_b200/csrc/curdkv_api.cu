@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "compact.cuh"
 #include "score_simt.cuh"
+#include "score_umma.cuh"
 #include "select.cuh"
 
 namespace {
@@ -46,6 +47,64 @@ inline int tiles_per_head(const curdkv_desc* d) { return (d->n_max + kTileRows -
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
+// ---- TMA descriptors for the tensor-core sketch kernel ---------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// bf16 tensor [batch][heads][n_max][128] -> 4-D map (channel, row, head, batch) with a
+// box of 64 channels x 128 rows and the 128-byte swizzle the MMA descriptors expect.
+bool make_tile_map(CUtensorMap* map, const void* base, const curdkv_desc* d, int64_t sb, int64_t sh,
+                   int64_t sn) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)d->d, (cuuint64_t)d->n_max, (cuuint64_t)d->kv_heads,
+                              (cuuint64_t)d->batch};
+  // a size-1 axis never moves: give it any legal stride
+  const cuuint64_t row = (cuuint64_t)sn * 2;
+  const cuuint64_t strides[3] = {row, d->kv_heads > 1 ? (cuuint64_t)sh * 2 : row,
+                                 d->batch > 1 ? (cuuint64_t)sb * 2 : row};
+  const cuuint32_t box[4] = {64, (cuuint32_t)kTileRows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return n;
+}
+
+template <int R>
+cudaError_t launch_umma(const CUtensorMap& mk, const CUtensorMap& mv, const umma::Args& a,
+                        cudaStream_t stream) {
+  using L = umma::Smem<R>;
+  cudaError_t e = cudaFuncSetAttribute(umma::sketch_umma_kernel<R>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+  if (e != cudaSuccess) return e;
+  const int sms = sm_count();
+  if (sms <= 0) return cudaErrorUnknown;
+  const unsigned grid = (unsigned)(a.total_tiles < sms ? a.total_tiles : sms);
+  umma::sketch_umma_kernel<R><<<grid, umma::kThreads, L::kDynamic, stream>>>(mk, mv, a);
+  return cudaSuccess;
+}
+
 KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
   return KvView{static_cast<const __nv_bfloat16*>(base), sb, sh, sn};
 }
@@ -59,7 +118,7 @@ size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32
   (void)adaptive;
   if (check_desc(desc) != CURDKV_OK) return 0;
   const size_t tiles = (size_t)desc->batch * desc->kv_heads * tiles_per_head(desc);
-  return kStatusBytes + round256(tiles * sizeof(float));
+  return kStatusBytes + round256(tiles * umma::kPartsPerTile * sizeof(float));
 }
 
 curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
@@ -100,21 +159,49 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
   a.tile_sums = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
 
   const unsigned grid = (unsigned)(P * tiles);
-  if (desc->use_projection) {
-    const int r_pad = (desc->r + 31) / 32 * 32;
-    const size_t smem = 2 * (size_t)kTileRows * kFmaD * 2 + (size_t)kFmaD * r_pad * sizeof(float);
-    if (cudaFuncSetAttribute(sketch_fma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess)
-      return CURDKV_ERR_CUDA;
-    sketch_fma_kernel<<<grid, 256, smem, stream>>>(a, r_pad);
-  } else {
-    row_norm_kernel<<<grid, 256, 0, stream>>>(a);
+  int parts = 1;                                  // partial sums per 128-row tile
+  bool launched = false;
+  if (desc->use_projection && !g_per_head && desc->n_max >= kTileRows) {
+    // tensor-core path: one G for all heads, TMA tiles of 128 rows
+    CUtensorMap mk, mv;
+    if (make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) &&
+        make_tile_map(&mv, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n)) {
+      umma::Args u;
+      u.G = G;
+      u.seqlens = desc->seqlens;
+      u.heads = desc->kv_heads;
+      u.n_max = desc->n_max;
+      u.r = desc->r;
+      u.tiles_per_head = tiles;
+      u.total_tiles = P * tiles;
+      u.score_mode = desc->score_mode;
+      u.scores = scores;
+      u.tile_sums = a.tile_sums;
+      u.status = static_cast<uint32_t*>(workspace);
+      const cudaError_t e = desc->r <= 32 ? launch_umma<32>(mk, mv, u, stream)
+                                          : launch_umma<64>(mk, mv, u, stream);
+      if (e != cudaSuccess) return CURDKV_ERR_CUDA;
+      parts = umma::kPartsPerTile;
+      launched = true;
+    }
+  }
+  if (!launched) {
+    if (desc->use_projection) {
+      const int r_pad = (desc->r + 31) / 32 * 32;
+      const size_t smem = 2 * (size_t)kTileRows * kFmaD * 2 + (size_t)kFmaD * r_pad * sizeof(float);
+      if (cudaFuncSetAttribute(sketch_fma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem) != cudaSuccess)
+        return CURDKV_ERR_CUDA;
+      sketch_fma_kernel<<<grid, 256, smem, stream>>>(a, r_pad);
+    } else {
+      row_norm_kernel<<<grid, 256, 0, stream>>>(a);
+    }
   }
   if (!launch_ok()) return CURDKV_ERR_CUDA;
 
   const int chunks = (desc->n_max + kNormChunk - 1) / kNormChunk;
   normalise_kernel<<<(unsigned)(P * chunks), 256, 0, stream>>>(scores, a.tile_sums, head_sums,
-                                                              desc->n_max, tiles, chunks);
+                                                              desc->n_max, tiles * parts, chunks);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }

@@ -192,12 +192,12 @@ constexpr int kNormChunk = 4096;
 
 __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const float* tile_sums,
                                                         float* head_sums, int n_max,
-                                                        int tiles_per_head, int chunks_per_head) {
+                                                        int parts_per_head, int chunks_per_head) {
   __shared__ float red[256];
   const int p = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;
   const int tid = threadIdx.x;
   float part = 0.f;
-  for (int i = tid; i < tiles_per_head; i += 256) part += tile_sums[(size_t)p * tiles_per_head + i];
+  for (int i = tid; i < parts_per_head; i += 256) part += tile_sums[(size_t)p * parts_per_head + i];
   red[tid] = part;
   __syncthreads();
   for (int o = 128; o > 0; o >>= 1) {

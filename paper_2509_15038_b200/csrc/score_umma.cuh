@@ -1,0 +1,367 @@
+// Fused sketch + squared-norm + combine kernel on the 5th-gen tensor cores
+// (Alg. 1 lines 2-5) for d = 128 and r <= 64.
+//
+// Per 128-token tile and tensor (K, then V):  Y = A G  with A the bf16 tile
+// [128 x 128] brought in by TMA (128-byte swizzle) and G held in shared memory
+// for the whole kernel.  fp32 G is split G = G_hi + G_lo into two bf16 matrices
+// (bf16 x bf16 products are exact in fp32, the residual of the split is
+// ~2^-17 relative), and both halves ride in one MMA as the N = 2*R columns
+// [G_hi | G_lo]; the epilogue adds the two column halves, squares and sums.
+// Y never leaves TMEM.  One tcgen05.mma (M = 128, N = 2R, K = 16) per 16
+// channels, fp32 accumulators double-buffered in TMEM.
+//
+// Persistent CTAs (one per SM), 6 warps:
+//   warp 0      TMA producer (one lane): 32 KB tensor tiles into a 6-slot ring
+//   warp 1      MMA issuer (one lane); owns the TMEM allocation
+//   warps 2-5   epilogue: tcgen05.ld -> (hi+lo)^2 row sums -> lK*lV -> scores,
+//               one partial sum per warp quarter for the head normaliser
+// Every mbarrier wait is bounded; on expiry the kernel flags
+// CURDKV_DEV_TIMEOUT, drains what it issued, frees TMEM and returns.
+#pragma once
+#include <climits>
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace curdkv {
+namespace umma {
+
+constexpr int kThreads = 192;
+constexpr int kSlots = 6;                         // ring of tensor tiles
+constexpr int kHalfBytes = kTileRows * 128;       // 128 rows x 64 bf16 (one 128-byte swizzle span)
+constexpr int kSlotBytes = 2 * kHalfBytes;        // d = 128 -> two spans
+constexpr int kPartsPerTile = 4;                  // partial sums per tile (one per epilogue warp)
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct Args {
+  const float* G;          // [128][r]
+  const int32_t* seqlens;
+  int heads, n_max, r;
+  int tiles_per_head;
+  long long total_tiles;   // batch*heads*tiles_per_head
+  int score_mode;
+  float* scores;
+  float* tile_sums;        // [total_tiles][kPartsPerTile]
+  uint32_t* status;
+};
+
+template <int R>
+struct Smem {                                     // offsets from the 1024-aligned base
+  static constexpr int kN = 2 * R;                // MMA N: [G_hi | G_lo]
+  static constexpr int kGHalf = kN * 128;         // bytes per 64-channel span of G^T
+  static constexpr int kG = 0;
+  static constexpr int kSlot0 = 2 * kGHalf;
+  static constexpr int kBar = kSlot0 + kSlots * kSlotBytes;
+  static constexpr int kTotal = kBar + 256;
+  static constexpr int kDynamic = kTotal + 1024;  // slack for manual alignment
+  static constexpr int kTmemCols = 4 * kN;        // 2 accumulator stages x {K, V} x N
+};
+
+// ---- PTX wrappers --------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Gives up when another role has aborted or after kWaitLimitNs;
+// then raises the CTA's abort flag and the device status bit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t* status) {
+  unsigned long long t0 = 0;
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 0xffu) == 0) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        flag_status(status, CURDKV_DEV_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
+      "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t* u = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]),
+        "=r"(u[7]), "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]),
+        "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]),
+        "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]),
+        "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major, 128-byte-swizzled operand:
+// rows 128 B apart, 8-row groups 1024 B apart (stride offset 64 x 16 B),
+// leading offset unused by swizzled K-major layouts (1), sm_100 version tag.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  return (uint64_t)((addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Sum over c < R of (hi_c + lo_c)^2 for this thread's row; hi at columns
+// [col, col+R), lo at [col+R, col+2R).
+template <int R>
+__device__ __forceinline__ float sketch_row_norm(uint32_t taddr) {
+  float acc = 0.f;
+#pragma unroll
+  for (int c0 = 0; c0 < R; c0 += 32) {
+    float hi[32], lo[32];
+    tmem_ld32(taddr + c0, hi);
+    tmem_ld32(taddr + R + c0, lo);
+    tmem_ld_wait();
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+      const float y = hi[c] + lo[c];
+      acc = fmaf(y, y, acc);
+    }
+  }
+  return acc;
+}
+
+// ---------------------------------------------------------------------------
+template <int R>
+__global__ void __launch_bounds__(kThreads, 1)
+sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const Args a) {
+  using L = Smem<R>;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t bar0 = base + L::kBar;
+  // barriers: full[kSlots], empty[kSlots], acc_full[2], acc_empty[2], drain
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kSlots + s); };
+  auto acc_full_bar = [&](int s) { return bar0 + 8u * (2 * kSlots + s); };
+  auto acc_empty_bar = [&](int s) { return bar0 + 8u * (2 * kSlots + 2 + s); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kSlots + 4);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + L::kBar + 8 * (2 * kSlots + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // ---- set-up: barriers, TMEM, G^T = [G_hi | G_lo] in swizzled K-major form
+  if (tid == 0) {
+    for (int s = 0; s < kSlots; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), 128); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_holder)),
+                 "r"((uint32_t)L::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int i = tid; i < 128 * R; i += kThreads) {
+    const int t = i / R, c = i % R;                        // channel t, sketch column c
+    const float g = c < a.r ? __ldg(a.G + (size_t)t * a.r + c) : 0.f;
+    const __nv_bfloat16 hi = __float2bfloat16_rn(g);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(g - __bfloat162float(hi));
+    const int span = t >> 6, tt = t & 63;
+    auto put = [&](int row, __nv_bfloat16 v) {             // row of G^T = sketch column
+      const int chunk = (tt >> 3) ^ (row & 7);             // 128-byte swizzle on 16-byte chunks
+      *reinterpret_cast<__nv_bfloat16*>(base_ptr + L::kG + span * L::kGHalf + row * 128 +
+                                        chunk * 16 + (tt & 7) * 2) = v;
+    };
+    put(c, hi);
+    put(R + c, lo);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const long long first = blockIdx.x, stride = gridDim.x;
+  // tile t -> problem p and first row; returns the head's valid rows n_b in a way that makes
+  // "result <= row0" mean "tile holds no valid row"
+  auto tile_rows = [&](long long t, int& p, int& row0) -> int {
+    p = (int)(t / a.tiles_per_head);
+    const int r0 = (int)(t % a.tiles_per_head) * kTileRows;
+    const int n = seq_len_of(a.seqlens, p / a.heads, a.n_max);
+    row0 = r0;
+    return n > r0 ? n : INT_MIN;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      uint32_t it = 0;
+      bool ok = true;
+      for (long long t = first; ok && t < a.total_tiles; t += stride) {
+        int p, row0;
+        if (tile_rows(t, p, row0) <= row0) continue;       // no valid row in this tile
+        const int b = p / a.heads, h = p % a.heads;
+        for (int tensor = 0; tensor < 2; ++tensor, ++it) {
+          const int slot = it % kSlots;
+          const uint32_t phase = (it / kSlots) & 1u;
+          if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status))) break;
+          mbar_arrive_expect_tx(full_bar(slot), kSlotBytes);
+          const uint32_t dst = base + L::kSlot0 + slot * kSlotBytes;
+          const CUtensorMap* map = tensor ? &map_v : &map_k;
+          tma_load_4d(dst, map, full_bar(slot), 0, row0, h, b, policy);
+          tma_load_4d(dst + kHalfBytes, map, full_bar(slot), 64, row0, h, b, policy);
+        }
+      }
+      if (!ok) {
+        // let the copies already issued land before the CTA gives up its shared memory
+        const uint32_t pending = it < (uint32_t)kSlots ? it : (uint32_t)kSlots;
+        for (uint32_t q = it - pending; q < it; ++q) {
+          unsigned long long t0 = global_ns();
+          while (!mbar_try_wait(full_bar(q % kSlots), (q / kSlots) & 1u) &&
+                 global_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(L::kN);
+      uint32_t it = 0, tile_it = 0;
+      bool ok = true;
+      for (long long t = first; ok && t < a.total_tiles; t += stride) {
+        int p, row0;
+        if (tile_rows(t, p, row0) <= row0) continue;
+        const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
+        if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status))) break;
+        tc_fence_after();
+        for (int tensor = 0; tensor < 2; ++tensor, ++it) {
+          const int slot = it % kSlots;
+          if (!(ok = mbar_wait(full_bar(slot), (it / kSlots) & 1u, abort_flag, a.status))) break;
+          tc_fence_after();
+          const uint32_t a_base = base + L::kSlot0 + slot * kSlotBytes;
+          const uint32_t d_tmem = tmem_base + acc * (2 * L::kN) + tensor * L::kN;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {                    // 16 channels per MMA
+            const uint32_t koff = (k >> 2) * kHalfBytes + (k & 3) * 32;
+            const uint32_t goff = (k >> 2) * L::kGHalf + (k & 3) * 32;
+            tc_mma_bf16(d_tmem, smem_desc_sw128(a_base + koff),
+                        smem_desc_sw128(base + L::kG + goff), idesc, k > 0);
+          }
+          tc_commit(empty_bar(slot));                      // slot reusable once these MMAs retire
+        }
+        if (!ok) break;
+        tc_commit(acc_full_bar(acc));
+        ++tile_it;
+      }
+      if (!ok) {                                           // drain MMAs in flight before TMEM is freed
+        tc_commit(drain_bar);
+        unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;                          // TMEM lanes this warp may read
+    uint32_t tile_it = 0;
+    bool ok = true;
+    for (long long t = first; ok && t < a.total_tiles; t += stride) {
+      int p, row0;
+      const int n = tile_rows(t, p, row0);
+      const int j = row0 + quarter * 32 + lane;
+      float s = 0.f;
+      if (n > row0) {
+        const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
+        ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status);
+        if (!(ok = __all_sync(0xffffffffu, ok))) break;    // the TMEM loads need the whole warp
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * (2 * L::kN);
+        const float lk = sketch_row_norm<R>(taddr);
+        const float lv = sketch_row_norm<R>(taddr + L::kN);
+        tc_fence_before();
+        mbar_arrive(acc_empty_bar(acc));
+        ++tile_it;
+        if (j < n) s = combine_scores(lk, lv, a.score_mode);
+      }
+      if (j < a.n_max) a.scores[(size_t)p * a.n_max + j] = s;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) a.tile_sums[(size_t)t * kPartsPerTile + quarter] = s;
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"((uint32_t)L::kTmemCols)
+                 : "memory");
+  }
+}
+
+}  // namespace umma
+}  // namespace curdkv

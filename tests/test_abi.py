@@ -29,8 +29,8 @@ def test_host_only_calls_work_without_a_device():
     assert binding.status_string(0) == "ok"
     assert "workspace" in binding.status_string(3)
     desc = binding.Desc(4, 8, 32, 1000, 128, 32, 0, 0, 128, 0, 0, 128, None, 0, 1)
-    # 256 status bytes + one fp32 partial per 128-row tile, rounded to 256 bytes
-    assert binding.workspace_bytes(desc) == 256 + 4 * 8 * 8 * 4
+    # 256 status bytes + four fp32 partials per 128-row tile, rounded to 256 bytes
+    assert binding.workspace_bytes(desc) == 256 + 4 * 8 * 8 * 4 * 4
     bad = binding.Desc(4, 8, 12, 1000, 128, 32, 0, 0, 128, 0, 0, 128, None, 0, 1)
     assert binding.workspace_bytes(bad) == 0
     assert lib.curdkv_score(None, None, None, 0, None, None, None, None, 0, None) == 1
