@@ -44,7 +44,8 @@ typedef enum curdkv_status {
   CURDKV_ERR_UNSUPPORTED = 2, /* shape outside what the kernels handle (see curdkv_score)       */
   CURDKV_ERR_WORKSPACE = 3,   /* workspace smaller than curdkv_workspace_bytes()                 */
   CURDKV_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed                               */
-  CURDKV_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (from the status word)       */
+  CURDKV_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (from the status word)       */
+  CURDKV_ERR_STATIC_LIMIT = 6 /* curdkv_score_static: shape needs more than its built-in scratch */
 } curdkv_status;
 
 /* Bits of the device status word (workspace[0], int32). */
@@ -91,6 +92,33 @@ size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32
 curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
                            const curdkv_desc* desc, float* scores, float* head_sums,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The paper has no counterpart of this call: it is curdkv_score for callers that
+ * cannot give the library a workspace because they must not allocate device
+ * memory -- code running where cudaMalloc is off limits (inside a host
+ * framework that owns the whole memory pool, in a plugin that is handed only its
+ * inputs and outputs, or late in a process that has already given all memory
+ * away).  The scratch that curdkv_score takes from the caller (status words and
+ * the per-tile partial sums of the head normaliser) lives here in an array built
+ * into the library: 4 MiB + 256 bytes of device memory held by every GPU that
+ * loads the library, until the process exits.
+ *   - Same arguments and results as curdkv_score, minus the workspace.
+ *   - Limit: batch * kv_heads * ceil(n_max / 128) <= 262144 tiles (2^20 partial
+ *     sums); larger shapes return CURDKV_ERR_STATIC_LIMIT and enqueue nothing.
+ *   - status_flags: NULL, or a device uint32 that receives the device status
+ *     word of this call (copied on the stream after the kernels).
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - The call itself allocates and frees nothing, on the device or through any
+ *     allocating library routine.
+ *   - All calls on a device share the one array, and it keeps whatever the last
+ *     call left in it; this call rewrites every word it later reads.  Two calls
+ *     whose kernels overlap on the GPU (different streams, or different host
+ *     threads without ordering) race on it: order them on one stream or with
+ *     events. */
+curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, int32_t g_per_head,
+                                  const curdkv_desc* desc, float* scores, float* head_sums,
+                                  uint32_t* status_flags, void* cuda_stream);
 
 /* Alg. 1 lines 7-9 (adaptive = 0) or AdaCurDKV (adaptive = 1).
  * Forced set of a sequence of n_b rows: the last `window` rows and the first

@@ -23,6 +23,7 @@ DEV_BAD_INDEX = 0x2
 EXPORTS = (
     "curdkv_workspace_bytes", "curdkv_score", "curdkv_select", "curdkv_compact",
     "curdkv_gqa_map", "curdkv_device_status", "curdkv_launch_count", "curdkv_status_string",
+    "curdkv_score_static",
 )
 
 
@@ -59,6 +60,8 @@ def load():
     lib.curdkv_workspace_bytes.argtypes = [dp, i32, i32]
     lib.curdkv_score.restype = ctypes.c_int
     lib.curdkv_score.argtypes = [vp, vp, vp, i32, dp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.curdkv_score_static.restype = ctypes.c_int
+    lib.curdkv_score_static.argtypes = [vp, vp, vp, i32, dp, vp, vp, vp, vp]
     lib.curdkv_select.restype = ctypes.c_int
     lib.curdkv_select.argtypes = [vp, dp, i32, vp, i32, i32, i32, ctypes.c_double, vp, vp, vp, vp,
                                   ctypes.c_size_t, vp]
@@ -141,6 +144,22 @@ def curdkv_score(K, V, G, desc: Desc, workspace: torch.Tensor, scores=None, head
                                _ptr(scores), _ptr(head_sums), _ptr(workspace),
                                workspace.numel(), _stream())
     _check(code, "curdkv_score")
+    return scores, head_sums
+
+
+def curdkv_score_static(K, V, G, desc: Desc, scores=None, head_sums=None, status_flags=None):
+    """curdkv_score for callers that may not allocate device memory: the library's built-in
+    scratch array stands in for the workspace (see the header for its limit and sharing rules).
+    Output tensors are still the caller's; pass them in to keep this call allocation-free."""
+    dev = K.device
+    if scores is None:
+        scores = torch.empty((desc.batch, desc.kv_heads, desc.n_max), dtype=torch.float32, device=dev)
+    if head_sums is None:
+        head_sums = torch.empty((desc.batch, desc.kv_heads), dtype=torch.float32, device=dev)
+    g_per_head = int(G is not None and G.dim() == 3)
+    code = load().curdkv_score_static(_ptr(K), _ptr(V), _ptr(G), g_per_head, ctypes.byref(desc),
+                                      _ptr(scores), _ptr(head_sums), _ptr(status_flags), _stream())
+    _check(code, "curdkv_score_static")
     return scores, head_sums
 
 

@@ -1,6 +1,7 @@
 // C ABI of the CurDKV library: argument checks and kernel launches.
 #include <atomic>
 #include <cstdint>
+#include <mutex>
 
 #include "common.cuh"
 #include "compact.cuh"
@@ -103,6 +104,31 @@ cudaError_t launch_umma(const CUtensorMap& mk, const CUtensorMap& mv, const umma
   const unsigned grid = (unsigned)(a.total_tiles < sms ? a.total_tiles : sms);
   umma::sketch_umma_kernel<R><<<grid, umma::kThreads, L::kDynamic, stream>>>(mk, mv, a);
   return cudaSuccess;
+}
+
+// ---- built-in scratch of curdkv_score_static --------------------------------
+// Status words plus up to kStaticParts fp32 tile partial sums.  The array lives
+// in every GPU context that loads this library, for the life of the process.
+constexpr size_t kStaticParts = size_t(1) << 20;
+constexpr size_t kStaticBytes = kStatusBytes + kStaticParts * sizeof(float);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device.  In host code the
+// array's name is only a handle, so the address is looked up once per device.
+void* static_scratch_ptr() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) return nullptr;
+    g_static_ptr[dev] = p;
+  }
+  return g_static_ptr[dev];
 }
 
 KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
@@ -297,6 +323,25 @@ curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, 
   return (*host_flags & CURDKV_DEV_TIMEOUT) ? CURDKV_ERR_TIMEOUT : CURDKV_OK;
 }
 
+curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, int32_t g_per_head,
+                                  const curdkv_desc* desc, float* scores, float* head_sums,
+                                  uint32_t* status_flags, void* cuda_stream) {
+  const size_t need = curdkv_workspace_bytes(desc, 0, 0);
+  if (need == 0) return CURDKV_ERR_INVALID_ARG;
+  if (need > kStaticBytes) return CURDKV_ERR_STATIC_LIMIT;
+  void* scratch = static_scratch_ptr();
+  if (scratch == nullptr) return CURDKV_ERR_CUDA;
+  // curdkv_score clears the status words itself; the partial sums are all rewritten
+  const curdkv_status st = curdkv_score(K, V, G, g_per_head, desc, scores, head_sums, scratch,
+                                        kStaticBytes, cuda_stream);
+  if (st != CURDKV_OK) return st;
+  if (status_flags != nullptr &&
+      cudaMemcpyAsync(status_flags, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice,
+                      static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
 uint64_t curdkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* curdkv_status_string(curdkv_status status) {
@@ -307,6 +352,8 @@ const char* curdkv_status_string(curdkv_status status) {
     case CURDKV_ERR_WORKSPACE: return "workspace too small";
     case CURDKV_ERR_CUDA: return "CUDA call failed";
     case CURDKV_ERR_TIMEOUT: return "device-side wait timed out";
+    case CURDKV_ERR_STATIC_LIMIT:
+      return "shape exceeds the built-in scratch of curdkv_score_static (2^20 tile partial sums)";
   }
   return "unknown status";
 }
