@@ -1,5 +1,6 @@
 // C ABI of the CurDKV library: argument checks and kernel launches.
 #include <atomic>
+#include <cmath>
 #include <cstdint>
 #include <mutex>
 
@@ -250,7 +251,32 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
   if (adaptive) {
     if (!(alpha >= 0.0 && alpha <= 1.0) || head_offsets == nullptr || head_budgets != nullptr)
       return CURDKV_ERR_INVALID_ARG;
-    return CURDKV_ERR_UNSUPPORTED;
+    if (desc->kv_heads > kMaxAdaptiveHeads) return CURDKV_ERR_UNSUPPORTED;
+    if (P * (int64_t)(budget < desc->n_max ? budget : desc->n_max) > 0x7fffffffLL)
+      return CURDKV_ERR_UNSUPPORTED;
+    const int min_protected = (int)floor(alpha * (double)budget);
+    if (desc->kv_heads > 8 &&
+        cudaFuncSetAttribute(select_adaptive_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
+                             1) != cudaSuccess)
+      return CURDKV_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)desc->kv_heads;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, select_adaptive_kernel, scores, desc->seqlens,
+                                             (int)desc->kv_heads, (int)desc->n_max, (int)budget,
+                                             (int)num_sink, (int)window, min_protected, idx,
+                                             head_counts, head_offsets);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+    return CURDKV_OK;
   }
   select_fixed_kernel<<<(unsigned)P, kSelThreads, 0, stream>>>(
       scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,

@@ -225,3 +225,92 @@ def test_determinism_and_gqa_map():
         assert torch.equal(a, b)
     m = cur.curdkv_gqa_map(desc).cpu().tolist()
     assert m == [orc.kv_head_of_query(q, w.q_heads, w.kv_heads) for q in range(w.q_heads)]
+
+
+# ---------------------------------------------------------------- AdaCurDKV
+
+def _adaptive_case(scores_np, budget, s, w, alpha, seqlens=None):
+    """GPU adaptive selection on given fp32 scores vs the oracle's rule on the same values."""
+    B, H, n = scores_np.shape
+    sc = torch.as_tensor(scores_np, dtype=torch.float32, device=DEV)
+    dummy = torch.empty((B, H, n, 8), dtype=torch.bfloat16, device=DEV)
+    sl = None if seqlens is None else torch.as_tensor(seqlens, dtype=torch.int32, device=DEV)
+    desc = cur.make_desc(dummy, dummy, 1, seqlens=sl)
+    idx, cnt, off = cur.curdkv_select(sc, desc, budget, num_sink=s, window=w, adaptive=True, alpha=alpha)
+    ridx, rcnt, roff = orc.select_adaptive(sc.cpu().numpy().astype(np.float64), budget, s, w, alpha,
+                                           seqlens=seqlens)
+    np.testing.assert_array_equal(cnt.cpu().numpy(), rcnt)
+    np.testing.assert_array_equal(off.cpu().numpy(), roff)
+    np.testing.assert_array_equal(idx.cpu().numpy()[: roff[-1]], ridx)
+    return idx, cnt, off
+
+
+@pytest.mark.parametrize("H", [1, 2, 3, 8, 16])
+def test_adaptive_select_matches_oracle_rule(H):
+    rng = np.random.default_rng(H)
+    B, n = 3, 3000
+    mass = rng.random((B, H, 1)) ** 3 + 0.01
+    sc = (rng.random((B, H, n)) ** 4 * mass).astype(np.float32)
+    for k, s, w, alpha in ((300, 0, 16, 0.2), (300, 4, 0, 0.0), (300, 4, 8, 1.0), (1, 0, 0, 0.5),
+                           (40, 4, 40, 0.2), (2999, 0, 5, 0.2), (3000, 0, 0, 0.2), (5000, 2, 2, 0.3),
+                           (0, 0, 0, 0.2)):
+        _adaptive_case(sc, k, s, w, alpha)
+    tied = (np.round(sc / sc.max() * 32) / 32).astype(np.float32)
+    for k, alpha in ((100, 0.2), (1500, 0.5), (700, 0.0)):
+        _adaptive_case(tied, k, 2, 3, alpha)
+    _adaptive_case(sc, 500, 1, 7, 0.2, seqlens=np.array([3000, 41, 0], dtype=np.int32))
+    one_head = np.zeros((1, H, n), dtype=np.float32)
+    one_head[0, H // 2] = rng.random(n) + 1.0
+    _adaptive_case(one_head, 200, 0, 10, 0.25)
+
+
+def test_adaptive_select_long_rows_cfg4_shape():
+    rng = np.random.default_rng(4)
+    H, n = 8, 131072
+    sc = (rng.random((1, H, n)) ** 6 * (rng.random((1, H, 1)) + 0.05)).astype(np.float32)
+    sc /= sc.sum(-1, keepdims=True)
+    w = synth.CONFIGS["cfg4"]
+    _adaptive_case(sc, w.budget, w.num_sink, w.window, w.alpha)
+
+
+def test_adaptive_pipeline_r64_packed_gather():
+    """cfg4 recipe at n = 16384: r = 64 sketch, adaptive budgets, packed gather."""
+    w = synth.shrink(synth.CONFIGS["cfg4"], layers=2, n_max=16384, budget=819 + 128)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, w.r, seed=0)
+    desc, ws, scores, sums, _ = gpu_score(K, V, G, q_heads=w.q_heads)
+    Ku, Vu = synth.to_u16(K), synth.to_u16(V)
+    rs, rS = orc.score(Ku, Vu, G)
+    pu.assert_scores_close(scores.cpu().numpy(), rs, "cfg4-shaped scores")
+    idx, cnt, off = cur.curdkv_select(scores, desc, w.budget, num_sink=w.num_sink, window=w.window,
+                                      adaptive=True, alpha=w.alpha, workspace=ws)
+    Ko, Vo = cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=True, workspace=ws)
+    assert cur.curdkv_device_status(ws) == 0
+    gi, gc, go = idx.cpu().numpy(), cnt.cpu().numpy(), off.cpu().numpy()
+    # the oracle's rule on the GPU's own fp32 scores: bit-exact
+    eidx, ecnt, eoff = orc.select_adaptive(scores.cpu().numpy().astype(np.float64), w.budget,
+                                           w.num_sink, w.window, w.alpha)
+    np.testing.assert_array_equal(gc, ecnt)
+    np.testing.assert_array_equal(go, eoff)
+    np.testing.assert_array_equal(gi[: eoff[-1]], eidx)
+    # against the oracle's fp64 scores: same totals, per-head budgets equal up to tokens whose
+    # score lies within the tie band of a cut
+    ridx, rcnt, roff = orc.select_adaptive(rs, w.budget, w.num_sink, w.window, w.alpha)
+    assert np.all(gc.sum(-1) == rcnt.sum(-1)) and go[-1] == roff[-1]
+    H = w.kv_heads
+    for b in range(w.folded_batch):
+        cuts = []
+        for h in range(H):
+            kept = ridx[roff[b * H + h]: roff[b * H + h + 1]]
+            cuts.append(rs[b, h][kept[kept < w.n_max - w.window]].min())
+        lo_cut = min(cuts)
+        for h in range(H):
+            g = set(gi[go[b * H + h]: go[b * H + h + 1]].tolist())
+            r = set(ridx[roff[b * H + h]: roff[b * H + h + 1]].tolist())
+            for j in g ^ r:
+                rel = min(abs(rs[b, h, j] / c - 1.0) for c in (lo_cut, cuts[h]))
+                assert rel < pu.TIE_BAND, (b, h, j, rel)
+    # gathered bytes of the rows the GPU selected
+    Kg, Vg = orc.compact(Ku, Vu, gi[: go[-1]], gc, go)
+    np.testing.assert_array_equal(synth.to_u16(Ko)[: go[-1]], Kg)
+    np.testing.assert_array_equal(synth.to_u16(Vo)[: go[-1]], Vg)
