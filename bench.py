@@ -102,6 +102,30 @@ def workload_bytes(w, seqlens):
     return tokens, tokens * row_pair, kept * row_pair
 
 
+# --------------------------------------------------------------------------- multi-rank helpers
+
+def rank_workload(w, rank):
+    """Weak scaling: every rank holds one full copy of the workload with its own data seed.
+    The problems are independent, so no rank ever needs another rank's data."""
+    return synth.shrink(w, data_seed=w.data_seed + 100 * rank)
+
+
+def max_over_ranks(x, device, world):
+    """The slowest rank's time: what the whole job waits for."""
+    if world == 1:
+        return float(x)
+    import torch.distributed as dist
+
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank, world, seconds):
+    """Whole-job rate: the units all ranks processed over the slowest rank's time."""
+    return world * units_per_rank / seconds
+
+
 # --------------------------------------------------------------------------- CUDA arm
 
 def run_cuda(args):
@@ -118,10 +142,7 @@ def run_cuda(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    w = synth.CONFIGS[args.workload]
-    # weak scaling: every rank holds one full copy of the workload with its own data seed;
-    # the problems are independent, so there is no data-path collective.
-    w = synth.shrink(w, data_seed=w.data_seed + 100 * rank)
+    w = rank_workload(synth.CONFIGS[args.workload], rank)
     K, V, seqlens = synth.make_kv(w, dev)
     G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
     sl = None if seqlens is None else torch.as_tensor(seqlens, device=dev)
@@ -185,17 +206,12 @@ def run_cuda(args):
     barrier()
     launches = cur.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_step = ms_total / args.steps
+    ms_step = max_over_ranks(t0.elapsed_time(t1), dev, world) / args.steps
     stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in ev]).mean(0)
 
     tokens, read_bytes, write_bytes = workload_bytes(w, seqlens)
-    value = world * tokens / (ms_step * 1e-3)
-    gbs = world * (read_bytes + write_bytes) / (ms_step * 1e-3) / 1e9
+    value = job_throughput(tokens, world, ms_step * 1e-3)
+    gbs = job_throughput(read_bytes + write_bytes, world, ms_step * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
     score_gbs = read_bytes / (stage_ms[0] * 1e-3) / 1e9
 
@@ -228,12 +244,60 @@ def run_cuda(args):
             "algorithmic_bytes_per_launch": read_bytes,
         },
     }
+    out["e2e"] = run_e2e(cur, w, K, V, seqlens, value_tokens=tokens, world=world, dev=dev,
+                         steps=min(args.steps, args.e2e_steps))
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(w, core_seconds=20.0)
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_e2e(cur, w, K, V, seqlens, value_tokens, world, dev, steps):
+    """Same metric through curdkv_compress_host: K, V start in pinned host memory, results end
+    in pinned host memory; every step pays the host->device and device->host copies."""
+    import ctypes
+
+    if steps <= 0:
+        return None
+    Kh = torch.empty(K.shape, dtype=K.dtype, pin_memory=True)
+    Vh = torch.empty(V.shape, dtype=V.dtype, pin_memory=True)
+    Kh.copy_(K)
+    Vh.copy_(V)
+    Gh = torch.as_tensor(synth.make_G(w.d, w.r, seed=0))
+    sl_host = None if seqlens is None else np.ascontiguousarray(seqlens, dtype=np.int32)
+    desc = cur.make_desc(Kh, Vh, w.r, q_heads=w.q_heads)
+    if sl_host is not None:
+        desc.seqlens = sl_host.ctypes.data
+    elem_bytes = 2 * w.kv_heads * w.n_max * w.d * 2
+    chunk_batch = int(max(1, min(w.folded_batch, (512 << 20) // elem_bytes)))
+    bufs = cur.HostBuffers(desc, w.budget, w.adaptive, chunk_batch, device=dev)
+
+    def once():
+        flags = cur.curdkv_compress_host(Kh, Vh, Gh, desc, w.budget, bufs, num_sink=w.num_sink,
+                                         window=w.window, adaptive=w.adaptive, alpha=w.alpha)
+        if flags:
+            raise RuntimeError(f"device status flags {flags:#x} in the end-to-end run")
+
+    once()
+    torch.cuda.synchronize()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        once()
+    torch.cuda.synchronize()
+    dt = max_over_ranks((time.perf_counter() - t0) / steps, dev, world)
+    h2d = Kh.numel() * 2 + Vh.numel() * 2 + (0 if sl_host is None else sl_host.nbytes)
+    d2h = (bufs.idx.numel() * 4 + bufs.counts.numel() * 4 + bufs.K_out.numel() * 2
+           + bufs.V_out.numel() * 2 + (bufs.offsets.numel() * 4 if w.adaptive else 0))
+    return {"value": job_throughput(value_tokens, world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": dt * 1e3, "steps": steps,
+            "api": "curdkv_compress_host (pinned host K, V in; pinned host idx, K', V' out)",
+            "chunk_batch": chunk_batch, "timer": "host wall clock around the synchronous calls",
+            "host_link_gb_per_s": (h2d + d2h) / dt / 1e9}
 
 
 # --------------------------------------------------------------------------- oracle arm
@@ -325,6 +389,8 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3,
+                    help="steps of the host-buffer end-to-end leg (0 disables it)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

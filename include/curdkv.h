@@ -160,6 +160,29 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
                              const int32_t* head_offsets, void* K_out, void* V_out,
                              int64_t out_stride_h, void* workspace, void* cuda_stream);
 
+/* The whole path (Alg. 1 lines 2-10, or AdaCurDKV) for a cache that lives in HOST
+ * memory: chunks of `chunk_batch` batch elements are copied to the device,
+ * scored, selected and gathered, and the results copied back, double-buffered on
+ * two internal streams so that copies overlap kernels.  Synchronous: returns when
+ * every output is in host memory.  Pinned host buffers are needed for the overlap
+ * (pageable ones work, serially).
+ *   K_host, V_host   host bf16 [batch][kv_heads][n_max][d], dense (desc strides must say so)
+ *   G_host           host fp32 [d][r] or [kv_heads][d][r]
+ *   desc->seqlens    HOST int32 [batch] or NULL in this call
+ *   K_out_host, V_out_host, idx_host, counts_host, offsets_host
+ *                    host outputs with the layouts of curdkv_select / curdkv_compact
+ *                    (offsets_host may be NULL when adaptive = 0)
+ *   arena            device scratch of curdkv_host_arena_bytes() bytes, 256-byte aligned
+ *   status_flags_host  NULL or host uint32: OR of the device status words of all chunks */
+size_t curdkv_host_arena_bytes(const curdkv_desc* desc, int32_t budget, int32_t adaptive,
+                               int32_t chunk_batch);
+curdkv_status curdkv_compress_host(const void* K_host, const void* V_host, const float* G_host,
+                                   int32_t g_per_head, const curdkv_desc* desc, int32_t budget,
+                                   int32_t num_sink, int32_t window, int32_t adaptive, double alpha,
+                                   void* K_out_host, void* V_out_host, int32_t* idx_host,
+                                   int32_t* counts_host, int32_t* offsets_host, void* arena,
+                                   size_t arena_bytes, int32_t chunk_batch, uint32_t* status_flags_host);
+
 /* GQA (Sec. 3.2): query head q uses KV head q / (q_heads / kv_heads).  Writes
  * kv_head_of_q int32 [q_heads] (device) so that attention consumers can index
  * the shared selection without replicating the compacted cache. */

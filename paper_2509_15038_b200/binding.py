@@ -23,7 +23,7 @@ DEV_BAD_INDEX = 0x2
 EXPORTS = (
     "curdkv_workspace_bytes", "curdkv_score", "curdkv_select", "curdkv_compact",
     "curdkv_gqa_map", "curdkv_device_status", "curdkv_launch_count", "curdkv_status_string",
-    "curdkv_score_static",
+    "curdkv_score_static", "curdkv_host_arena_bytes", "curdkv_compress_host",
 )
 
 
@@ -67,6 +67,12 @@ def load():
                                   ctypes.c_size_t, vp]
     lib.curdkv_compact.restype = ctypes.c_int
     lib.curdkv_compact.argtypes = [vp, vp, dp, vp, i64, vp, vp, vp, vp, i64, vp, vp]
+    lib.curdkv_host_arena_bytes.restype = ctypes.c_size_t
+    lib.curdkv_host_arena_bytes.argtypes = [dp, i32, i32, i32]
+    lib.curdkv_compress_host.restype = ctypes.c_int
+    lib.curdkv_compress_host.argtypes = [vp, vp, vp, i32, dp, i32, i32, i32, i32, ctypes.c_double,
+                                         vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i32,
+                                         ctypes.POINTER(ctypes.c_uint32)]
     lib.curdkv_gqa_map.restype = ctypes.c_int
     lib.curdkv_gqa_map.argtypes = [dp, vp, vp]
     lib.curdkv_device_status.restype = ctypes.c_int
@@ -209,6 +215,50 @@ def curdkv_compact(K, V, desc: Desc, idx, head_counts, head_offsets=None, *, pac
                                  out_stride_h, _ptr(workspace), _stream())
     _check(code, "curdkv_compact")
     return K_out, V_out
+
+
+class HostBuffers:
+    """Pinned host outputs and the device arena of :func:`curdkv_compress_host`."""
+
+    def __init__(self, desc: Desc, budget: int, adaptive: bool, chunk_batch: int, device="cuda"):
+        P = desc.batch * desc.kv_heads
+        rows = P * (min(budget, desc.n_max) if adaptive else budget)
+        pin = dict(pin_memory=True)
+        self.idx = torch.empty((max(rows, 1),), dtype=torch.int32, **pin)[:rows]
+        self.K_out = torch.empty((max(rows, 1), desc.d), dtype=torch.bfloat16, **pin)[:rows]
+        self.V_out = torch.empty((max(rows, 1), desc.d), dtype=torch.bfloat16, **pin)[:rows]
+        self.counts = torch.empty((desc.batch, desc.kv_heads), dtype=torch.int32, **pin)
+        self.offsets = torch.empty((P + 1,), dtype=torch.int32, **pin)
+        nbytes = int(load().curdkv_host_arena_bytes(ctypes.byref(desc), int(budget), int(adaptive),
+                                                    int(chunk_batch)))
+        if nbytes == 0:
+            raise ValueError("invalid shape for curdkv_compress_host")
+        self.arena = torch.empty((nbytes,), dtype=torch.uint8, device=device)
+        self.chunk_batch = int(chunk_batch)
+        if not adaptive:
+            self.idx = self.idx.view(desc.batch, desc.kv_heads, budget)
+            self.K_out = self.K_out.view(desc.batch, desc.kv_heads, budget, desc.d)
+            self.V_out = self.V_out.view(desc.batch, desc.kv_heads, budget, desc.d)
+
+
+def curdkv_compress_host(K_host, V_host, G_host, desc: Desc, budget: int, buffers: HostBuffers, *,
+                         num_sink: int = 0, window: int = 0, adaptive: bool = False,
+                         alpha: float = 0.2) -> int:
+    """Whole path on host-resident K, V (CPU tensors, ideally pinned); ``desc`` must describe the
+    host tensors (``desc.seqlens`` = address of a host int32 array or None).  Results land in
+    ``buffers``; returns the device status flags."""
+    for t in (K_host, V_host):
+        if t.device.type != "cpu" or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    flags = ctypes.c_uint32(0)
+    g_per_head = int(G_host is not None and G_host.dim() == 3)
+    code = load().curdkv_compress_host(
+        _ptr(K_host), _ptr(V_host), _ptr(G_host), g_per_head, ctypes.byref(desc), int(budget),
+        int(num_sink), int(window), int(adaptive), float(alpha), _ptr(buffers.K_out),
+        _ptr(buffers.V_out), _ptr(buffers.idx), _ptr(buffers.counts), _ptr(buffers.offsets),
+        _ptr(buffers.arena), buffers.arena.numel(), buffers.chunk_batch, ctypes.byref(flags))
+    _check(code, "curdkv_compress_host")
+    return int(flags.value)
 
 
 def curdkv_gqa_map(desc: Desc, device="cuda") -> torch.Tensor:

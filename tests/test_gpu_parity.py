@@ -314,3 +314,45 @@ def test_adaptive_pipeline_r64_packed_gather():
     Kg, Vg = orc.compact(Ku, Vu, gi[: go[-1]], gc, go)
     np.testing.assert_array_equal(synth.to_u16(Ko)[: go[-1]], Kg)
     np.testing.assert_array_equal(synth.to_u16(Vo)[: go[-1]], Vg)
+
+
+# ---------------------------------------------------------------- host-buffer entry point
+
+@pytest.mark.parametrize("adaptive", [False, True])
+def test_compress_host_matches_device_calls(adaptive):
+    """curdkv_compress_host (pinned host buffers, chunked double-buffered pipeline) gives the
+    same bits as the three device calls, with ragged lengths and a chunk size that does not
+    divide the batch."""
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=5, n_max=2048)
+    K, V, _ = synth.make_kv(w, DEV)
+    lens = np.array([2048, 1500, 0, 129, 2047], dtype=np.int32)
+    G = synth.make_G(w.d, w.r)
+    budget, s, win = 300, 2, 32
+    desc, ws, scores, sums, sl = gpu_score(K, V, G, seqlens=lens)
+    idx, cnt, off = cur.curdkv_select(scores, desc, budget, num_sink=s, window=win, adaptive=adaptive,
+                                      alpha=0.2)
+    Ko, Vo = cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=adaptive)
+    torch.cuda.synchronize()
+
+    Kh, Vh = K.cpu().pin_memory(), V.cpu().pin_memory()
+    hdesc = cur.make_desc(Kh, Vh, w.r)
+    hdesc.seqlens = lens.ctypes.data
+    bufs = cur.HostBuffers(hdesc, budget, adaptive, chunk_batch=2)
+    for _ in range(2):      # the second call reuses the arena
+        flags = cur.curdkv_compress_host(Kh, Vh, torch.as_tensor(G), hdesc, budget, bufs, num_sink=s,
+                                         window=win, adaptive=adaptive, alpha=0.2)
+        assert flags == 0
+        np.testing.assert_array_equal(bufs.counts.numpy(), cnt.cpu().numpy())
+        total = int(cnt.sum().item())
+        if adaptive:
+            np.testing.assert_array_equal(bufs.offsets.numpy(), off.cpu().numpy())
+            np.testing.assert_array_equal(bufs.idx.numpy()[:total], idx.cpu().numpy()[:total])
+            assert torch.equal(bufs.K_out[:total], Ko.cpu()[:total])
+            assert torch.equal(bufs.V_out[:total], Vo.cpu()[:total])
+        else:
+            np.testing.assert_array_equal(bufs.idx.numpy(), idx.cpu().numpy())
+            c = cnt.cpu().numpy()
+            for b in range(5):
+                for h in range(w.kv_heads):
+                    assert torch.equal(bufs.K_out[b, h, : c[b, h]], Ko.cpu()[b, h, : c[b, h]])
+                    assert torch.equal(bufs.V_out[b, h, : c[b, h]], Vo.cpu()[b, h, : c[b, h]])
