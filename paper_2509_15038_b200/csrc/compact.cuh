@@ -1,6 +1,6 @@
 // Gather of the selected rows into the compacted cache (Alg. 1 line 10):
 // byte copies with 16-byte vectors, a half-warp per row (K in lanes 0-15, V in
-// lanes 16-31), four rows in flight per warp.
+// lanes 16-31), eight rows in flight per warp.
 #pragma once
 #include "common.cuh"
 
@@ -21,7 +21,7 @@ struct CompactArgs {
 };
 
 constexpr int kCompactWarps = 8;
-constexpr int kCompactRowsPerWarp = 4;
+constexpr int kCompactRowsPerWarp = 8;
 constexpr int kCompactRowsPerCta = kCompactWarps * kCompactRowsPerWarp;
 
 // grid = batch*heads*ctas_per_head; the CTAs of a head stride over its rows.

@@ -278,9 +278,15 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
     return CURDKV_OK;
   }
-  select_fixed_kernel<<<(unsigned)P, kSelThreads, 0, stream>>>(
+  // rows that fit are staged in shared memory once and re-read from there by every pass
+  const size_t row_bytes = (((size_t)desc->n_max + 3) / 4) * sizeof(uint4);
+  const size_t stage_bytes = row_bytes <= (size_t)kSelStageBytes ? row_bytes : 0;
+  if (cudaFuncSetAttribute(select_fixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSelStageBytes) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  select_fixed_kernel<<<(unsigned)P, kSelThreads, stage_bytes, stream>>>(
       scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,
-      idx, head_counts, head_offsets);
+      (int)(stage_bytes / sizeof(uint4)), idx, head_counts, head_offsets);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }

@@ -11,7 +11,7 @@
 // channels, fp32 accumulators double-buffered in TMEM.
 //
 // Persistent CTAs (one per SM), 6 warps:
-//   warp 0      TMA producer (one lane): 32 KB tensor tiles into a 6-slot ring
+//   warp 0      TMA producer (one lane): 32 KB tensor tiles into a 4-slot ring
 //   warp 1      MMA issuer (one lane); owns the TMEM allocation
 //   warps 2-5   epilogue: tcgen05.ld -> (hi+lo)^2 row sums -> lK*lV -> scores,
 //               one partial sum per warp quarter for the head normaliser
@@ -27,7 +27,9 @@ namespace curdkv {
 namespace umma {
 
 constexpr int kThreads = 192;
-constexpr int kSlots = 6;                         // ring of tensor tiles
+// Ring of tensor tiles.  Four 32 KB slots per SM keep HBM saturated; a deeper
+// ring measurably lowers the achieved read bandwidth on B200.
+constexpr int kSlots = 4;
 constexpr int kHalfBytes = kTileRows * 128;       // 128 rows x 64 bf16 (one 128-byte swizzle span)
 constexpr int kSlotBytes = 2 * kHalfBytes;        // d = 128 -> two spans
 constexpr int kPartsPerTile = 4;                  // partial sums per tile (one per epilogue warp)
@@ -325,6 +327,10 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
   } else {
     // ------------------------------------------------------------ epilogue
     const int quarter = warp & 3;                          // TMEM lanes this warp may read
+    // scores are read again by the normaliser and the selection: ask L2 to keep them over
+    // the K/V stream, which also defers their write-back into larger bursts
+    uint64_t keep;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
     uint32_t tile_it = 0;
     bool ok = true;
     for (long long t = first; ok && t < a.total_tiles; t += stride) {
@@ -345,7 +351,10 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
         ++tile_it;
         if (j < n) s = combine_scores(lk, lv, a.score_mode);
       }
-      if (j < a.n_max) a.scores[(size_t)p * a.n_max + j] = s;
+      if (j < a.n_max)
+        asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(a.scores + (size_t)p * a.n_max + j),
+                     "f"(s), "l"(keep)
+                     : "memory");
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
       if (lane == 0) a.tile_sums[(size_t)t * kPartsPerTile + quarter] = s;

@@ -12,8 +12,7 @@ namespace curdkv {
 namespace cg = cooperative_groups;
 
 constexpr int kSelThreads = 1024;
-constexpr int kSelItems = 4;                               // consecutive tokens per thread
-constexpr int kSelChunk = kSelThreads * kSelItems;
+constexpr int kSelStageBytes = 192 * 1024;                 // largest row copy kept in shared memory
 constexpr int kMaxAdaptiveHeads = 16;                      // one CTA per head in a cluster
 
 // NaN and non-positive scores rank as 0.
@@ -42,196 +41,345 @@ struct Cut {
   bool any;                                                // false: forced tokens only
 };
 
-// One radix-select step over a 256-bin digit histogram in shared memory.
-// Finds the digit holding the `remaining`-th largest key, returns it, sets
-// `remaining` to the rank inside that digit's bucket and `above` to the number
-// of keys in higher bins.  Called by one full warp; all lanes get the results.
-__device__ __forceinline__ uint32_t pick_digit(const uint32_t* hist, uint32_t& remaining,
-                                               uint32_t& above_out) {
-  const int lane = threadIdx.x & 31;
-  uint32_t c[8], mine = 0;
-#pragma unroll
-  for (int u = 0; u < 8; ++u) { c[u] = hist[lane * 8 + u]; mine += c[u]; }
-  uint32_t above = mine;                                   // inclusive suffix sum over lanes
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
-    if (lane + o < 32) above += v;
-  }
-  above -= mine;                                           // keys in higher lanes' bins
-  uint32_t found = 0xffffffffu, rank = 0, found_above = 0;
-#pragma unroll
-  for (int u = 7; u >= 0; --u) {
-    if (above < remaining && above + c[u] >= remaining) {
-      found = lane * 8 + u;
-      rank = remaining - above;
-      found_above = above;
-    }
-    above += c[u];
-  }
-  const uint32_t who = __ballot_sync(0xffffffffu, found != 0xffffffffu);
-  const int src = who ? __ffs(who) - 1 : 0;
-  remaining = __shfl_sync(0xffffffffu, rank, src);
-  above_out = __shfl_sync(0xffffffffu, found_above, src);
-  return __shfl_sync(0xffffffffu, found, src);
-}
-
-// Number of keys in bins above `digit` (one full warp; all lanes get the sum).
-__device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t digit) {
-  const int lane = threadIdx.x & 31;
-  uint32_t s = 0;
-#pragma unroll
-  for (int u = 0; u < 8; ++u) {
-    const uint32_t bin = lane * 8 + u;
-    if (bin > digit) s += hist[bin];
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  return s;
-}
-
-// Adds the candidates [lo, hi) with key <= ceiling whose bits under `mask`
-// equal `prefix` to the 256-bin histogram of digit (key >> shift).  Runs of
-// equal digits are merged per thread before touching shared memory:
-// normalised scores share their exponent bits, so the leading digits are
-// nearly constant.
-__device__ __forceinline__ void digit_histogram(const float* row, int lo, int hi, uint32_t ceiling,
-                                                uint32_t mask, uint32_t prefix, int shift,
-                                                uint32_t* hist) {
-  uint32_t run_digit = 0, run = 0;
-  for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) {
-    const uint32_t key = score_key(__ldg(row + j));
-    if (key > ceiling || (key & mask) != prefix) continue;
-    const uint32_t dgt = (key >> shift) & 0xffu;
-    if (dgt == run_digit) { ++run; continue; }
-    if (run) atomicAdd(&hist[run_digit], run);
-    run_digit = dgt;
-    run = 1;
-  }
-  if (run) atomicAdd(&hist[run_digit], run);
-}
+// The 32-bit keys are consumed most significant digit first in three radix
+// passes of 12, 12 and 8 bits.  A wide leading digit matters: normalised scores
+// of one head span only a few binades, so an 8-bit leading digit would send
+// nearly every key to the same two or three histogram bins and serialise the
+// shared-memory atomics.
+constexpr int kSelPasses = 3;
+constexpr int kSelBins = 4096;
+__device__ __forceinline__ int pass_shift(int pass) { return pass == 0 ? 20 : (pass == 1 ? 8 : 0); }
+__device__ __forceinline__ uint32_t pass_digit_mask(int pass) { return pass == 2 ? 0xffu : 0xfffu; }
 
 struct SelectSmem {
-  uint32_t hist[256];
-  uint32_t warp_tot[32];
+  alignas(16) uint32_t hist[kSelBins];                     // read and cleared as 16-byte vectors
+  uint32_t warp_def[32], warp_eq[32];
   uint32_t digit, remaining, above;
 };
 
-// Top-kk cut of the candidates [lo, hi) of one row (0 < kk < hi - lo).  Whole CTA.
-__device__ __forceinline__ Cut local_cut(const float* row, int lo, int hi, int kk, SelectSmem& sm) {
-  const int tid = threadIdx.x;
+__device__ __forceinline__ void clear_hist(uint32_t* hist) {
+  reinterpret_cast<uint4*>(hist)[threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);   // 1024 threads x 4 bins
+}
+
+// One radix-select step over the kSelBins-bin histogram `hist`: finds the digit
+// holding the `remaining`-th largest key and leaves it in sm.digit, the rank
+// inside that digit's bucket in sm.remaining and the number of keys in higher
+// bins in sm.above.  Whole CTA (1024 threads, four bins each); the results are
+// readable after the call.
+__device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint4 c4 = reinterpret_cast<const uint4*>(hist)[tid];
+  const uint32_t c[4] = {c4.x, c4.y, c4.z, c4.w};
+  const uint32_t mine = c[0] + c[1] + c[2] + c[3];
+  uint32_t suffix = mine;                                  // inclusive suffix sum over the warp
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_down_sync(0xffffffffu, suffix, o);
+    if (lane + o < 32) suffix += v;
+  }
+  if (lane == 0) sm.warp_def[warp] = suffix;
+  if (tid == 0) { sm.digit = 0; sm.remaining = 0; sm.above = 0; }
+  __syncthreads();
+  uint32_t w = sm.warp_def[lane], wsuf = w;                // inclusive suffix sum over the warps
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_down_sync(0xffffffffu, wsuf, o);
+    if (lane + o < 32) wsuf += v;
+  }
+  uint32_t above = __shfl_sync(0xffffffffu, wsuf - w, warp) + (suffix - mine);
+#pragma unroll
+  for (int u = 3; u >= 0; --u) {
+    if (above < remaining && above + c[u] >= remaining) {
+      sm.digit = (uint32_t)(tid * 4 + u);
+      sm.remaining = remaining - above;
+      sm.above = above;
+    }
+    above += c[u];
+  }
+  __syncthreads();
+}
+
+// Number of keys of `hist` in bins above `digit`.  Whole CTA; every thread gets the sum.
+__device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint4 c4 = reinterpret_cast<const uint4*>(hist)[tid];
+  const uint32_t c[4] = {c4.x, c4.y, c4.z, c4.w};
+  uint32_t v = 0;
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+    if ((uint32_t)(tid * 4 + u) > digit) v += c[u];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if (lane == 0) sm.warp_eq[warp] = v;
+  __syncthreads();
+  uint32_t t = sm.warp_eq[lane];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  __syncthreads();
+  return t;
+}
+
+// Keys of one row, four tokens at a time ("quad" q holds tokens 4q .. 4q+3).
+// They come from the copy staged in shared memory when the row fits there,
+// otherwise from the fp32 scores in global memory (16-byte loads when the row
+// is aligned).  Tokens at or beyond n read as key 0; callers mask them by index.
+struct RowKeys {
+  const float* row;
+  const uint4* staged;                                     // nullptr: read global memory
+  int n;
+  bool vec;                                                // row is 16-byte aligned
+
+  __device__ __forceinline__ uint4 load4(int q) const {
+    if (staged != nullptr) return staged[q];
+    const int j = 4 * q;
+    float4 f;
+    if (vec && j + 3 < n) {
+      f = __ldg(reinterpret_cast<const float4*>(row) + q);
+    } else {
+      f.x = j < n ? __ldg(row + j) : 0.f;
+      f.y = j + 1 < n ? __ldg(row + j + 1) : 0.f;
+      f.z = j + 2 < n ? __ldg(row + j + 2) : 0.f;
+      f.w = j + 3 < n ? __ldg(row + j + 3) : 0.f;
+    }
+    return make_uint4(score_key(f.x), score_key(f.y), score_key(f.z), score_key(f.w));
+  }
+};
+
+__device__ __forceinline__ RowKeys global_keys(const float* row, int n) {
+  return RowKeys{row, nullptr, n, (reinterpret_cast<uintptr_t>(row) & 15u) == 0};
+}
+
+// Running (digit, count) pair of one thread: equal neighbouring digits are
+// merged before they reach the shared-memory histogram.  Normalised scores
+// share their exponent bits, so the leading digits are nearly constant.
+struct DigitRun {
+  uint32_t digit = 0, count = 0;
+  __device__ __forceinline__ void add(uint32_t d, uint32_t* hist) {
+    if (d == digit) { ++count; return; }
+    if (count) atomicAdd(&hist[digit], count);
+    digit = d;
+    count = 1;
+  }
+  __device__ __forceinline__ void flush(uint32_t* hist) {
+    if (count) atomicAdd(&hist[digit], count);
+    count = 0;
+  }
+};
+
+constexpr int kSelUnroll = 4;                              // quads in flight per thread
+
+// Adds the candidates [lo, hi) with key <= ceiling whose bits under `mask`
+// equal `prefix` to the histogram of this pass's digit.  Whole CTA.
+__device__ __forceinline__ void digit_histogram(const RowKeys& keys, int lo, int hi, uint32_t ceiling,
+                                                uint32_t mask, uint32_t prefix, int pass,
+                                                uint32_t* hist) {
+  const int shift = pass_shift(pass);
+  const uint32_t dmask = pass_digit_mask(pass);
+  if (hi <= lo) return;
+  const int q_lo = lo >> 2, q_hi = (hi + 3) >> 2, step = (int)blockDim.x;
+  DigitRun run;
+  for (int q0 = q_lo + (int)threadIdx.x; q0 < q_hi; q0 += kSelUnroll * step) {
+    uint4 v[kSelUnroll];
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u)
+      if (q0 + u * step < q_hi) v[u] = keys.load4(q0 + u * step);
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u) {
+      const int q = q0 + u * step;
+      if (q < q_hi) {
+        const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+        const bool edge = 4 * q < lo || 4 * q + 3 >= hi;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t key = k4[i];
+          if (edge && (4 * q + i < lo || 4 * q + i >= hi)) continue;
+          if (key > ceiling || (key & mask) != prefix) continue;
+          run.add((key >> shift) & dmask, hist);
+        }
+      }
+    }
+  }
+  run.flush(hist);
+}
+
+// Copies the keys of a row into shared memory and, on the way, builds the
+// histogram of the leading digit of the candidates [lo, hi).  Whole CTA;
+// hist must be zero on entry.
+__device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, int lo, int hi,
+                                           uint32_t* hist) {
+  const int quads = (src.n + 3) >> 2, step = (int)blockDim.x;
+  DigitRun run;
+  for (int q0 = (int)threadIdx.x; q0 < quads; q0 += kSelUnroll * step) {
+    uint4 v[kSelUnroll];
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u)
+      if (q0 + u * step < quads) v[u] = src.load4(q0 + u * step);
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u) {
+      const int q = q0 + u * step;
+      if (q < quads) {
+        staged[q] = v[u];
+        const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (4 * q + i >= lo && 4 * q + i < hi) run.add(k4[i] >> 20, hist);
+      }
+    }
+  }
+  run.flush(hist);
+}
+
+// Top-kk cut of the candidates [lo, hi) of one row (0 < kk < hi - lo).  Whole
+// CTA.  With first_hist_ready the leading-digit histogram is already in
+// sm.hist (built by stage_keys).
+__device__ __forceinline__ Cut local_cut(const RowKeys& keys, int lo, int hi, int kk, SelectSmem& sm,
+                                         bool first_hist_ready) {
   uint32_t prefix = 0, mask = 0, remaining = (uint32_t)kk;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) sm.hist[tid] = 0;
-    __syncthreads();
-    digit_histogram(row, lo, hi, 0xffffffffu, mask, prefix, shift, sm.hist);
-    __syncthreads();
-    if (tid < 32) {
-      uint32_t rem = remaining, above;
-      const uint32_t dgt = pick_digit(sm.hist, rem, above);
-      if (tid == 0) { sm.digit = dgt; sm.remaining = rem; }
+  for (int pass = 0; pass < kSelPasses; ++pass) {
+    if (!(first_hist_ready && pass == 0)) {
+      clear_hist(sm.hist);
+      __syncthreads();
+      digit_histogram(keys, lo, hi, 0xffffffffu, mask, prefix, pass, sm.hist);
     }
     __syncthreads();
-    prefix |= sm.digit << shift;
-    mask |= 0xffu << shift;
+    pick_digit(sm.hist, remaining, sm);
+    prefix |= sm.digit << pass_shift(pass);
+    mask |= pass_digit_mask(pass) << pass_shift(pass);
     remaining = sm.remaining;
     __syncthreads();
   }
   return Cut{prefix, remaining, true};
 }
 
-// Exclusive block scan of a packed (lo16 | hi16 << 16) counter; returns the
-// exclusive prefix of this thread and the block total.  blockDim = 1024.
-__device__ __forceinline__ uint32_t block_scan_packed(uint32_t v, uint32_t* warp_tot,
-                                                      uint32_t& total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  if (lane == 31) warp_tot[warp] = inc;
-  __syncthreads();
-  uint32_t w = warp_tot[lane];
-  uint32_t winc = w;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xffffffffu, winc, o);
-    if (lane >= o) winc += t;
-  }
-  total = __shfl_sync(0xffffffffu, winc, 31);
-  const uint32_t wexc = __shfl_sync(0xffffffffu, winc - w, warp);
-  __syncthreads();                                         // warp_tot may be reused
-  return wexc + inc - v;
-}
-
 // Ordered compaction of one row: forced tokens, keys above cut.T and the first
 // cut.eq_take keys equal to cut.T, written to `out` in ascending token order.
-__device__ __forceinline__ void ordered_compact(const float* row, int n, const ForcedSet& F,
+// Every warp owns a contiguous run of quads; a first sweep counts what each
+// warp keeps, one scan over the warp totals places the warps, a second sweep
+// writes.  Whole CTA, blockDim = 1024.
+__device__ __forceinline__ void ordered_compact(const RowKeys& keys, const ForcedSet& F,
                                                 const Cut& cut, int32_t* out, SelectSmem& sm) {
-  const int tid = threadIdx.x;
-  uint32_t def_base = 0, eq_base = 0;
-  for (int j0 = 0; j0 < n; j0 += kSelChunk) {
-    const int j = j0 + tid * kSelItems;
-    uint32_t def_f = 0, eq_f = 0;                          // bit i: item i
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n = keys.n, quads = (n + 3) >> 2;
+  const int per_warp = (((quads + 31) >> 5) + 31) & ~31;   // quads per warp, whole warp sweeps
+  const int q_begin = min(warp * per_warp, quads), q_end = min(q_begin + per_warp, quads);
+
+  // flags of the four tokens of quad q: bits 0-3 kept for sure, bits 4-7 equal to the cut
+  auto classify = [&](int q, const uint4& v) -> uint32_t {
+    const uint32_t k4[4] = {v.x, v.y, v.z, v.w};
+    uint32_t f = 0;
 #pragma unroll
-    for (int i = 0; i < kSelItems; ++i) {
-      const int jj = j + i;
-      if (jj < n) {
-        const bool forced = jj < F.sinks || jj >= F.hi;
-        if (forced) {
-          def_f |= 1u << i;
-        } else if (cut.any) {
-          const uint32_t key = score_key(__ldg(row + jj));
-          if (key > cut.T) def_f |= 1u << i;
-          else if (key == cut.T) eq_f |= 1u << i;
+    for (int i = 0; i < 4; ++i) {
+      const int j = 4 * q + i;
+      if (j < n) {
+        if (j < F.sinks || j >= F.hi) f |= 1u << i;
+        else if (cut.any) {
+          if (k4[i] > cut.T) f |= 1u << i;
+          else if (k4[i] == cut.T) f |= 16u << i;
         }
       }
     }
-    uint32_t total;
-    const uint32_t exc = block_scan_packed(
-        (uint32_t)__popc(def_f) | ((uint32_t)__popc(eq_f) << 16), sm.warp_tot, total);
-    uint32_t def_before = def_base + (exc & 0xffffu);
-    uint32_t eq_before = eq_base + (exc >> 16);
+    return f;
+  };
+
+  uint32_t def_cnt = 0, eq_cnt = 0;
+  for (int q0 = q_begin + lane; q0 < q_end; q0 += kSelUnroll * 32) {
+    uint4 v[kSelUnroll];
 #pragma unroll
-    for (int i = 0; i < kSelItems; ++i) {
-      if (def_f & (1u << i)) {
-        out[def_before + min(eq_before, cut.eq_take)] = j + i;
-        ++def_before;
-      } else if (eq_f & (1u << i)) {
-        if (eq_before < cut.eq_take) out[def_before + eq_before] = j + i;
-        ++eq_before;
+    for (int u = 0; u < kSelUnroll; ++u)
+      if (q0 + u * 32 < q_end) v[u] = keys.load4(q0 + u * 32);
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u) {
+      if (q0 + u * 32 < q_end) {
+        const uint32_t f = classify(q0 + u * 32, v[u]);
+        def_cnt += __popc(f & 15u);
+        eq_cnt += __popc(f >> 4);
       }
     }
-    def_base += total & 0xffffu;
-    eq_base += total >> 16;
   }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    def_cnt += __shfl_xor_sync(0xffffffffu, def_cnt, o);
+    eq_cnt += __shfl_xor_sync(0xffffffffu, eq_cnt, o);
+  }
+  if (lane == 0) { sm.warp_def[warp] = def_cnt; sm.warp_eq[warp] = eq_cnt; }
+  __syncthreads();
+  uint32_t def_before = 0, eq_before = 0;                  // kept / equal tokens of earlier warps
+  {
+    const uint32_t d = sm.warp_def[lane], e = sm.warp_eq[lane];
+    uint32_t di = d, ei = e;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t td = __shfl_up_sync(0xffffffffu, di, o), te = __shfl_up_sync(0xffffffffu, ei, o);
+      if (lane >= o) { di += td; ei += te; }
+    }
+    def_before = __shfl_sync(0xffffffffu, di - d, warp);
+    eq_before = __shfl_sync(0xffffffffu, ei - e, warp);
+  }
+
+  for (int q0 = q_begin; q0 < q_end; q0 += 32) {           // uniform trip count across the warp
+    const int q = q0 + lane;
+    uint32_t f = 0;
+    if (q < q_end) f = classify(q, keys.load4(q));
+    const uint32_t mine = (uint32_t)__popc(f & 15u) | ((uint32_t)__popc(f >> 4) << 16);
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
+    uint32_t d = def_before + ((inc - mine) & 0xffffu), e = eq_before + ((inc - mine) >> 16);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (f & (1u << i)) {
+        out[d + min(e, cut.eq_take)] = 4 * q + i;
+        ++d;
+      } else if (f & (16u << i)) {
+        if (e < cut.eq_take) out[d + e] = 4 * q + i;
+        ++e;
+      }
+    }
+    def_before += total & 0xffffu;
+    eq_before += total >> 16;
+  }
+  __syncthreads();                                         // sm.warp_* may be reused
 }
 
 // ---------------------------------------------------------------------------
-// Fixed per-head budget.  grid = batch*heads, block = 1024.
+// Fixed per-head budget.  grid = batch*heads, block = 1024, dynamic shared
+// memory = 16 * stage_quads bytes (0: rows are read from global memory).
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
-    int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window,
+    int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window, int stage_quads,
     int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   __shared__ SelectSmem sm;
+  extern __shared__ uint4 staged_keys[];                   // stage_quads quads, or nothing
   const int p = blockIdx.x, b = p / heads, tid = threadIdx.x;
   const int n = seq_len_of(seqlens, b, n_max);
   int k = budget;
   if (head_budgets != nullptr) k = max(0, min(head_budgets[p], budget));
   const int k_eff = min(k, n);
   const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  const float* row = scores + (size_t)p * n_max;
+  RowKeys keys = global_keys(scores + (size_t)p * n_max, n);
   int32_t* out = idx + (size_t)p * budget;
   const int cand = F.hi - F.sinks;
 
   Cut cut{0u, 0u, F.free_slots > 0};
-  if (F.free_slots >= cand) cut.eq_take = (uint32_t)max(cand, 0);   // every candidate is kept
-  else if (cut.any) cut = local_cut(row, F.sinks, F.hi, F.free_slots, sm);
+  if (F.free_slots >= cand) {
+    cut.eq_take = (uint32_t)max(cand, 0);                  // every candidate is kept
+  } else if (cut.any) {
+    const bool stage = ((n + 3) >> 2) <= stage_quads;      // the row fits in shared memory
+    if (stage) {
+      clear_hist(sm.hist);
+      __syncthreads();
+      stage_keys(keys, staged_keys, F.sinks, F.hi, sm.hist);
+      keys.staged = staged_keys;
+    }
+    cut = local_cut(keys, F.sinks, F.hi, F.free_slots, sm, stage);
+  }
 
-  ordered_compact(row, n, F, cut, out, sm);
+  ordered_compact(keys, F, cut, out, sm);
   for (int t = k_eff + tid; t < budget; t += kSelThreads) out[t] = -1;
   if (tid == 0) {
     counts[p] = k_eff;
@@ -253,7 +401,7 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
 // ---------------------------------------------------------------------------
 struct AdaptiveSmem {
   SelectSmem s;
-  uint32_t hist_local[256];                                // read by the other CTAs of the cluster
+  alignas(16) uint32_t hist_local[kSelBins];               // read by the other CTAs of the cluster
   uint32_t pub_eq;                                         // unprotected keys equal to the global cut
   uint32_t pub_count;                                      // rows this head keeps
 };
@@ -270,7 +418,7 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   const int n = seq_len_of(seqlens, b, n_max);
   const int k_eff = min(budget, n);
   const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  const float* row = scores + (size_t)p * n_max;
+  const RowKeys keys = global_keys(scores + (size_t)p * n_max, n);
   const int cand = F.hi - F.sinks;
   const int forced = k_eff - F.free_slots;
   const int prot = min(max(min_protected, forced), k_eff);  // protected rows per head, forced included
@@ -280,7 +428,7 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   const bool prot_all = pp >= cand;                         // every candidate is protected
   const bool prot_none = pp == 0 && !prot_all;
   Cut own{0u, 0u, false};
-  if (!prot_all && !prot_none) own = local_cut(row, F.sinks, F.hi, pp, sm.s);
+  if (!prot_all && !prot_none) own = local_cut(keys, F.sinks, F.hi, pp, sm.s, false);
   // unprotected keys: candidates with key <= ceiling, minus the first own.eq_take equal to it
   const uint32_t ceiling = prot_none ? 0xffffffffu : own.T;
 
@@ -289,32 +437,31 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   uint32_t Tg = 0, eq_g = 0, local_gt = 0, local_eq = 0;
   if (pool > 0) {
     uint32_t prefix = 0, mask = 0, remaining = pool;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      if (tid < 256) sm.hist_local[tid] = 0;
+    for (int pass = 0; pass < kSelPasses; ++pass) {
+      const int shift = pass_shift(pass);
+      clear_hist(sm.hist_local);
       __syncthreads();
-      if (!prot_all) digit_histogram(row, F.sinks, F.hi, ceiling, mask, prefix, shift, sm.hist_local);
+      if (!prot_all) digit_histogram(keys, F.sinks, F.hi, ceiling, mask, prefix, pass, sm.hist_local);
       __syncthreads();
       if (tid == 0 && !prot_all && !prot_none && (own.T & mask) == prefix)
-        sm.hist_local[(own.T >> shift) & 0xffu] -= own.eq_take;   // those are protected
+        sm.hist_local[(own.T >> shift) & pass_digit_mask(pass)] -= own.eq_take;   // those are protected
       cluster.sync();
-      if (tid < 256) {
-        uint32_t s = 0;
-        for (int r = 0; r < heads; ++r) s += cluster.map_shared_rank(sm.hist_local, r)[tid];
-        sm.s.hist[tid] = s;
+      {
+        uint4 acc = make_uint4(0u, 0u, 0u, 0u);            // this thread's four bins over all heads
+        for (int r = 0; r < heads; ++r) {
+          const uint4 v = reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid];
+          acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        reinterpret_cast<uint4*>(sm.s.hist)[tid] = acc;
       }
       __syncthreads();
-      if (tid < 32) {
-        uint32_t rem = remaining, above;
-        const uint32_t dgt = pick_digit(sm.s.hist, rem, above);
-        const uint32_t mine_above = count_above(sm.hist_local, dgt);
-        if (tid == 0) { sm.s.digit = dgt; sm.s.remaining = rem; sm.s.above = mine_above; }
-      }
-      __syncthreads();
-      prefix |= sm.s.digit << shift;
-      mask |= 0xffu << shift;
+      pick_digit(sm.s.hist, remaining, sm.s);
+      const uint32_t dgt = sm.s.digit;
       remaining = sm.s.remaining;
-      local_gt += sm.s.above;
-      if (shift == 0) local_eq = sm.hist_local[sm.s.digit];
+      prefix |= dgt << shift;
+      mask |= pass_digit_mask(pass) << shift;
+      local_gt += count_above(sm.hist_local, dgt, sm.s);
+      if (pass == kSelPasses - 1) local_eq = sm.hist_local[dgt];
       cluster.sync();                                      // peers are done reading hist_local
     }
     Tg = prefix;
@@ -349,14 +496,14 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
     part += (uint32_t)heads * (uint32_t)min(budget, seq_len_of(seqlens, bb, n_max));
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-  if ((tid & 31) == 0) sm.s.warp_tot[tid >> 5] = part;
+  if ((tid & 31) == 0) sm.s.warp_def[tid >> 5] = part;
   __syncthreads();
   uint32_t off = 0;
-  for (int w = 0; w < kSelThreads / 32; ++w) off += sm.s.warp_tot[w];
+  for (int w = 0; w < kSelThreads / 32; ++w) off += sm.s.warp_def[w];
   for (int r = 0; r < h; ++r) off += *cluster.map_shared_rank(&sm.pub_count, r);
   __syncthreads();
 
-  ordered_compact(row, n, F, cut, idx + off, sm.s);
+  ordered_compact(keys, F, cut, idx + off, sm.s);
   if (tid == 0) {
     counts[p] = (int32_t)kept;
     offsets[p] = (int32_t)off;
