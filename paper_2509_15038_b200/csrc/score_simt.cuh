@@ -193,23 +193,43 @@ constexpr int kNormChunk = 4096;
 __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const float* tile_sums,
                                                         float* head_sums, int n_max,
                                                         int parts_per_head, int chunks_per_head) {
-  __shared__ float red[256];
+  __shared__ float red[8];
   const int p = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;
-  const int tid = threadIdx.x;
-  float part = 0.f;
-  for (int i = tid; i < parts_per_head; i += 256) part += tile_sums[(size_t)p * parts_per_head + i];
-  red[tid] = part;
-  __syncthreads();
-  for (int o = 128; o > 0; o >>= 1) {
-    if (tid < o) red[tid] += red[tid + o];
-    __syncthreads();
-  }
-  const float S = red[0];
-  if (chunk == 0 && tid == 0) head_sums[p] = S;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   float* row = scores + (size_t)p * n_max;
   const int j0 = chunk * kNormChunk;
-  for (int j = j0 + tid; j < j0 + kNormChunk && j < n_max; j += 256)
-    row[j] = S > 0.f ? __fdiv_rn(row[j], S) : 0.f;
+  const int j1 = min(j0 + kNormChunk, n_max);
+  // this thread's scores are on their way while the head sum is formed
+  const bool vec = (reinterpret_cast<uintptr_t>(row) & 15u) == 0 && j1 - j0 == kNormChunk;
+  float4 v[4];
+  if (vec) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = reinterpret_cast<const float4*>(row + j0)[tid + 256 * u];
+  }
+  float part = 0.f;                                        // fixed order: thread, warp tree, warp order
+  for (int i = tid; i < parts_per_head; i += 256) part += tile_sums[(size_t)p * parts_per_head + i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+  if (lane == 0) red[warp] = part;
+  __syncthreads();
+  float S = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) S += red[w];
+  if (chunk == 0 && tid == 0) head_sums[p] = S;
+  const bool live = S > 0.f;
+  if (vec) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float4 o;
+      o.x = live ? __fdiv_rn(v[u].x, S) : 0.f;
+      o.y = live ? __fdiv_rn(v[u].y, S) : 0.f;
+      o.z = live ? __fdiv_rn(v[u].z, S) : 0.f;
+      o.w = live ? __fdiv_rn(v[u].w, S) : 0.f;
+      reinterpret_cast<float4*>(row + j0)[tid + 256 * u] = o;
+    }
+  } else {
+    for (int j = j0 + tid; j < j1; j += 256) row[j] = live ? __fdiv_rn(row[j], S) : 0.f;
+  }
 }
 
 }  // namespace curdkv

@@ -2,6 +2,13 @@
 // window, then an exact top-k of the remaining scores by radix select on the
 // fp32 bit patterns (scores are >= 0, so the patterns order like the values),
 // ties to the lower token index, output in ascending token order.
+//
+// Every token of a row gets a 32-bit rank key:
+//   0             position at or beyond the sequence length (never kept)
+//   bits(s) + 1   candidate with score s (NaN and s <= 0 rank as score 0)
+//   0xffffffff    forced token (sink or window; always kept)
+// so "keep the forced tokens and the best k - |forced| candidates" becomes
+// "keep the k largest keys", and no pass needs the token index again.
 #pragma once
 #include <cooperative_groups.h>
 
@@ -14,9 +21,9 @@ namespace cg = cooperative_groups;
 constexpr int kSelThreads = 1024;
 constexpr int kSelStageBytes = 192 * 1024;                 // largest row copy kept in shared memory
 constexpr int kMaxAdaptiveHeads = 16;                      // one CTA per head in a cluster
+constexpr uint32_t kForcedKey = 0xffffffffu;
 
-// NaN and non-positive scores rank as 0.
-__device__ __forceinline__ uint32_t score_key(float s) { return s > 0.f ? __float_as_uint(s) : 0u; }
+__device__ __forceinline__ uint32_t score_key(float s) { return s > 0.f ? __float_as_uint(s) + 1u : 1u; }
 
 // The forced-keep set of a sequence of n rows under a budget of k_eff rows:
 // sinks [0, sinks) and window [hi, n); candidates are [sinks, hi).
@@ -34,17 +41,19 @@ __device__ __forceinline__ ForcedSet forced_set(int n, int k_eff, int num_sink, 
   return f;
 }
 
-// What the ordered compaction keeps besides the forced tokens: every candidate
-// key above T and the first eq_take candidates (by token index) equal to T.
+// What the ordered compaction keeps: every key above T and the first eq_take
+// keys (by token index) equal to T.
 struct Cut {
   uint32_t T, eq_take;
-  bool any;                                                // false: forced tokens only
 };
+__device__ __forceinline__ Cut keep_nothing() { return Cut{0xffffffffu, 0u}; }
+__device__ __forceinline__ Cut keep_forced_only() { return Cut{0xfffffffeu, 0u}; }
+__device__ __forceinline__ Cut keep_every_token() { return Cut{0u, 0u}; }
 
-// The 32-bit keys are consumed most significant digit first in three radix
-// passes of 12, 12 and 8 bits.  A wide leading digit matters: normalised scores
-// of one head span only a few binades, so an 8-bit leading digit would send
-// nearly every key to the same two or three histogram bins and serialise the
+// The keys are consumed most significant digit first in three radix passes of
+// 12, 12 and 8 bits.  A wide leading digit matters: normalised scores of one
+// head span only a few binades, so an 8-bit leading digit would send nearly
+// every key to the same two or three histogram bins and serialise the
 // shared-memory atomics.
 constexpr int kSelPasses = 3;
 constexpr int kSelBins = 4096;
@@ -119,39 +128,45 @@ __device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t d
   return t;
 }
 
-// Keys of one row, four tokens at a time ("quad" q holds tokens 4q .. 4q+3).
-// They come from the copy staged in shared memory when the row fits there,
-// otherwise from the fp32 scores in global memory (16-byte loads when the row
-// is aligned).  Tokens at or beyond n read as key 0; callers mask them by index.
+// Rank keys of one row, four tokens at a time ("quad" q holds tokens
+// 4q .. 4q+3).  They come from the copy staged in shared memory when the row
+// fits there, otherwise they are rebuilt from the fp32 scores in global memory
+// (16-byte loads when the row is aligned).
 struct RowKeys {
   const float* row;
   const uint4* staged;                                     // nullptr: read global memory
-  int n;
+  int n, sinks, hi;                                        // candidates are [sinks, hi)
   bool vec;                                                // row is 16-byte aligned
+
+  __device__ __forceinline__ int quads() const { return (n + 3) >> 2; }
+
+  __device__ __forceinline__ uint32_t key_of(float s, int j) const {
+    if (j >= n) return 0u;
+    if (j < sinks || j >= hi) return kForcedKey;
+    return score_key(s);
+  }
 
   __device__ __forceinline__ uint4 load4(int q) const {
     if (staged != nullptr) return staged[q];
     const int j = 4 * q;
-    float4 f;
-    if (vec && j + 3 < n) {
-      f = __ldg(reinterpret_cast<const float4*>(row) + q);
-    } else {
-      f.x = j < n ? __ldg(row + j) : 0.f;
-      f.y = j + 1 < n ? __ldg(row + j + 1) : 0.f;
-      f.z = j + 2 < n ? __ldg(row + j + 2) : 0.f;
-      f.w = j + 3 < n ? __ldg(row + j + 3) : 0.f;
+    if (vec && j >= sinks && j + 3 < hi) {                 // interior quad: four candidates
+      const float4 f = __ldg(reinterpret_cast<const float4*>(row) + q);
+      return make_uint4(score_key(f.x), score_key(f.y), score_key(f.z), score_key(f.w));
     }
-    return make_uint4(score_key(f.x), score_key(f.y), score_key(f.z), score_key(f.w));
+    float f[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f[i] = j + i < n ? __ldg(row + j + i) : 0.f;
+    return make_uint4(key_of(f[0], j), key_of(f[1], j + 1), key_of(f[2], j + 2), key_of(f[3], j + 3));
   }
 };
 
-__device__ __forceinline__ RowKeys global_keys(const float* row, int n) {
-  return RowKeys{row, nullptr, n, (reinterpret_cast<uintptr_t>(row) & 15u) == 0};
+__device__ __forceinline__ RowKeys global_keys(const float* row, int n, const ForcedSet& F) {
+  return RowKeys{row, nullptr, n, F.sinks, F.hi, (reinterpret_cast<uintptr_t>(row) & 15u) == 0};
 }
 
 // Running (digit, count) pair of one thread: equal neighbouring digits are
-// merged before they reach the shared-memory histogram.  Normalised scores
-// share their exponent bits, so the leading digits are nearly constant.
+// merged before they reach the shared-memory histogram, which keeps runs of
+// equal scores (padding, constant rows) from hammering one bin.
 struct DigitRun {
   uint32_t digit = 0, count = 0;
   __device__ __forceinline__ void add(uint32_t d, uint32_t* hist) {
@@ -168,33 +183,31 @@ struct DigitRun {
 
 constexpr int kSelUnroll = 4;                              // quads in flight per thread
 
-// Adds the candidates [lo, hi) with key <= ceiling whose bits under `mask`
-// equal `prefix` to the histogram of this pass's digit.  Whole CTA.
-__device__ __forceinline__ void digit_histogram(const RowKeys& keys, int lo, int hi, uint32_t ceiling,
-                                                uint32_t mask, uint32_t prefix, int pass,
-                                                uint32_t* hist) {
+// Adds the keys <= ceiling whose bits under `mask` equal `prefix` to the
+// histogram of this pass's digit.  Whole CTA.
+__device__ __forceinline__ void digit_histogram(const RowKeys& keys, uint32_t ceiling, uint32_t mask,
+                                                uint32_t prefix, int pass, uint32_t* hist) {
+  const int quads = keys.quads(), step = (int)blockDim.x;
   const int shift = pass_shift(pass);
   const uint32_t dmask = pass_digit_mask(pass);
-  if (hi <= lo) return;
-  const int q_lo = lo >> 2, q_hi = (hi + 3) >> 2, step = (int)blockDim.x;
   DigitRun run;
-  for (int q0 = q_lo + (int)threadIdx.x; q0 < q_hi; q0 += kSelUnroll * step) {
+  for (int q0 = (int)threadIdx.x; q0 < quads; q0 += kSelUnroll * step) {
     uint4 v[kSelUnroll];
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u)
-      if (q0 + u * step < q_hi) v[u] = keys.load4(q0 + u * step);
+      if (q0 + u * step < quads) v[u] = keys.load4(q0 + u * step);
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u) {
-      const int q = q0 + u * step;
-      if (q < q_hi) {
+      if (q0 + u * step < quads) {
         const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-        const bool edge = 4 * q < lo || 4 * q + 3 >= hi;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint32_t key = k4[i];
-          if (edge && (4 * q + i < lo || 4 * q + i >= hi)) continue;
-          if (key > ceiling || (key & mask) != prefix) continue;
-          run.add((key >> shift) & dmask, hist);
+          if (pass == 0) {                                 // every key takes part: merge runs
+            if (key <= ceiling) run.add(key >> shift, hist);
+          } else if ((key & mask) == prefix && key <= ceiling) {
+            atomicAdd(&hist[(key >> shift) & dmask], 1u);  // few keys share the prefix
+          }
         }
       }
     }
@@ -202,12 +215,10 @@ __device__ __forceinline__ void digit_histogram(const RowKeys& keys, int lo, int
   run.flush(hist);
 }
 
-// Copies the keys of a row into shared memory and, on the way, builds the
-// histogram of the leading digit of the candidates [lo, hi).  Whole CTA;
-// hist must be zero on entry.
-__device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, int lo, int hi,
-                                           uint32_t* hist) {
-  const int quads = (src.n + 3) >> 2, step = (int)blockDim.x;
+// Copies the rank keys of a row into shared memory and, on the way, builds the
+// histogram of their leading digit.  Whole CTA; hist must be zero on entry.
+__device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, uint32_t* hist) {
+  const int quads = src.quads(), step = (int)blockDim.x;
   DigitRun run;
   for (int q0 = (int)threadIdx.x; q0 < quads; q0 += kSelUnroll * step) {
     uint4 v[kSelUnroll];
@@ -216,30 +227,29 @@ __device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, in
       if (q0 + u * step < quads) v[u] = src.load4(q0 + u * step);
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u) {
-      const int q = q0 + u * step;
-      if (q < quads) {
-        staged[q] = v[u];
-        const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (4 * q + i >= lo && 4 * q + i < hi) run.add(k4[i] >> 20, hist);
+      if (q0 + u * step < quads) {
+        staged[q0 + u * step] = v[u];
+        run.add(v[u].x >> 20, hist);
+        run.add(v[u].y >> 20, hist);
+        run.add(v[u].z >> 20, hist);
+        run.add(v[u].w >> 20, hist);
       }
     }
   }
   run.flush(hist);
 }
 
-// Top-kk cut of the candidates [lo, hi) of one row (0 < kk < hi - lo).  Whole
-// CTA.  With first_hist_ready the leading-digit histogram is already in
-// sm.hist (built by stage_keys).
-__device__ __forceinline__ Cut local_cut(const RowKeys& keys, int lo, int hi, int kk, SelectSmem& sm,
+// Cut that keeps the `want` largest keys of a row (0 < want <= n).  Whole CTA.
+// With first_hist_ready the leading-digit histogram is already in sm.hist
+// (built by stage_keys).
+__device__ __forceinline__ Cut local_cut(const RowKeys& keys, int want, SelectSmem& sm,
                                          bool first_hist_ready) {
-  uint32_t prefix = 0, mask = 0, remaining = (uint32_t)kk;
+  uint32_t prefix = 0, mask = 0, remaining = (uint32_t)want;
   for (int pass = 0; pass < kSelPasses; ++pass) {
     if (!(first_hist_ready && pass == 0)) {
       clear_hist(sm.hist);
       __syncthreads();
-      digit_histogram(keys, lo, hi, 0xffffffffu, mask, prefix, pass, sm.hist);
+      digit_histogram(keys, 0xffffffffu, mask, prefix, pass, sm.hist);
     }
     __syncthreads();
     pick_digit(sm.hist, remaining, sm);
@@ -248,37 +258,26 @@ __device__ __forceinline__ Cut local_cut(const RowKeys& keys, int lo, int hi, in
     remaining = sm.remaining;
     __syncthreads();
   }
-  return Cut{prefix, remaining, true};
+  return Cut{prefix, remaining};
 }
 
-// Ordered compaction of one row: forced tokens, keys above cut.T and the first
-// cut.eq_take keys equal to cut.T, written to `out` in ascending token order.
-// Every warp owns a contiguous run of quads; a first sweep counts what each
-// warp keeps, one scan over the warp totals places the warps, a second sweep
-// writes.  Whole CTA, blockDim = 1024.
-__device__ __forceinline__ void ordered_compact(const RowKeys& keys, const ForcedSet& F,
-                                                const Cut& cut, int32_t* out, SelectSmem& sm) {
+// Ordered compaction of one row: the tokens whose key is above cut.T and the
+// first cut.eq_take tokens whose key equals cut.T, written to `out` in
+// ascending token order.  Every warp owns a contiguous run of quads; a first
+// sweep counts what each warp keeps, one scan over the warp totals places the
+// warps, a second sweep writes.  Whole CTA, blockDim = 1024.
+__device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Cut& cut, int32_t* out,
+                                                SelectSmem& sm) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int n = keys.n, quads = (n + 3) >> 2;
+  const int quads = keys.quads();
   const int per_warp = (((quads + 31) >> 5) + 31) & ~31;   // quads per warp, whole warp sweeps
   const int q_begin = min(warp * per_warp, quads), q_end = min(q_begin + per_warp, quads);
+  const uint32_t T = cut.T;
 
-  // flags of the four tokens of quad q: bits 0-3 kept for sure, bits 4-7 equal to the cut
-  auto classify = [&](int q, const uint4& v) -> uint32_t {
-    const uint32_t k4[4] = {v.x, v.y, v.z, v.w};
-    uint32_t f = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int j = 4 * q + i;
-      if (j < n) {
-        if (j < F.sinks || j >= F.hi) f |= 1u << i;
-        else if (cut.any) {
-          if (k4[i] > cut.T) f |= 1u << i;
-          else if (k4[i] == cut.T) f |= 16u << i;
-        }
-      }
-    }
-    return f;
+  // flags of the four tokens of a quad: bits 0-3 key above the cut, bits 4-7 key equal to it
+  auto classify = [&](const uint4& v) -> uint32_t {
+    return (v.x > T ? 1u : 0u) | (v.y > T ? 2u : 0u) | (v.z > T ? 4u : 0u) | (v.w > T ? 8u : 0u) |
+           (v.x == T ? 16u : 0u) | (v.y == T ? 32u : 0u) | (v.z == T ? 64u : 0u) | (v.w == T ? 128u : 0u);
   };
 
   uint32_t def_cnt = 0, eq_cnt = 0;
@@ -290,7 +289,7 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Force
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u) {
       if (q0 + u * 32 < q_end) {
-        const uint32_t f = classify(q0 + u * 32, v[u]);
+        const uint32_t f = classify(v[u]);
         def_cnt += __popc(f & 15u);
         eq_cnt += __popc(f >> 4);
       }
@@ -319,7 +318,7 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Force
   for (int q0 = q_begin; q0 < q_end; q0 += 32) {           // uniform trip count across the warp
     const int q = q0 + lane;
     uint32_t f = 0;
-    if (q < q_end) f = classify(q, keys.load4(q));
+    if (q < q_end) f = classify(keys.load4(q));
     const uint32_t mine = (uint32_t)__popc(f & 15u) | ((uint32_t)__popc(f >> 4) << 16);
     uint32_t inc = mine;
 #pragma unroll
@@ -329,14 +328,16 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Force
     }
     const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
     uint32_t d = def_before + ((inc - mine) & 0xffffu), e = eq_before + ((inc - mine) >> 16);
+    if (f) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if (f & (1u << i)) {
-        out[d + min(e, cut.eq_take)] = 4 * q + i;
-        ++d;
-      } else if (f & (16u << i)) {
-        if (e < cut.eq_take) out[d + e] = 4 * q + i;
-        ++e;
+      for (int i = 0; i < 4; ++i) {
+        if (f & (1u << i)) {
+          out[d + min(e, cut.eq_take)] = 4 * q + i;
+          ++d;
+        } else if (f & (16u << i)) {
+          if (e < cut.eq_take) out[d + e] = 4 * q + i;
+          ++e;
+        }
       }
     }
     def_before += total & 0xffffu;
@@ -361,25 +362,28 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
   if (head_budgets != nullptr) k = max(0, min(head_budgets[p], budget));
   const int k_eff = min(k, n);
   const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  RowKeys keys = global_keys(scores + (size_t)p * n_max, n);
+  RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
   int32_t* out = idx + (size_t)p * budget;
-  const int cand = F.hi - F.sinks;
 
-  Cut cut{0u, 0u, F.free_slots > 0};
-  if (F.free_slots >= cand) {
-    cut.eq_take = (uint32_t)max(cand, 0);                  // every candidate is kept
-  } else if (cut.any) {
-    const bool stage = ((n + 3) >> 2) <= stage_quads;      // the row fits in shared memory
+  Cut cut;
+  if (k_eff == 0) {
+    cut = keep_nothing();
+  } else if (k_eff == n) {
+    cut = keep_every_token();
+  } else if (F.free_slots == 0) {
+    cut = keep_forced_only();
+  } else {
+    const bool stage = keys.quads() <= stage_quads;        // the row fits in shared memory
     if (stage) {
       clear_hist(sm.hist);
       __syncthreads();
-      stage_keys(keys, staged_keys, F.sinks, F.hi, sm.hist);
+      stage_keys(keys, staged_keys, sm.hist);
       keys.staged = staged_keys;
     }
-    cut = local_cut(keys, F.sinks, F.hi, F.free_slots, sm, stage);
+    cut = local_cut(keys, k_eff, sm, stage);
   }
 
-  ordered_compact(keys, F, cut, out, sm);
+  ordered_compact(keys, cut, out, sm);
   for (int t = k_eff + tid; t < budget; t += kSelThreads) out[t] = -1;
   if (tid == 0) {
     counts[p] = k_eff;
@@ -418,19 +422,17 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   const int n = seq_len_of(seqlens, b, n_max);
   const int k_eff = min(budget, n);
   const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  const RowKeys keys = global_keys(scores + (size_t)p * n_max, n);
-  const int cand = F.hi - F.sinks;
+  const RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
   const int forced = k_eff - F.free_slots;
   const int prot = min(max(min_protected, forced), k_eff);  // protected rows per head, forced included
-  const int pp = prot - forced;                             // protected candidates
 
-  // ---- this head's safeguard share
-  const bool prot_all = pp >= cand;                         // every candidate is protected
-  const bool prot_none = pp == 0 && !prot_all;
-  Cut own{0u, 0u, false};
-  if (!prot_all && !prot_none) own = local_cut(keys, F.sinks, F.hi, pp, sm.s, false);
-  // unprotected keys: candidates with key <= ceiling, minus the first own.eq_take equal to it
-  const uint32_t ceiling = prot_none ? 0xffffffffu : own.T;
+  // ---- this head's safeguard share: its `prot` largest keys
+  Cut own = keep_nothing();
+  if (prot >= n) own = keep_every_token();
+  else if (prot > 0 && prot == forced) own = Cut{kForcedKey, (uint32_t)forced};
+  else if (prot > 0) own = local_cut(keys, prot, sm.s, false);
+  // unprotected keys: those <= own.T, minus the first own.eq_take equal to it
+  const uint32_t ceiling = own.T;
 
   // ---- layer-wide cut over the unprotected keys of all heads
   const uint32_t pool = (uint32_t)heads * (uint32_t)(k_eff - prot);
@@ -441,9 +443,9 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
       const int shift = pass_shift(pass);
       clear_hist(sm.hist_local);
       __syncthreads();
-      if (!prot_all) digit_histogram(keys, F.sinks, F.hi, ceiling, mask, prefix, pass, sm.hist_local);
+      digit_histogram(keys, ceiling, mask, prefix, pass, sm.hist_local);
       __syncthreads();
-      if (tid == 0 && !prot_all && !prot_none && (own.T & mask) == prefix)
+      if (tid == 0 && own.eq_take > 0 && (own.T & mask) == prefix)
         sm.hist_local[(own.T >> shift) & pass_digit_mask(pass)] -= own.eq_take;   // those are protected
       cluster.sync();
       {
@@ -475,17 +477,11 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   const uint32_t e_h = eq_g > eq_before_me ? min(eq_g - eq_before_me, local_eq) : 0u;
 
   // ---- this head's final cut and row count
-  Cut cut;
-  uint32_t kept;
-  if (prot_all) {
-    cut = Cut{0u, (uint32_t)max(cand, 0), cand > 0};
-    kept = (uint32_t)(forced + max(cand, 0));
-  } else {
-    kept = (uint32_t)prot + local_gt + e_h;
-    if (pool == 0) cut = Cut{own.T, own.eq_take, !prot_none};
-    else if (prot_none || Tg < own.T) cut = Cut{Tg, e_h, true};
-    else if (Tg == own.T) cut = Cut{own.T, own.eq_take + e_h, true};
-    else cut = Cut{own.T, own.eq_take, true};
+  const uint32_t kept = (uint32_t)prot + local_gt + e_h;
+  Cut cut = own;
+  if (pool > 0) {
+    if (Tg < own.T) cut = Cut{Tg, e_h};
+    else if (Tg == own.T) cut = Cut{own.T, own.eq_take + e_h};
   }
   if (tid == 0) sm.pub_count = kept;
   cluster.sync();
@@ -503,7 +499,7 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   for (int r = 0; r < h; ++r) off += *cluster.map_shared_rank(&sm.pub_count, r);
   __syncthreads();
 
-  ordered_compact(keys, F, cut, idx + off, sm.s);
+  ordered_compact(keys, cut, idx + off, sm.s);
   if (tid == 0) {
     counts[p] = (int32_t)kept;
     offsets[p] = (int32_t)off;
