@@ -193,6 +193,15 @@ curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, voi
  * set, CURDKV_OK otherwise (other bits are reported through *host_flags). */
 curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, void* cuda_stream);
 
+/* Profiling aid (no counterpart in the paper): asks the next curdkv_score or
+ * curdkv_score_static call of THIS host thread to record the two cudaEvent_t
+ * handles (passed as void*, either may be NULL) on its stream immediately
+ * before and after its sketch kernel -- the kernel that streams K and V -- so
+ * that a benchmark can time that kernel alone without a profiler.  The request
+ * is cleared by that call.  With projection off, per-head G or n_max < 128 the
+ * sketch runs on another kernel and nothing is recorded. */
+curdkv_status curdkv_profile_next_score(void* start_event, void* stop_event);
+
 /* Number of kernels this library has launched in this process so far. */
 uint64_t curdkv_launch_count(void);
 

@@ -24,6 +24,7 @@ EXPORTS = (
     "curdkv_workspace_bytes", "curdkv_score", "curdkv_select", "curdkv_compact",
     "curdkv_gqa_map", "curdkv_device_status", "curdkv_launch_count", "curdkv_status_string",
     "curdkv_score_static", "curdkv_host_arena_bytes", "curdkv_compress_host",
+    "curdkv_profile_next_score",
 )
 
 
@@ -77,6 +78,8 @@ def load():
     lib.curdkv_gqa_map.argtypes = [dp, vp, vp]
     lib.curdkv_device_status.restype = ctypes.c_int
     lib.curdkv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.curdkv_profile_next_score.restype = ctypes.c_int
+    lib.curdkv_profile_next_score.argtypes = [vp, vp]
     lib.curdkv_launch_count.restype = ctypes.c_uint64
     lib.curdkv_launch_count.argtypes = []
     lib.curdkv_status_string.restype = ctypes.c_char_p
@@ -259,6 +262,14 @@ def curdkv_compress_host(K_host, V_host, G_host, desc: Desc, budget: int, buffer
         _ptr(buffers.arena), buffers.arena.numel(), buffers.chunk_batch, ctypes.byref(flags))
     _check(code, "curdkv_compress_host")
     return int(flags.value)
+
+
+def curdkv_profile_next_score(start: torch.cuda.Event, stop: torch.cuda.Event) -> None:
+    """Have the next curdkv_score call of this thread record ``start`` / ``stop`` (timing events
+    that have been recorded at least once, so that their handles exist) around its sketch kernel."""
+    _check(load().curdkv_profile_next_score(ctypes.c_void_p(start.cuda_event),
+                                            ctypes.c_void_p(stop.cuda_event)),
+           "curdkv_profile_next_score")
 
 
 def curdkv_gqa_map(desc: Desc, device="cuda") -> torch.Tensor:

@@ -93,17 +93,26 @@ int sm_count() {
   return n;
 }
 
+// Events a caller asked to have recorded around the next sketch kernel of this
+// host thread (curdkv_profile_next_score).
+thread_local cudaEvent_t g_profile_start = nullptr, g_profile_stop = nullptr;
+
 template <int R>
 cudaError_t launch_umma(const CUtensorMap& mk, const CUtensorMap& mv, const umma::Args& a,
                         cudaStream_t stream) {
   using L = umma::Smem<R>;
+  const int smem = L::dynamic_bytes(a.seqlens != nullptr ? a.batch : 0);
   cudaError_t e = cudaFuncSetAttribute(umma::sketch_umma_kernel<R>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       L::dynamic_bytes(umma::kMaxRaggedBatch));
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
-  const unsigned grid = (unsigned)(a.total_tiles < sms ? a.total_tiles : sms);
-  umma::sketch_umma_kernel<R><<<grid, umma::kThreads, L::kDynamic, stream>>>(mk, mv, a);
+  const int64_t tiles = (int64_t)a.batch * a.heads * a.tiles_per_head;   // upper bound if ragged
+  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  if (g_profile_start != nullptr) cudaEventRecord(g_profile_start, stream);
+  umma::sketch_umma_kernel<R><<<grid, umma::kThreads, smem, stream>>>(mk, mv, a);
+  if (g_profile_stop != nullptr) cudaEventRecord(g_profile_stop, stream);
   return cudaSuccess;
 }
 
@@ -189,29 +198,43 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
   int parts = 1;                                  // partial sums per 128-row tile
   bool launched = false;
   if (desc->use_projection && !g_per_head && desc->n_max >= kTileRows) {
-    // tensor-core path: one G for all heads, TMA tiles of 128 rows
-    CUtensorMap mk, mv;
-    if (make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) &&
-        make_tile_map(&mv, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n)) {
+    // tensor-core path: one G for all heads, TMA tiles of 128 rows.  A ragged batch goes in
+    // slices of at most kMaxRaggedBatch sequences (the kernel keeps their tile prefix sums
+    // in shared memory).
+    const int slice = desc->seqlens != nullptr ? umma::kMaxRaggedBatch : desc->batch;
+    bool maps_ok = true;
+    for (int b0 = 0; b0 < desc->batch && maps_ok; b0 += slice) {
+      curdkv_desc part = *desc;
+      part.batch = desc->batch - b0 < slice ? desc->batch - b0 : slice;
+      const __nv_bfloat16* Kb = static_cast<const __nv_bfloat16*>(K) + (int64_t)b0 * desc->k_stride_b;
+      const __nv_bfloat16* Vb = static_cast<const __nv_bfloat16*>(V) + (int64_t)b0 * desc->v_stride_b;
+      CUtensorMap mk, mv;
+      maps_ok = make_tile_map(&mk, Kb, &part, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) &&
+                make_tile_map(&mv, Vb, &part, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n);
+      if (!maps_ok) break;
+      const size_t p0 = (size_t)b0 * desc->kv_heads;
       umma::Args u;
       u.G = G;
-      u.seqlens = desc->seqlens;
+      u.seqlens = desc->seqlens != nullptr ? desc->seqlens + b0 : nullptr;
+      u.batch = part.batch;
       u.heads = desc->kv_heads;
       u.n_max = desc->n_max;
       u.r = desc->r;
       u.tiles_per_head = tiles;
-      u.total_tiles = P * tiles;
       u.score_mode = desc->score_mode;
-      u.scores = scores;
-      u.tile_sums = a.tile_sums;
+      u.scores = scores + p0 * desc->n_max;
+      u.tile_sums = a.tile_sums + p0 * tiles * umma::kPartsPerTile;
       u.status = static_cast<uint32_t*>(workspace);
       const cudaError_t e = desc->r <= 32 ? launch_umma<32>(mk, mv, u, stream)
                                           : launch_umma<64>(mk, mv, u, stream);
       if (e != cudaSuccess) return CURDKV_ERR_CUDA;
+      if (!launch_ok()) return CURDKV_ERR_CUDA;
       parts = umma::kPartsPerTile;
       launched = true;
     }
+    if (launched && !maps_ok) return CURDKV_ERR_CUDA;      // a later slice could not be described
   }
+  g_profile_start = g_profile_stop = nullptr;
   if (!launched) {
     if (desc->use_projection) {
       const int r_pad = (desc->r + 31) / 32 * 32;
@@ -223,12 +246,13 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
     } else {
       row_norm_kernel<<<grid, 256, 0, stream>>>(a);
     }
+    if (!launch_ok()) return CURDKV_ERR_CUDA;
   }
-  if (!launch_ok()) return CURDKV_ERR_CUDA;
 
   const int chunks = (desc->n_max + kNormChunk - 1) / kNormChunk;
   normalise_kernel<<<(unsigned)(P * chunks), 256, 0, stream>>>(scores, a.tile_sums, head_sums,
-                                                              desc->n_max, tiles * parts, chunks);
+                                                              desc->seqlens, desc->kv_heads,
+                                                              desc->n_max, tiles, parts, chunks);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }
@@ -371,6 +395,12 @@ curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, 
       cudaMemcpyAsync(status_flags, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice,
                       static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
     return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_profile_next_score(void* start_event, void* stop_event) {
+  g_profile_start = static_cast<cudaEvent_t>(start_event);
+  g_profile_stop = static_cast<cudaEvent_t>(stop_event);
   return CURDKV_OK;
 }
 

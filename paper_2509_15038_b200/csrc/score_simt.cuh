@@ -185,29 +185,34 @@ __global__ void __launch_bounds__(256) sketch_fma_kernel(const ScoreArgs a, cons
 }
 
 // ---------------------------------------------------------------------------
-// Alg. 1 line 6: S = sum of the tile partials in a fixed order, scores /= S.
+// Alg. 1 line 6: S = sum of the partial sums of the head's valid tiles in a
+// fixed order, scores /= S; scores at or beyond the sequence length become 0.
 // grid = batch*heads*ceil(n_max / 4096) (chunk fastest), block = 256.
 // ---------------------------------------------------------------------------
 constexpr int kNormChunk = 4096;
 
 __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const float* tile_sums,
-                                                        float* head_sums, int n_max,
-                                                        int parts_per_head, int chunks_per_head) {
+                                                        float* head_sums, const int32_t* seqlens,
+                                                        int heads, int n_max, int tiles_per_head,
+                                                        int parts_per_tile, int chunks_per_head) {
   __shared__ float red[8];
   const int p = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = seq_len_of(seqlens, p / heads, n_max);
   float* row = scores + (size_t)p * n_max;
   const int j0 = chunk * kNormChunk;
   const int j1 = min(j0 + kNormChunk, n_max);
-  // this thread's scores are on their way while the head sum is formed
-  const bool vec = (reinterpret_cast<uintptr_t>(row) & 15u) == 0 && j1 - j0 == kNormChunk;
+  // a full chunk of valid scores is put on its way while the head sum is formed
+  const bool vec = (reinterpret_cast<uintptr_t>(row) & 15u) == 0 && j0 + kNormChunk <= n;
   float4 v[4];
   if (vec) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) v[u] = reinterpret_cast<const float4*>(row + j0)[tid + 256 * u];
   }
+  const int parts = ((n + kTileRows - 1) / kTileRows) * parts_per_tile;
+  const float* mine = tile_sums + (size_t)p * tiles_per_head * parts_per_tile;
   float part = 0.f;                                        // fixed order: thread, warp tree, warp order
-  for (int i = tid; i < parts_per_head; i += 256) part += tile_sums[(size_t)p * parts_per_head + i];
+  for (int i = tid; i < parts; i += 256) part += mine[i];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
   if (lane == 0) red[warp] = part;
@@ -228,7 +233,7 @@ __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const flo
       reinterpret_cast<float4*>(row + j0)[tid + 256 * u] = o;
     }
   } else {
-    for (int j = j0 + tid; j < j1; j += 256) row[j] = live ? __fdiv_rn(row[j], S) : 0.f;
+    for (int j = j0 + tid; j < j1; j += 256) row[j] = (live && j < n) ? __fdiv_rn(row[j], S) : 0.f;
   }
 }
 

@@ -18,7 +18,6 @@
 // Every mbarrier wait is bounded; on expiry the kernel flags
 // CURDKV_DEV_TIMEOUT, drains what it issued, frees TMEM and returns.
 #pragma once
-#include <climits>
 #include <cuda.h>
 
 #include "common.cuh"
@@ -37,15 +36,20 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct Args {
   const float* G;          // [128][r]
-  const int32_t* seqlens;
-  int heads, n_max, r;
-  int tiles_per_head;
-  long long total_tiles;   // batch*heads*tiles_per_head
+  const int32_t* seqlens;  // nullptr: every sequence has n_max rows
+  int batch, heads, n_max, r;
+  int tiles_per_head;      // ceil(n_max / kTileRows): row stride of tile_sums
   int score_mode;
   float* scores;
-  float* tile_sums;        // [total_tiles][kPartsPerTile]
+  float* tile_sums;        // [batch*heads][tiles_per_head][kPartsPerTile]
   uint32_t* status;
 };
+
+// Ragged batches: the kernel walks only the tiles that hold valid rows.  Every
+// CTA builds the exclusive prefix sums of the per-sequence tile counts in shared
+// memory and maps a running tile number to (sequence, head, tile) by binary
+// search, so all CTAs get the same number of real tiles.
+constexpr int kMaxRaggedBatch = 8192;                      // sequences per launch with seqlens
 
 template <int R>
 struct Smem {                                     // offsets from the 1024-aligned base
@@ -54,8 +58,11 @@ struct Smem {                                     // offsets from the 1024-align
   static constexpr int kG = 0;
   static constexpr int kSlot0 = 2 * kGHalf;
   static constexpr int kBar = kSlot0 + kSlots * kSlotBytes;
-  static constexpr int kTotal = kBar + 256;
-  static constexpr int kDynamic = kTotal + 1024;  // slack for manual alignment
+  static constexpr int kPrefix = kBar + 256;      // int32 [batch + 1], ragged launches only
+  static constexpr int kFixed = kPrefix + 1024;   // + slack for manual alignment
+  static constexpr int dynamic_bytes(int ragged_batch) {
+    return kFixed + (ragged_batch > 0 ? (ragged_batch + 1) * 4 : 0);
+  }
   static constexpr int kTmemCols = 4 * kN;        // 2 accumulator stages x {K, V} x N
 };
 
@@ -224,6 +231,27 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (a.seqlens != nullptr) {
+    // exclusive prefix sums of heads * ceil(n_b / 128): a chunk of sequences per thread,
+    // a scan over the chunk totals, then the running sums inside each chunk
+    uint32_t* pre = reinterpret_cast<uint32_t*>(base_ptr + L::kPrefix);
+    uint32_t* chunk_tot = reinterpret_cast<uint32_t*>(base_ptr + L::kSlot0);   // ring not in use yet
+    const int per = (a.batch + kThreads - 1) / kThreads;
+    const int b0 = min(tid * per, a.batch), b1 = min(b0 + per, a.batch);
+    uint32_t sum = 0;
+    for (int b = b0; b < b1; ++b)
+      sum += (uint32_t)a.heads * (uint32_t)((seq_len_of(a.seqlens, b, a.n_max) + kTileRows - 1) / kTileRows);
+    chunk_tot[tid] = sum;
+    __syncthreads();
+    uint32_t before = 0;
+    for (int i = 0; i < tid; ++i) before += chunk_tot[i];
+    for (int b = b0; b < b1; ++b) {
+      pre[b] = before;
+      before += (uint32_t)a.heads * (uint32_t)((seq_len_of(a.seqlens, b, a.n_max) + kTileRows - 1) / kTileRows);
+    }
+    if (tid == kThreads - 1) pre[a.batch] = before;
+    // made visible to every role by the barrier at the end of the set-up
+  }
   for (int i = tid; i < 128 * R; i += kThreads) {
     const int t = i / R, c = i % R;                        // channel t, sketch column c
     const float g = c < a.r ? __ldg(a.G + (size_t)t * a.r + c) : 0.f;
@@ -244,15 +272,32 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  const long long first = blockIdx.x, stride = gridDim.x;
-  // tile t -> problem p and first row; returns the head's valid rows n_b in a way that makes
-  // "result <= row0" mean "tile holds no valid row"
-  auto tile_rows = [&](long long t, int& p, int& row0) -> int {
-    p = (int)(t / a.tiles_per_head);
-    const int r0 = (int)(t % a.tiles_per_head) * kTileRows;
-    const int n = seq_len_of(a.seqlens, p / a.heads, a.n_max);
-    row0 = r0;
-    return n > r0 ? n : INT_MIN;
+  // ---- tile schedule: running tile number -> (problem p, first row, valid rows n)
+  const uint32_t* prefix = reinterpret_cast<const uint32_t*>(base_ptr + L::kPrefix);
+  uint32_t total_tiles;
+  if (a.seqlens != nullptr) {
+    total_tiles = prefix[a.batch];
+  } else {
+    total_tiles = (uint32_t)a.batch * (uint32_t)a.heads * (uint32_t)a.tiles_per_head;
+  }
+  const uint32_t first = blockIdx.x, stride = gridDim.x;
+  auto locate = [&](uint32_t t, int& p, int& row0) -> int {
+    if (a.seqlens == nullptr) {
+      p = (int)(t / (uint32_t)a.tiles_per_head);
+      row0 = (int)(t % (uint32_t)a.tiles_per_head) * kTileRows;
+      return a.n_max;
+    }
+    int lo = 0, hi = a.batch;                              // last b with prefix[b] <= t
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (prefix[mid] <= t) lo = mid; else hi = mid;
+    }
+    const int n = seq_len_of(a.seqlens, lo, a.n_max);
+    const uint32_t tiles_b = (uint32_t)((n + kTileRows - 1) / kTileRows);
+    const uint32_t local = t - prefix[lo];
+    p = lo * a.heads + (int)(local / tiles_b);
+    row0 = (int)(local % tiles_b) * kTileRows;
+    return n;
   };
 
   if (warp == 0) {
@@ -262,9 +307,9 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
       uint32_t it = 0;
       bool ok = true;
-      for (long long t = first; ok && t < a.total_tiles; t += stride) {
+      for (uint32_t t = first; ok && t < total_tiles; t += stride) {
         int p, row0;
-        if (tile_rows(t, p, row0) <= row0) continue;       // no valid row in this tile
+        locate(t, p, row0);
         const int b = p / a.heads, h = p % a.heads;
         for (int tensor = 0; tensor < 2; ++tensor, ++it) {
           const int slot = it % kSlots;
@@ -293,9 +338,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       constexpr uint32_t idesc = instr_desc_bf16(L::kN);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
-      for (long long t = first; ok && t < a.total_tiles; t += stride) {
-        int p, row0;
-        if (tile_rows(t, p, row0) <= row0) continue;
+      for (uint32_t t = first; ok && t < total_tiles; t += stride) {
         const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
         if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status))) break;
         tc_fence_after();
@@ -333,12 +376,12 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
     uint32_t tile_it = 0;
     bool ok = true;
-    for (long long t = first; ok && t < a.total_tiles; t += stride) {
+    for (uint32_t t = first; ok && t < total_tiles; t += stride) {
       int p, row0;
-      const int n = tile_rows(t, p, row0);
+      const int n = locate(t, p, row0);
       const int j = row0 + quarter * 32 + lane;
       float s = 0.f;
-      if (n > row0) {
+      {
         const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
         ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status);
         if (!(ok = __all_sync(0xffffffffu, ok))) break;    // the TMEM loads need the whole warp
@@ -357,7 +400,8 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
                      : "memory");
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      if (lane == 0) a.tile_sums[(size_t)t * kPartsPerTile + quarter] = s;
+      if (lane == 0)
+        a.tile_sums[((size_t)p * a.tiles_per_head + row0 / kTileRows) * kPartsPerTile + quarter] = s;
     }
   }
 
