@@ -84,6 +84,28 @@ def test_ragged_tail_and_sinks():
         full_pipeline_check(K, V, G, k, s, win, seqlens=lens, what=f"ragged s={s} w={win} k={k}")
 
 
+def test_ragged_batch_larger_than_one_kernel_slice():
+    """More ragged sequences than one sketch launch keeps prefix sums for: the batch is cut into
+    slices; lengths include 0 and non-multiples of the tile."""
+    B, H, n, d = 8200, 1, 256, 128
+    g = torch.Generator(device=DEV).manual_seed(11)
+    K = torch.randn((B, H, n, d), generator=g, device=DEV).to(torch.bfloat16)
+    V = torch.randn((B, H, n, d), generator=g, device=DEV).to(torch.bfloat16)
+    lens = np.random.default_rng(5).integers(0, n + 1, size=B).astype(np.int32)
+    lens[:4] = [0, 1, 129, 256]
+    G = synth.make_G(d, 32, seed=0)
+    desc, ws, scores, sums, sl = gpu_score(K, V, G, lens)
+    assert cur.curdkv_device_status(ws) == 0
+    rs, rS = orc.score(synth.to_u16(K), synth.to_u16(V), G, seqlens=lens)
+    pu.assert_scores_close(scores.cpu().numpy(), rs, "sliced ragged batch")
+    np.testing.assert_allclose(sums.cpu().numpy(), rS, rtol=1e-4)
+    idx, cnt, _ = cur.curdkv_select(scores, desc, 40, num_sink=2, window=8, workspace=ws)
+    eidx, ecnt = orc.select_fixed(scores.cpu().numpy().astype(np.float64), 40, num_sink=2, window=8,
+                                  seqlens=lens)
+    np.testing.assert_array_equal(cnt.cpu().numpy(), ecnt)
+    np.testing.assert_array_equal(idx.cpu().numpy(), eidx)
+
+
 def test_strided_token_major_layout():
     """K, V stored [B, n, H, d] (token-major) and viewed as [B, H, n, d]."""
     B, H, n, d = 2, 4, 640, 128
