@@ -437,3 +437,57 @@ def test_cache_byte_accounting_matches_paper_128k_figure():
     per_token = w.layers * w.batch * w.kv_heads * w.d * 2 * 2      # K and V, 2 bytes each
     assert per_token * w.n_max == 16 * 2 ** 30
     assert round(per_token * 128_000 / 2 ** 30, 1) == 15.6
+
+
+# --------------------------------------------------------------------------- generation phase
+def _history(B, H, N, d, seed, quantise=False):
+    rng = np.random.default_rng(seed)
+    K = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    V = rng.standard_normal((B, H, N, d)).astype(np.float32)
+    if quantise:                       # few distinct rows -> many exactly equal scores
+        K = np.round(K[:, :, :, :1] * 1.5) * np.ones((1, 1, 1, d), np.float32)
+        V = np.ones_like(V)
+    to_bits = lambda a: (a.view(np.uint32) >> 16).astype(np.uint16)     # truncation: still bf16 values
+    return to_bits(np.ascontiguousarray(K)), to_bits(np.ascontiguousarray(V))
+
+
+@pytest.mark.parametrize("quantise", [False, True])
+@pytest.mark.parametrize("k,s,w", [(24, 4, 0), (24, 0, 8), (24, 2, 6), (10, 4, 6), (200, 4, 8)])
+def test_generation_phase_equals_one_shot_selection(k, s, w, quantise):
+    """Sec. 3.2 (method applies during generation): compressing incrementally, on any schedule,
+    keeps exactly the tokens Alg. 1 keeps when applied once to the whole history."""
+    from oracle import curdkv_decode_oracle as dec
+
+    B, H, N, d, r = 2, 3, 150, 16, 8
+    Ku, Vu = _history(B, H, N, d, seed=k + 7 * s + w, quantise=quantise)
+    G = np.random.default_rng(1).standard_normal((d, r)).astype(np.float32) / np.sqrt(r)
+    for schedule in ([40, 1, 1, 1, 30, 17, 60], [150], [1] * 150, [64, 64, 22]):
+        cache = dec.CacheOracle(B, H, d)
+        at = 0
+        for step, t in enumerate(schedule):
+            cache.append(Ku[:, :, at:at + t], Vu[:, :, at:at + t], G)
+            at += t
+            if step % 2 == 1 or at == N:            # compress now and then, and at the end
+                cache.compress(k, s, w)
+        assert at == N
+        sc, _ = orc.score(Ku, Vu, G)
+        idx, cnt = orc.select_fixed(sc, k, s, w)
+        for b in range(B):
+            for h in range(H):
+                want = idx[b, h, : cnt[b, h]]
+                np.testing.assert_array_equal(cache.pos[b][h], want)
+                np.testing.assert_array_equal(cache.K[b][h], Ku[b, h, want])
+                np.testing.assert_array_equal(cache.V[b][h], Vu[b, h, want])
+
+
+def test_generation_phase_raw_scores_are_row_local():
+    """A row's unnormalised score does not depend on which other rows are scored with it."""
+    from oracle import curdkv_decode_oracle as dec
+
+    Ku, Vu = _history(1, 2, 40, 16, seed=3)
+    G = np.random.default_rng(2).standard_normal((16, 8)).astype(np.float32)
+    full = dec.raw_scores(Ku, Vu, G)
+    part = dec.raw_scores(Ku[:, :, 10:25], Vu[:, :, 10:25], G)
+    np.testing.assert_array_equal(full[:, :, 10:25], part)
+    sc, S = orc.score(Ku, Vu, G)
+    np.testing.assert_allclose(full / S[..., None], sc, rtol=1e-14)
