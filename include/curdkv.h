@@ -51,6 +51,7 @@ typedef enum curdkv_status {
 /* Bits of the device status word (workspace[0], int32). */
 #define CURDKV_DEV_TIMEOUT 0x1u   /* a pipeline wait gave up; results of that launch are invalid */
 #define CURDKV_DEV_BAD_INDEX 0x2u /* an index outside [0, n) was skipped by the gather           */
+#define CURDKV_DEV_CACHE_FULL 0x4u /* curdkv_cache_append dropped rows that exceeded the capacity */
 
 /* Shape of one call: K and V are bf16 tensors addressed as
  *   K[b][h][j][c] = K_base[b*k_stride_b + h*k_stride_h + j*k_stride_n + c]
@@ -72,6 +73,9 @@ typedef struct curdkv_desc {
   int32_t score_mode;     /* 0: l = lK * lV (Alg. 1 line 5)  1: key only  2: value only
                              (ablation of App. C.3)                                         */
   int32_t use_projection; /* 1: sketch with G (Alg. 1 lines 2-3); 0: raw squared row norms  */
+  int32_t raw_scores;     /* 0: normalise per head (Alg. 1 line 6); 1: leave l^KV of line 5 as
+                             it is (head_sums is still written) -- what the generation-phase
+                             cache stores, since a row's l^KV does not depend on other rows  */
 } curdkv_desc;
 
 /* Bytes of device workspace the calls below need for this shape (256-byte
@@ -182,6 +186,50 @@ curdkv_status curdkv_compress_host(const void* K_host, const void* V_host, const
                                    void* K_out_host, void* V_out_host, int32_t* idx_host,
                                    int32_t* counts_host, int32_t* offsets_host, void* arena,
                                    size_t arena_bytes, int32_t chunk_batch, uint32_t* status_flags_host);
+
+/* ---- Generation phase (Sec. 3.2: "can be applied during the pre-filling as well as
+ * the token generation phase"; the paper leaves the procedure open).  Reading used:
+ * a cache holds, per (sequence, KV head), up to `capacity` rows of K and V with their
+ * original token positions and their unnormalised scores l^KV (Alg. 1 lines 2-5).
+ * curdkv_cache_append scores newly generated rows and appends them;
+ * curdkv_cache_compress applies Alg. 1 lines 6-10 to the rows held at that moment
+ * (sinks = positions < num_sink, window = the most recent `window` rows, the
+ * best-scoring rest up to `budget`, ascending position order).  Incremental
+ * compression keeps exactly the tokens a single application of Alg. 1 to the whole
+ * history would keep.  All heads of a sequence hold the same number of rows.
+ * Every pointer is a device pointer owned by the caller. */
+typedef struct curdkv_cache {
+  void* K;          /* bf16 [batch][kv_heads][capacity][d], dense                      */
+  void* V;
+  float* raw;       /* fp32 [batch][kv_heads][capacity]: l^KV of the held rows          */
+  int32_t* pos;     /* int32 [batch][kv_heads][capacity]: token position of each row    */
+  int32_t* count;   /* int32 [batch]: rows held per head; the caller zeroes it at start */
+  int32_t* total;   /* int32 [batch]: tokens appended so far (= next position); idem    */
+  int32_t capacity;
+} curdkv_cache;
+
+/* Workspace (256-byte aligned) for the two calls below: `t_max` = most rows appended
+ * per head in one call, `budget` = largest budget compressed to.  0 = invalid. */
+size_t curdkv_cache_workspace_bytes(int32_t batch, int32_t kv_heads, int32_t t_max,
+                                    int32_t capacity, int32_t budget);
+
+/* Appends K_new, V_new (bf16, described by desc_new exactly as in curdkv_score:
+ * n_max = rows offered per head, seqlens = device int32 [batch] rows that are real,
+ * or NULL) to the cache with their positions and l^KV under G.  Rows that would
+ * exceed `capacity` are dropped and CURDKV_DEV_CACHE_FULL is set in the status word
+ * (workspace[0]).  desc_new->raw_scores and ->score_mode are ignored (l^K * l^V). */
+curdkv_status curdkv_cache_append(const curdkv_cache* cache, const void* K_new, const void* V_new,
+                                  const float* G, int32_t g_per_head, const curdkv_desc* desc_new,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Alg. 1 lines 6-10 on the rows held in `in`; the kept rows, scores and positions go
+ * to `out` (a different cache with capacity >= min(budget, in->capacity); the two
+ * must not overlap), which also receives the counters.  Sequences holding at most
+ * `budget` rows are copied unchanged.  desc supplies batch, kv_heads and d. */
+curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* out,
+                                    const curdkv_desc* desc, int32_t budget, int32_t num_sink,
+                                    int32_t window, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream);
 
 /* GQA (Sec. 3.2): query head q uses KV head q / (q_heads / kv_heads).  Writes
  * kv_head_of_q int32 [q_heads] (device) so that attention consumers can index

@@ -24,7 +24,8 @@ EXPORTS = (
     "curdkv_workspace_bytes", "curdkv_score", "curdkv_select", "curdkv_compact",
     "curdkv_gqa_map", "curdkv_device_status", "curdkv_launch_count", "curdkv_status_string",
     "curdkv_score_static", "curdkv_host_arena_bytes", "curdkv_compress_host",
-    "curdkv_profile_next_score",
+    "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
+    "curdkv_cache_compress",
 )
 
 
@@ -42,6 +43,17 @@ class Desc(ctypes.Structure):
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_n", ctypes.c_int64),
         ("seqlens", ctypes.c_void_p),
         ("score_mode", ctypes.c_int32), ("use_projection", ctypes.c_int32),
+        ("raw_scores", ctypes.c_int32),
+    ]
+
+
+class Cache(ctypes.Structure):
+    """``curdkv_cache``: device pointers of one layer's generation-phase cache."""
+
+    _fields_ = [
+        ("K", ctypes.c_void_p), ("V", ctypes.c_void_p), ("raw", ctypes.c_void_p),
+        ("pos", ctypes.c_void_p), ("count", ctypes.c_void_p), ("total", ctypes.c_void_p),
+        ("capacity", ctypes.c_int32),
     ]
 
 
@@ -78,6 +90,13 @@ def load():
     lib.curdkv_gqa_map.argtypes = [dp, vp, vp]
     lib.curdkv_device_status.restype = ctypes.c_int
     lib.curdkv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    cp = ctypes.POINTER(Cache)
+    lib.curdkv_cache_workspace_bytes.restype = ctypes.c_size_t
+    lib.curdkv_cache_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.curdkv_cache_append.restype = ctypes.c_int
+    lib.curdkv_cache_append.argtypes = [cp, vp, vp, vp, i32, dp, vp, ctypes.c_size_t, vp]
+    lib.curdkv_cache_compress.restype = ctypes.c_int
+    lib.curdkv_cache_compress.argtypes = [cp, cp, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
     lib.curdkv_profile_next_score.restype = ctypes.c_int
     lib.curdkv_profile_next_score.argtypes = [vp, vp]
     lib.curdkv_launch_count.restype = ctypes.c_uint64
@@ -114,7 +133,7 @@ def _check(code: int, what: str):
 
 def make_desc(K: torch.Tensor, V: torch.Tensor, r: int, *, q_heads: Optional[int] = None,
               seqlens: Optional[torch.Tensor] = None, score_mode: int = 0,
-              use_projection: int = 1) -> Desc:
+              use_projection: int = 1, raw_scores: int = 0) -> Desc:
     """Descriptor of bf16 K, V ``[B, Hkv, n_max, d]`` (any strides with d contiguous)."""
     if K.dtype != torch.bfloat16 or V.dtype != torch.bfloat16:
         raise TypeError("K and V must be bf16")
@@ -127,7 +146,7 @@ def make_desc(K: torch.Tensor, V: torch.Tensor, r: int, *, q_heads: Optional[int
     return Desc(B, H, q_heads or H, n, d, int(r),
                 K.stride(0), K.stride(1), K.stride(2), V.stride(0), V.stride(1), V.stride(2),
                 seqlens.data_ptr() if seqlens is not None else None,
-                int(score_mode), int(use_projection))
+                int(score_mode), int(use_projection), int(raw_scores))
 
 
 def workspace_bytes(desc: Desc, max_budget: int = 0, adaptive: bool = False) -> int:
@@ -262,6 +281,50 @@ def curdkv_compress_host(K_host, V_host, G_host, desc: Desc, budget: int, buffer
         _ptr(buffers.arena), buffers.arena.numel(), buffers.chunk_batch, ctypes.byref(flags))
     _check(code, "curdkv_compress_host")
     return int(flags.value)
+
+
+class DeviceCache:
+    """Torch-owned buffers of one generation-phase cache plus the ``curdkv_cache`` view of them."""
+
+    def __init__(self, batch: int, kv_heads: int, capacity: int, d: int, device="cuda"):
+        self.batch, self.kv_heads, self.capacity, self.d = batch, kv_heads, capacity, d
+        self.K = torch.zeros((batch, kv_heads, capacity, d), dtype=torch.bfloat16, device=device)
+        self.V = torch.zeros_like(self.K)
+        self.raw = torch.zeros((batch, kv_heads, capacity), dtype=torch.float32, device=device)
+        self.pos = torch.full((batch, kv_heads, capacity), -1, dtype=torch.int32, device=device)
+        self.count = torch.zeros((batch,), dtype=torch.int32, device=device)
+        self.total = torch.zeros((batch,), dtype=torch.int32, device=device)
+        self.c = Cache(self.K.data_ptr(), self.V.data_ptr(), self.raw.data_ptr(), self.pos.data_ptr(),
+                       self.count.data_ptr(), self.total.data_ptr(), capacity)
+
+
+def cache_workspace(batch: int, kv_heads: int, t_max: int, capacity: int, budget: int,
+                    device="cuda") -> torch.Tensor:
+    nbytes = int(load().curdkv_cache_workspace_bytes(batch, kv_heads, t_max, capacity, budget))
+    if nbytes == 0:
+        raise ValueError("invalid shape for the generation-phase cache")
+    return torch.zeros((nbytes,), dtype=torch.uint8, device=device)
+
+
+def curdkv_cache_append(cache: DeviceCache, K_new, V_new, G, workspace: torch.Tensor, *,
+                        t_new: Optional[torch.Tensor] = None) -> None:
+    """Sec. 3.2, generation phase: score K_new, V_new ``[B, Hkv, t, d]`` and append them."""
+    desc = make_desc(K_new, V_new, G.shape[-1], seqlens=t_new)
+    code = load().curdkv_cache_append(ctypes.byref(cache.c), _ptr(K_new), _ptr(V_new), _ptr(G),
+                                      int(G.dim() == 3), ctypes.byref(desc), _ptr(workspace),
+                                      workspace.numel(), _stream())
+    _check(code, "curdkv_cache_append")
+
+
+def curdkv_cache_compress(src: DeviceCache, dst: DeviceCache, budget: int, workspace: torch.Tensor, *,
+                          num_sink: int = 0, window: int = 0) -> None:
+    """Alg. 1 lines 6-10 on the rows held in ``src``; survivors go to ``dst``."""
+    desc = Desc(src.batch, src.kv_heads, src.kv_heads, src.capacity, src.d, 1)
+    desc.use_projection = 1
+    code = load().curdkv_cache_compress(ctypes.byref(src.c), ctypes.byref(dst.c), ctypes.byref(desc),
+                                        int(budget), int(num_sink), int(window), _ptr(workspace),
+                                        workspace.numel(), _stream())
+    _check(code, "curdkv_cache_compress")
 
 
 def curdkv_profile_next_score(start: torch.cuda.Event, stop: torch.cuda.Event) -> None:

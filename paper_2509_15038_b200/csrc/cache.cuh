@@ -1,0 +1,97 @@
+// Bookkeeping kernels of the generation-phase cache (Sec. 3.2: the method also
+// applies while tokens are generated): rows are appended with their
+// unnormalised scores l^KV (Alg. 1 lines 2-5) and original positions, and a
+// compression step carries scores and positions along with the gathered rows.
+#pragma once
+#include "common.cuh"
+
+namespace curdkv {
+
+struct CacheView {
+  __nv_bfloat16* K;
+  __nv_bfloat16* V;        // [batch][heads][capacity][d]
+  float* raw;              // [batch][heads][capacity]
+  int32_t* pos;            // [batch][heads][capacity]
+  int32_t* count;          // [batch]
+  int32_t* total;          // [batch]
+  int capacity;
+};
+
+struct AppendArgs {
+  CacheView cache;
+  KvView K_new, V_new;     // [batch][heads][t][d]
+  const float* raw_new;    // [batch][heads][t]
+  const int32_t* t_new;    // [batch] or nullptr (every sequence brings t rows)
+  int heads, t, d;
+  uint32_t* status;
+};
+
+constexpr int kAppendWarps = 8;
+constexpr int kAppendRowsPerCta = 32;
+
+// grid = batch*heads*ceil(t / 32), block = 256: a half-warp per row (K in lanes
+// 0-15, V in lanes 16-31).  Rows that do not fit under `capacity` are dropped
+// and flagged.  Reads count/total, never writes them (cache_advance_kernel does).
+__global__ void __launch_bounds__(kAppendWarps * 32) cache_append_kernel(const AppendArgs a) {
+  const int chunks_per_head = (a.t + kAppendRowsPerCta - 1) / kAppendRowsPerCta;
+  const int p = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;
+  const int b = p / a.heads, h = p % a.heads;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+  int tb = a.t_new != nullptr ? a.t_new[b] : a.t;
+  tb = tb < 0 ? 0 : (tb > a.t ? a.t : tb);
+  const int held = a.cache.count[b];
+  const int room = a.cache.capacity - held;
+  if (tb > room) {
+    if (threadIdx.x == 0 && chunk == 0) flag_status(a.status, CURDKV_DEV_CACHE_FULL);
+    tb = room > 0 ? room : 0;
+  }
+  const int first_pos = a.cache.total[b];
+  const KvView& T = half ? a.V_new : a.K_new;
+  const __nv_bfloat16* src = T.base + b * T.stride_b + h * T.stride_h;
+  __nv_bfloat16* dst = (half ? a.cache.V : a.cache.K) + ((size_t)p * a.cache.capacity + held) * a.d;
+  const int chunks = a.d >> 3;
+  for (int i = chunk * kAppendRowsPerCta + warp; i < min((chunk + 1) * kAppendRowsPerCta, tb);
+       i += kAppendWarps) {
+    for (int c = l16; c < chunks; c += 16)
+      reinterpret_cast<uint4*>(dst + (size_t)i * a.d)[c] =
+          __ldg(reinterpret_cast<const uint4*>(src + i * T.stride_n) + c);
+    if (lane == 0) {
+      a.cache.raw[(size_t)p * a.cache.capacity + held + i] = a.raw_new[(size_t)p * a.t + i];
+      a.cache.pos[(size_t)p * a.cache.capacity + held + i] = first_pos + i;
+    }
+  }
+}
+
+// count[b] += rows that fitted, total[b] += rows offered.  grid = ceil(batch / 256).
+__global__ void cache_advance_kernel(CacheView cache, const int32_t* t_new, int t, int batch) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  int tb = t_new != nullptr ? t_new[b] : t;
+  tb = tb < 0 ? 0 : (tb > t ? t : tb);
+  const int room = cache.capacity - cache.count[b];
+  cache.count[b] += tb < room ? tb : (room > 0 ? room : 0);
+  cache.total[b] += tb;
+}
+
+// Scores, positions and counters of the rows a compression keeps.
+// grid = batch*heads, block = 256.  idx: [batch][heads][budget]; counts: [batch][heads].
+__global__ void __launch_bounds__(256) cache_gather_meta_kernel(const CacheView in, const CacheView out,
+                                                                const int32_t* idx, int budget,
+                                                                const int32_t* counts, int heads) {
+  const int p = blockIdx.x, b = p / heads, h = p % heads;
+  const int kept = min(counts[p], out.capacity);
+  const int held = in.count[b];
+  for (int t = threadIdx.x; t < kept; t += blockDim.x) {
+    const int j = idx[(size_t)p * budget + t];
+    if (j >= 0 && j < held) {
+      out.raw[(size_t)p * out.capacity + t] = in.raw[(size_t)p * in.capacity + j];
+      out.pos[(size_t)p * out.capacity + t] = in.pos[(size_t)p * in.capacity + j];
+    }
+  }
+  if (h == 0 && threadIdx.x == 0) {
+    out.count[b] = kept;
+    out.total[b] = in.total[b];
+  }
+}
+
+}  // namespace curdkv

@@ -15,6 +15,9 @@ constexpr int kTileRows = 128;
 // Workspace layout: [0, 256) status words, then tile partial sums.
 constexpr size_t kStatusBytes = 256;
 
+// Adds one to the library's launch counter (defined beside the C ABI).
+void count_launch();
+
 struct KvView {          // one bf16 tensor [batch][heads][n_max][d], strides in elements
   const __nv_bfloat16* base;
   int64_t stride_b, stride_h, stride_n;

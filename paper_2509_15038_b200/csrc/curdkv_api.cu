@@ -29,6 +29,7 @@ curdkv_status check_desc(const curdkv_desc* d) {
   if (d->q_heads < d->kv_heads || d->q_heads % d->kv_heads != 0) return CURDKV_ERR_INVALID_ARG;
   if (d->score_mode < 0 || d->score_mode > 2) return CURDKV_ERR_INVALID_ARG;
   if (d->use_projection != 0 && d->use_projection != 1) return CURDKV_ERR_INVALID_ARG;
+  if (d->raw_scores != 0 && d->raw_scores != 1) return CURDKV_ERR_INVALID_ARG;
   if ((int64_t)d->batch * d->kv_heads > (int64_t)1 << 24) return CURDKV_ERR_UNSUPPORTED;
   return CURDKV_OK;
 }
@@ -147,6 +148,10 @@ KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
 
 }  // namespace
 
+namespace curdkv {
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+}  // namespace curdkv
+
 extern "C" {
 
 size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32_t adaptive) {
@@ -252,7 +257,8 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
   const int chunks = (desc->n_max + kNormChunk - 1) / kNormChunk;
   normalise_kernel<<<(unsigned)(P * chunks), 256, 0, stream>>>(scores, a.tile_sums, head_sums,
                                                               desc->seqlens, desc->kv_heads,
-                                                              desc->n_max, tiles, parts, chunks);
+                                                              desc->n_max, tiles, parts, chunks,
+                                                              desc->raw_scores);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }

@@ -1,0 +1,155 @@
+// Generation-phase cache (Sec. 3.2): append newly generated rows with their
+// l^KV, compress the held rows with Alg. 1 lines 6-10.  Built on the public
+// entry points of curdkv.h plus the bookkeeping kernels of cache.cuh.
+#include <cstdint>
+
+#include "cache.cuh"
+#include "common.cuh"
+
+namespace {
+
+using namespace curdkv;
+
+inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
+
+struct CacheWorkspace {     // byte offsets from the workspace base
+  size_t score_ws, raw_new, sums, idx, counts, total;
+};
+
+bool layout(int32_t batch, int32_t heads, int32_t t_max, int32_t capacity, int32_t budget,
+            CacheWorkspace* L) {
+  if (batch < 0 || heads < 1 || t_max < 0 || capacity < 1 || budget < 0) return false;
+  curdkv_desc d = {};
+  d.batch = batch;
+  d.kv_heads = d.q_heads = heads;
+  d.n_max = t_max;
+  d.d = 128;
+  d.r = 1;
+  d.use_projection = 1;
+  const size_t score_ws = curdkv_workspace_bytes(&d, 0, 0);
+  if (score_ws == 0) return false;
+  const size_t P = (size_t)batch * heads;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o += round256(bytes ? bytes : 1); return at; };
+  L->score_ws = take(score_ws);                 // first: its status word is the cache's too
+  L->raw_new = take(P * (size_t)t_max * 4);
+  L->sums = take(P * 4);
+  L->idx = take(P * (size_t)budget * 4);
+  L->counts = take(P * 4);
+  L->total = o;
+  return true;
+}
+
+bool cache_ok(const curdkv_cache* c) {
+  return c != nullptr && c->K != nullptr && c->V != nullptr && c->raw != nullptr && c->pos != nullptr &&
+         c->count != nullptr && c->total != nullptr && c->capacity >= 1;
+}
+
+CacheView view_of(const curdkv_cache* c) {
+  return CacheView{static_cast<__nv_bfloat16*>(c->K), static_cast<__nv_bfloat16*>(c->V), c->raw, c->pos,
+                   c->count, c->total, c->capacity};
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t curdkv_cache_workspace_bytes(int32_t batch, int32_t kv_heads, int32_t t_max, int32_t capacity,
+                                    int32_t budget) {
+  CacheWorkspace L;
+  return layout(batch, kv_heads, t_max, capacity, budget, &L) ? L.total : 0;
+}
+
+curdkv_status curdkv_cache_append(const curdkv_cache* cache, const void* K_new, const void* V_new,
+                                  const float* G, int32_t g_per_head, const curdkv_desc* desc_new,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!cache_ok(cache) || desc_new == nullptr || workspace == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  CacheWorkspace L;
+  if (!layout(desc_new->batch, desc_new->kv_heads, desc_new->n_max, cache->capacity, 0, &L))
+    return CURDKV_ERR_INVALID_ARG;
+  if (workspace_bytes < L.total) return CURDKV_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  float* raw_new = reinterpret_cast<float*>(ws + L.raw_new);
+
+  curdkv_desc d = *desc_new;
+  d.raw_scores = 1;
+  d.score_mode = 0;
+  curdkv_status st = curdkv_score(K_new, V_new, G, g_per_head, &d, raw_new,
+                                  reinterpret_cast<float*>(ws + L.sums), ws + L.score_ws,
+                                  L.raw_new - L.score_ws, cuda_stream);
+  if (st != CURDKV_OK) return st;
+  const int64_t P = (int64_t)d.batch * d.kv_heads;
+  if (P == 0 || d.n_max == 0) return CURDKV_OK;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  AppendArgs a;
+  a.cache = view_of(cache);
+  a.K_new = KvView{static_cast<const __nv_bfloat16*>(K_new), d.k_stride_b, d.k_stride_h, d.k_stride_n};
+  a.V_new = KvView{static_cast<const __nv_bfloat16*>(V_new), d.v_stride_b, d.v_stride_h, d.v_stride_n};
+  a.raw_new = raw_new;
+  a.t_new = d.seqlens;
+  a.heads = d.kv_heads;
+  a.t = d.n_max;
+  a.d = d.d;
+  a.status = reinterpret_cast<uint32_t*>(ws + L.score_ws);
+  const int64_t chunks = (d.n_max + kAppendRowsPerCta - 1) / kAppendRowsPerCta;
+  if (P * chunks > 0x7fffffffLL) return CURDKV_ERR_UNSUPPORTED;
+  cache_append_kernel<<<(unsigned)(P * chunks), kAppendWarps * 32, 0, stream>>>(a);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  cache_advance_kernel<<<(unsigned)((d.batch + 255) / 256), 256, 0, stream>>>(a.cache, d.seqlens, d.n_max,
+                                                                             d.batch);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* out,
+                                    const curdkv_desc* desc, int32_t budget, int32_t num_sink,
+                                    int32_t window, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+  if (!cache_ok(in) || !cache_ok(out) || desc == nullptr || workspace == nullptr)
+    return CURDKV_ERR_INVALID_ARG;
+  if (budget < 0 || num_sink < 0 || window < 0) return CURDKV_ERR_INVALID_ARG;
+  if (in->K == out->K || in->V == out->V || in->raw == out->raw || in->pos == out->pos)
+    return CURDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  const int32_t most = budget < in->capacity ? budget : in->capacity;
+  if (out->capacity < most) return CURDKV_ERR_INVALID_ARG;
+  CacheWorkspace L;
+  if (!layout(desc->batch, desc->kv_heads, 0, in->capacity, budget, &L)) return CURDKV_ERR_INVALID_ARG;
+  if (workspace_bytes < L.total) return CURDKV_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  if (P == 0) return CURDKV_OK;
+
+  // the held rows of every (sequence, head) seen as one [batch][heads][capacity] problem set
+  curdkv_desc d = *desc;
+  d.q_heads = d.kv_heads;
+  d.n_max = in->capacity;
+  d.k_stride_n = d.v_stride_n = d.d;
+  d.k_stride_h = d.v_stride_h = (int64_t)in->capacity * d.d;
+  d.k_stride_b = d.v_stride_b = d.k_stride_h * d.kv_heads;
+  d.seqlens = in->count;
+  d.score_mode = 0;
+  d.use_projection = 1;
+  d.raw_scores = 0;
+  curdkv_status st = curdkv_select(in->raw, &d, budget, nullptr, num_sink, window, 0, 0.0, idx, counts,
+                                   nullptr, ws + L.score_ws, L.raw_new - L.score_ws, cuda_stream);
+  if (st != CURDKV_OK) return st;
+  if (budget > 0) {
+    st = curdkv_compact(in->K, in->V, &d, idx, budget, counts, nullptr, out->K, out->V, out->capacity,
+                        ws + L.score_ws, cuda_stream);
+    if (st != CURDKV_OK) return st;
+  }
+  cache_gather_meta_kernel<<<(unsigned)P, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      view_of(in), view_of(out), idx, budget, counts, d.kv_heads);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+}  // extern "C"

@@ -187,6 +187,7 @@ __global__ void __launch_bounds__(256) sketch_fma_kernel(const ScoreArgs a, cons
 // ---------------------------------------------------------------------------
 // Alg. 1 line 6: S = sum of the partial sums of the head's valid tiles in a
 // fixed order, scores /= S; scores at or beyond the sequence length become 0.
+// With `raw` the division is left out (S is still reported).
 // grid = batch*heads*ceil(n_max / 4096) (chunk fastest), block = 256.
 // ---------------------------------------------------------------------------
 constexpr int kNormChunk = 4096;
@@ -194,7 +195,8 @@ constexpr int kNormChunk = 4096;
 __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const float* tile_sums,
                                                         float* head_sums, const int32_t* seqlens,
                                                         int heads, int n_max, int tiles_per_head,
-                                                        int parts_per_tile, int chunks_per_head) {
+                                                        int parts_per_tile, int chunks_per_head,
+                                                        int raw) {
   __shared__ float red[8];
   const int p = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -205,7 +207,7 @@ __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const flo
   // a full chunk of valid scores is put on its way while the head sum is formed
   const bool vec = (reinterpret_cast<uintptr_t>(row) & 15u) == 0 && j0 + kNormChunk <= n;
   float4 v[4];
-  if (vec) {
+  if (vec && !raw) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) v[u] = reinterpret_cast<const float4*>(row + j0)[tid + 256 * u];
   }
@@ -222,7 +224,9 @@ __global__ void __launch_bounds__(256) normalise_kernel(float* scores, const flo
   for (int w = 0; w < 8; ++w) S += red[w];
   if (chunk == 0 && tid == 0) head_sums[p] = S;
   const bool live = S > 0.f;
-  if (vec) {
+  if (raw) {                                               // only the padding is rewritten
+    for (int j = max(j0, n) + tid; j < j1; j += 256) row[j] = 0.f;
+  } else if (vec) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       float4 o;

@@ -1,0 +1,116 @@
+"""Generation-phase cache on the GPU (through the C ABI) against the step-by-step oracle and
+against one application of Alg. 1 to the whole history.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import curdkv_decode_oracle as dec
+from oracle import curdkv_oracle as orc
+from paper_2509_15038_b200 import binding as cur
+from paper_2509_15038_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _history(B, H, N, d, seed):
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=B, n_max=N, kv_heads=H, q_heads=H,
+                     data_seed=seed)
+    K, V, _ = synth.make_kv(w, DEV)
+    return K, V
+
+
+def _run(K, V, G, schedule, k, s, w, capacity, t_new=None):
+    """Feeds the history in chunks; compresses whenever a sequence could overflow and at the end."""
+    B, H, N, d = K.shape
+    Gd = torch.as_tensor(G, device=DEV)
+    caches = [cur.DeviceCache(B, H, capacity, d, DEV), cur.DeviceCache(B, H, capacity, d, DEV)]
+    ws = cur.cache_workspace(B, H, max(schedule), capacity, k, DEV)
+    ref = dec.CacheOracle(B, H, d)
+    Ku, Vu = synth.to_u16(K), synth.to_u16(V)
+    live, at, held = 0, 0, 0
+    for step, t in enumerate(schedule):
+        if held + t > capacity:
+            cur.curdkv_cache_compress(caches[live], caches[1 - live], k, ws, num_sink=s, window=w)
+            ref.compress(k, s, w)
+            live, held = 1 - live, min(held, k)
+        tn = None if t_new is None else torch.as_tensor(t_new[step], dtype=torch.int32, device=DEV)
+        cur.curdkv_cache_append(caches[live], K[:, :, at:at + t], V[:, :, at:at + t], Gd, ws, t_new=tn)
+        ref.append(Ku[:, :, at:at + t], Vu[:, :, at:at + t], G, None if t_new is None else t_new[step])
+        at += t
+        held += t
+    cur.curdkv_cache_compress(caches[live], caches[1 - live], k, ws, num_sink=s, window=w)
+    ref.compress(k, s, w)
+    live = 1 - live
+    assert cur.curdkv_device_status(ws) == 0
+    return caches[live], ref
+
+
+def _compare(cache, ref, k, s, w):
+    B, H = ref.B, ref.H
+    cnt = cache.count.cpu().numpy()
+    np.testing.assert_array_equal(cache.total.cpu().numpy(), ref.total)
+    pos, raw = cache.pos.cpu().numpy(), cache.raw.cpu().numpy()
+    Ko, Vo = synth.to_u16(cache.K), synth.to_u16(cache.V)
+    for b in range(B):
+        for h in range(H):
+            c = int(cnt[b])
+            assert c == len(ref.pos[b][h])
+            got = pos[b, h, :c]
+            assert np.all(np.diff(got) > 0)
+            want = ref.pos[b][h]
+            # fp32 vs fp64 scores can only disagree on a near-tie at the cut (gap < 1e-6 relative)
+            assert len(set(got.tolist()) ^ set(want.tolist())) <= 2, "more than one near-tie apart"
+            both = np.intersect1d(got, want)
+            gi = np.searchsorted(got, both)
+            ri = np.searchsorted(want, both)
+            np.testing.assert_array_equal(Ko[b, h][gi], ref.K[b][h][ri])
+            np.testing.assert_array_equal(Vo[b, h][gi], ref.V[b][h][ri])
+            np.testing.assert_allclose(raw[b, h][gi], ref.raw[b][h][ri], rtol=1e-3)
+
+
+@pytest.mark.parametrize("k,s,w", [(64, 4, 0), (64, 0, 16), (100, 4, 8)])
+def test_decode_chunks_match_oracle_and_one_shot(k, s, w):
+    B, H, N, d, r = 3, 2, 700, 128, 32
+    K, V = _history(B, H, N, d, seed=21)
+    G = synth.make_G(d, r, seed=0)
+    schedule = [256, 1, 1, 130, 7, 200, 64, 41]
+    assert sum(schedule) == N
+    cache, ref = _run(K, V, G, schedule, k, s, w, capacity=k + 256)
+    _compare(cache, ref, k, s, w)
+    # one application of Alg. 1 to the whole history keeps the same positions
+    sc, _ = orc.score(synth.to_u16(K), synth.to_u16(V), G)
+    idx, cnt = orc.select_fixed(sc, k, s, w)
+    pos = cache.pos.cpu().numpy()
+    for b in range(B):
+        for h in range(H):
+            forced = pu.forced_tokens(N, int(cnt[b, h]), s, w)
+            pu.assert_selection_within_band(pos[b, h, :cnt[b, h]], idx[b, h, :cnt[b, h]], sc[b, h], N,
+                                            forced, f"one-shot b={b} h={h}")
+
+
+def test_decode_token_by_token_and_ragged_appends():
+    B, H, N, d, r = 2, 2, 96, 128, 20
+    K, V = _history(B, H, N, d, seed=22)
+    G = synth.make_G(d, r, seed=1)
+    cache, ref = _run(K, V, G, [1] * N, 24, 4, 6, capacity=40)
+    _compare(cache, ref, 24, 4, 6)
+    # sequences that bring different numbers of rows per step (the rest of the block is padding)
+    schedule = [32, 32, 32]
+    t_new = [np.array([32, 5], np.int32), np.array([0, 32], np.int32), np.array([17, 1], np.int32)]
+    cache, ref = _run(K, V, G, schedule, 24, 2, 4, capacity=64, t_new=t_new)
+    _compare(cache, ref, 24, 2, 4)
+
+
+def test_decode_overflow_is_flagged_not_written():
+    B, H, d = 1, 1, 128
+    K, V = _history(B, H, 64, d, seed=23)
+    G = torch.as_tensor(synth.make_G(d, 32, seed=0), device=DEV)
+    cache = cur.DeviceCache(B, H, 40, d, DEV)
+    ws = cur.cache_workspace(B, H, 64, 40, 16, DEV)
+    cur.curdkv_cache_append(cache, K, V, G, ws)
+    flags = cur.curdkv_device_status(ws)
+    assert flags & 0x4
+    assert int(cache.count[0]) == 40 and int(cache.total[0]) == 64
+    np.testing.assert_array_equal(synth.to_u16(cache.K)[0, 0], synth.to_u16(K)[0, 0, :40])
