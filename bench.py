@@ -314,6 +314,83 @@ def run_e2e(cur, w, K, V, seqlens, value_tokens, world, dev, steps):
             "host_link_gb_per_s": (h2d + d2h) / dt / 1e9}
 
 
+# --------------------------------------------------------------------------- generation phase
+
+DECODE = dict(layers=32, batch=16, kv_heads=8, d=128, r=32, budget=2048, num_sink=4, window=64, chunk=256)
+
+
+def run_decode(args):
+    """Generation-phase workload (Sec. 3.2): every step appends `chunk` new rows per head to a cache
+    that holds `budget` rows and compresses it back to `budget` (Alg. 1 lines 2-10 on the cache)."""
+    from paper_2509_15038_b200 import binding as cur
+
+    c = DECODE
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    LB, H, d, t, k = c["layers"] * c["batch"], c["kv_heads"], c["d"], c["chunk"], c["budget"]
+    cap = k + t
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=c["layers"], batch=c["batch"], n_max=t, data_seed=6)
+    K_new, V_new, _ = synth.make_kv(w, dev)
+    w0 = synth.shrink(w, n_max=cap, data_seed=7)
+    K0, V0, _ = synth.make_kv(w0, dev)
+    G = torch.as_tensor(synth.make_G(d, c["r"], seed=0), device=dev)
+    caches = [cur.DeviceCache(LB, H, cap, d, dev), cur.DeviceCache(LB, H, cap, d, dev)]
+    ws = cur.cache_workspace(LB, H, cap, cap, k, dev)
+    cur.curdkv_cache_append(caches[0], K0, V0, G, ws)              # fill to capacity, then to budget
+    cur.curdkv_cache_compress(caches[0], caches[1], k, ws, num_sink=c["num_sink"], window=c["window"])
+    live = 1
+
+    def step():
+        nonlocal live
+        cur.curdkv_cache_append(caches[live], K_new, V_new, G, ws)
+        cur.curdkv_cache_compress(caches[live], caches[1 - live], k, ws, num_sink=c["num_sink"],
+                                  window=c["window"])
+        live = 1 - live
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if cur.curdkv_device_status(ws):
+        raise RuntimeError("device status flags set after warm-up")
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = cur.launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    launches = cur.launch_count() - launches0
+    clocks = sampler.stop()
+    assert int(caches[live].count.min()) == k and int(caches[live].count.max()) == k
+    ms = t0.elapsed_time(t1) / args.steps
+    P = LB * H
+    rows = P * (k + t)                       # rows the compression looks at per step
+    # new rows read and stored, their scores; held scores read; survivors read and written
+    counted = P * (t * 512 * 2 + (k + t) * 4 + k * 512 * 2)
+    peak, peak_kind = measured_peak()
+    gbs = counted / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": rows / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "decode: %(layers)d layers x batch %(batch)d x %(kv_heads)d KV heads, cache "
+                               "budget %(budget)d (sinks %(num_sink)d, window %(window)d), %(chunk)d new rows "
+                               "per head and step, r=%(r)d" % c,
+                   "head_tokens_per_step": rows,
+                   "l2": "caches (%.1f GB) exceed the 126 MB L2" % (2 * 2 * P * cap * d * 2 / 1e9)},
+        "gb_per_s": gbs, "counted_bytes_per_step": counted,
+        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "whole step (append + select + gather)", "achieved": gbs,
+                     "peak": peak, "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s",
+                     "frac": gbs / peak, "traffic": None},
+    }), flush=True)
+
+
 # --------------------------------------------------------------------------- oracle arm
 
 def oracle_sample(w, elements):
@@ -401,12 +478,16 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
-    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3,
                     help="steps of the host-buffer end-to-end leg (0 disables it)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "decode":
+        if args.impl == "reference":
+            raise SystemExit("the reference arm times the prefill workloads only")
+        run_decode(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)
