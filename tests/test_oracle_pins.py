@@ -491,3 +491,76 @@ def test_generation_phase_raw_scores_are_row_local():
     np.testing.assert_array_equal(full[:, :, 10:25], part)
     sc, S = orc.score(Ku, Vu, G)
     np.testing.assert_allclose(full / S[..., None], sc, rtol=1e-14)
+
+
+# --------------------------------------------------------------------------- whitened sketch
+def test_whitened_scores_are_exact_leverage_for_identity_G():
+    """Eq. (row leverage score): with G = I and no ridge, ||a_j L^-T||^2 = ||U(j,:)||^2 (numpy SVD),
+    the scores sum to rank(A) = d, and they ignore any invertible mixing of the columns."""
+    from oracle import curdkv_whiten_oracle as wh
+
+    rng = np.random.default_rng(0)
+    n, d = 300, 24
+    A = rng.standard_normal((n, d)) * np.exp(rng.standard_normal((1, d)) * 2.0)   # badly scaled columns
+    lev = wh.whitened_row_scores(A, np.eye(d), 0.0)
+    U = np.linalg.svd(A, full_matrices=False)[0]
+    np.testing.assert_allclose(lev, np.sum(U * U, axis=1), rtol=1e-9)
+    np.testing.assert_allclose(lev.sum(), d, rtol=1e-10)
+    T = rng.standard_normal((d, d)) + 3 * np.eye(d)
+    np.testing.assert_allclose(wh.whitened_row_scores(A @ T, np.eye(d), 0.0), lev, rtol=1e-7)
+    # the plain sketch of Alg. 1 is NOT invariant to such mixing: it follows the row norms
+    plain = np.sum(A * A, axis=1)
+    assert np.corrcoef(plain / plain.sum(), lev / lev.sum())[0, 1] < 0.9
+
+
+def test_whitened_sketch_is_unbiased_and_converges():
+    """Gaussian G ~ N(0, 1/r): E ||a_j W||^2 = leverage; the error shrinks like r^-1/2."""
+    from oracle import curdkv_whiten_oracle as wh
+
+    rng = np.random.default_rng(1)
+    n, d = 200, 16
+    A = rng.standard_normal((n, d)) @ np.diag(np.linspace(1, 30, d))
+    exact = wh.whitened_row_scores(A, np.eye(d), 0.0)
+    r = 8
+    draws = np.stack([wh.whitened_row_scores(A, rng.standard_normal((d, r)) / np.sqrt(r), 0.0)
+                      for _ in range(1500)])
+    sigma = exact * np.sqrt(2.0 / r) / np.sqrt(draws.shape[0])       # chi-square: var = 2 l^2 / r
+    assert np.all(np.abs(draws.mean(0) - exact) < 4.5 * sigma)
+    errs = []
+    for r in (8, 128, 2048):
+        G = rng.standard_normal((d, r)) / np.sqrt(r)
+        errs.append(np.median(np.abs(wh.whitened_row_scores(A, G, 0.0) - exact) / exact))
+    assert errs[0] > 2.5 * errs[1] > 6 * errs[2]
+
+
+def test_whitened_ridge_matches_direct_inverse_and_short_sequences():
+    from oracle import curdkv_whiten_oracle as wh
+
+    rng = np.random.default_rng(2)
+    n, d = 40, 16
+    A = rng.standard_normal((n, d))
+    ridge = 1e-2
+    lam = ridge * np.trace(A.T @ A) / d
+    want = np.einsum("ij,jk,ik->i", A, np.linalg.inv(A.T @ A + lam * np.eye(d)), A)
+    np.testing.assert_allclose(wh.whitened_row_scores(A, np.eye(d), ridge), want, rtol=1e-10)
+    assert np.all(want < wh.whitened_row_scores(A, np.eye(d), 0.0))
+    # fewer rows than columns: the Gram matrix is singular, the ridge keeps the factorisation defined
+    short = wh.whitened_row_scores(A[:5], np.eye(d), ridge)
+    assert np.all(np.isfinite(short)) and np.all(short > 0) and np.all(short < 1)
+
+
+def test_whitened_pipeline_normalises_and_respects_lengths():
+    from oracle import curdkv_whiten_oracle as wh
+
+    rng = np.random.default_rng(3)
+    B, H, n, d, r = 2, 2, 64, 16, 8
+    to_bits = lambda a: (np.ascontiguousarray(a, dtype=np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    K, V = to_bits(rng.standard_normal((B, H, n, d))), to_bits(rng.standard_normal((B, H, n, d)))
+    G = (rng.standard_normal((d, r)) / np.sqrt(r)).astype(np.float32)
+    lens = np.array([64, 37], np.int32)
+    sc, S, lK, lV = wh.score_whitened(K, V, G, 1e-4, seqlens=lens)
+    np.testing.assert_allclose(sc.sum(-1), 1.0, rtol=1e-12)
+    assert np.all(sc[1, :, 37:] == 0)
+    np.testing.assert_allclose(sc * S[..., None], lK * lV, rtol=1e-12)
+    sc2, _, _, _ = wh.score_whitened(K[1:, :, :37], V[1:, :, :37], G, 1e-4)
+    np.testing.assert_allclose(sc2[0], sc[1, :, :37], rtol=1e-12)
