@@ -52,6 +52,7 @@ typedef enum curdkv_status {
 #define CURDKV_DEV_TIMEOUT 0x1u   /* a pipeline wait gave up; results of that launch are invalid */
 #define CURDKV_DEV_BAD_INDEX 0x2u /* an index outside [0, n) was skipped by the gather           */
 #define CURDKV_DEV_CACHE_FULL 0x4u /* curdkv_cache_append dropped rows that exceeded the capacity */
+#define CURDKV_DEV_NOT_SPD 0x8u   /* whiten = 1: a Gram matrix was not positive definite (raise ridge) */
 
 /* Shape of one call: K and V are bf16 tensors addressed as
  *   K[b][h][j][c] = K_base[b*k_stride_b + h*k_stride_h + j*k_stride_n + c]
@@ -76,6 +77,15 @@ typedef struct curdkv_desc {
   int32_t raw_scores;     /* 0: normalise per head (Alg. 1 line 6); 1: leave l^KV of line 5 as
                              it is (head_sums is still written) -- what the generation-phase
                              cache stores, since a row's l^KV does not depend on other rows  */
+  int32_t whiten;         /* 0: Alg. 1 as printed (||a_j G||^2 follows the row norms).
+                             1: approximate the leverage scores ||U(j,:)||^2 of Eq. (row
+                             leverage score): per (b, h) and tensor A in {K, V} over the valid
+                             rows, M = A^T A + lambda I with lambda = ridge * trace(A^T A)/d,
+                             M = L L^T (Cholesky), W = L^{-T} G, l_j = ||a_j W||^2; the rest of
+                             Alg. 1 is unchanged.  Needs use_projection = 1, one shared G,
+                             d = 128, r <= 64, n_max >= 128; reads K and V twice.          */
+  double ridge;           /* whiten = 1 only: relative ridge >= 0 (1e-4 is a safe default;
+                             0 needs n_b >= d and full column rank)                        */
 } curdkv_desc;
 
 /* Bytes of device workspace the calls below need for this shape (256-byte

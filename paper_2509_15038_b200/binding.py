@@ -43,7 +43,7 @@ class Desc(ctypes.Structure):
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_n", ctypes.c_int64),
         ("seqlens", ctypes.c_void_p),
         ("score_mode", ctypes.c_int32), ("use_projection", ctypes.c_int32),
-        ("raw_scores", ctypes.c_int32),
+        ("raw_scores", ctypes.c_int32), ("whiten", ctypes.c_int32), ("ridge", ctypes.c_double),
     ]
 
 
@@ -133,7 +133,8 @@ def _check(code: int, what: str):
 
 def make_desc(K: torch.Tensor, V: torch.Tensor, r: int, *, q_heads: Optional[int] = None,
               seqlens: Optional[torch.Tensor] = None, score_mode: int = 0,
-              use_projection: int = 1, raw_scores: int = 0) -> Desc:
+              use_projection: int = 1, raw_scores: int = 0, whiten: int = 0,
+              ridge: float = 0.0) -> Desc:
     """Descriptor of bf16 K, V ``[B, Hkv, n_max, d]`` (any strides with d contiguous)."""
     if K.dtype != torch.bfloat16 or V.dtype != torch.bfloat16:
         raise TypeError("K and V must be bf16")
@@ -146,7 +147,7 @@ def make_desc(K: torch.Tensor, V: torch.Tensor, r: int, *, q_heads: Optional[int
     return Desc(B, H, q_heads or H, n, d, int(r),
                 K.stride(0), K.stride(1), K.stride(2), V.stride(0), V.stride(1), V.stride(2),
                 seqlens.data_ptr() if seqlens is not None else None,
-                int(score_mode), int(use_projection), int(raw_scores))
+                int(score_mode), int(use_projection), int(raw_scores), int(whiten), float(ridge))
 
 
 def workspace_bytes(desc: Desc, max_budget: int = 0, adaptive: bool = False) -> int:

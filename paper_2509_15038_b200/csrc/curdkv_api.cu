@@ -9,6 +9,8 @@
 #include "score_simt.cuh"
 #include "score_umma.cuh"
 #include "select.cuh"
+#include "whiten_factor.cuh"
+#include "whiten_umma.cuh"
 
 namespace {
 
@@ -30,6 +32,8 @@ curdkv_status check_desc(const curdkv_desc* d) {
   if (d->score_mode < 0 || d->score_mode > 2) return CURDKV_ERR_INVALID_ARG;
   if (d->use_projection != 0 && d->use_projection != 1) return CURDKV_ERR_INVALID_ARG;
   if (d->raw_scores != 0 && d->raw_scores != 1) return CURDKV_ERR_INVALID_ARG;
+  if (d->whiten != 0 && d->whiten != 1) return CURDKV_ERR_INVALID_ARG;
+  if (d->whiten && !(d->ridge >= 0.0)) return CURDKV_ERR_INVALID_ARG;
   if ((int64_t)d->batch * d->kv_heads > (int64_t)1 << 24) return CURDKV_ERR_UNSUPPORTED;
   return CURDKV_OK;
 }
@@ -142,6 +146,30 @@ void* static_scratch_ptr() {
   return g_static_ptr[dev];
 }
 
+// Whitened scoring cuts every head into this many runs of tiles (the work items of the two
+// streaming kernels): enough items to balance the SMs, never more than the head has tiles.
+int whiten_segments(const curdkv_desc* d) {
+  const int64_t P = (int64_t)d->batch * d->kv_heads;
+  if (P <= 0) return 1;
+  int64_t s = (8 * 148 + P - 1) / P;
+  const int tiles = tiles_per_head(d);
+  if (s > tiles) s = tiles;
+  return s < 1 ? 1 : (int)s;
+}
+
+struct WhitenLayout {      // byte offsets from the workspace base, after the tile sums
+  size_t partials, W, total;
+};
+
+WhitenLayout whiten_layout(const curdkv_desc* d, size_t after_tile_sums) {
+  WhitenLayout L;
+  const size_t P = (size_t)d->batch * d->kv_heads;
+  L.partials = after_tile_sums;
+  L.W = L.partials + round256(P * whiten_segments(d) * 2 * 128 * 128 * sizeof(float));
+  L.total = L.W + round256(P * 2 * 128 * (size_t)(d->r > 0 ? d->r : 1) * sizeof(float));
+  return L;
+}
+
 KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
   return KvView{static_cast<const __nv_bfloat16*>(base), sb, sh, sn};
 }
@@ -159,7 +187,8 @@ size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32
   (void)adaptive;
   if (check_desc(desc) != CURDKV_OK) return 0;
   const size_t tiles = (size_t)desc->batch * desc->kv_heads * tiles_per_head(desc);
-  return kStatusBytes + round256(tiles * umma::kPartsPerTile * sizeof(float));
+  const size_t plain = kStatusBytes + round256(tiles * umma::kPartsPerTile * sizeof(float));
+  return desc->whiten ? whiten_layout(desc, plain).total : plain;
 }
 
 curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
@@ -174,6 +203,8 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
     if (G == nullptr || desc->r < 1) return CURDKV_ERR_INVALID_ARG;
     if (desc->d != 128 || desc->r > 64) return CURDKV_ERR_UNSUPPORTED;
   }
+  if (desc->whiten && (!desc->use_projection || g_per_head || desc->n_max < kTileRows))
+    return CURDKV_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
   if (workspace_bytes < curdkv_workspace_bytes(desc, 0, 0)) return CURDKV_ERR_WORKSPACE;
 
@@ -202,7 +233,71 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
   const unsigned grid = (unsigned)(P * tiles);
   int parts = 1;                                  // partial sums per 128-row tile
   bool launched = false;
-  if (desc->use_projection && !g_per_head && desc->n_max >= kTileRows) {
+  if (desc->whiten) {
+    // two passes over K and V: Gram matrices, their factors, then the sketch with W = L^-T G
+    CUtensorMap mk, mv;
+    if (!make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) ||
+        !make_tile_map(&mv, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n))
+      return CURDKV_ERR_CUDA;
+    const size_t plain = kStatusBytes + round256((size_t)P * tiles * umma::kPartsPerTile * sizeof(float));
+    const WhitenLayout L = whiten_layout(desc, plain);
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    umma::ItemArgs u;
+    u.seqlens = desc->seqlens;
+    u.batch = desc->batch;
+    u.heads = desc->kv_heads;
+    u.n_max = desc->n_max;
+    u.segments = whiten_segments(desc);
+    u.status = static_cast<uint32_t*>(workspace);
+    u.partials = reinterpret_cast<float*>(ws + L.partials);
+    u.W = reinterpret_cast<const float*>(ws + L.W);
+    u.r = desc->r;
+    u.tiles_per_head = tiles;
+    u.score_mode = desc->score_mode;
+    u.scores = scores;
+    u.tile_sums = a.tile_sums;
+    const int sms = sm_count();
+    if (sms <= 0) return CURDKV_ERR_CUDA;
+    const int64_t items = P * u.segments;
+    const unsigned grid_items = (unsigned)(items < sms ? items : sms);
+    if (cudaFuncSetAttribute(umma::gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             umma::kGramDynamic) != cudaSuccess)
+      return CURDKV_ERR_CUDA;
+    umma::gram_umma_kernel<<<grid_items, umma::kThreads, umma::kGramDynamic, stream>>>(mk, mv, u);
+    if (!launch_ok()) return CURDKV_ERR_CUDA;
+    FactorArgs f;
+    f.partials = u.partials;
+    f.G = G;
+    f.W = reinterpret_cast<float*>(ws + L.W);
+    f.segments = u.segments;
+    f.r = desc->r;
+    f.ridge = desc->ridge;
+    f.status = u.status;
+    const size_t fsm = ((size_t)kFactorD * (kFactorD + 1) + (size_t)kFactorD * desc->r) * sizeof(double);
+    if (cudaFuncSetAttribute(whiten_factor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)fsm) != cudaSuccess)
+      return CURDKV_ERR_CUDA;
+    whiten_factor_kernel<<<(unsigned)(2 * P), kFactorThreads, fsm, stream>>>(f);
+    if (!launch_ok()) return CURDKV_ERR_CUDA;
+    if (g_profile_start != nullptr) cudaEventRecord(g_profile_start, stream);
+    if (desc->r <= 32) {
+      using S = umma::ItemSmem<32>;
+      if (cudaFuncSetAttribute(umma::sketch_items_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               S::kDynamic) != cudaSuccess)
+        return CURDKV_ERR_CUDA;
+      umma::sketch_items_kernel<32><<<grid_items, umma::kThreads, S::kDynamic, stream>>>(mk, mv, u);
+    } else {
+      using S = umma::ItemSmem<64>;
+      if (cudaFuncSetAttribute(umma::sketch_items_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               S::kDynamic) != cudaSuccess)
+        return CURDKV_ERR_CUDA;
+      umma::sketch_items_kernel<64><<<grid_items, umma::kThreads, S::kDynamic, stream>>>(mk, mv, u);
+    }
+    if (g_profile_stop != nullptr) cudaEventRecord(g_profile_stop, stream);
+    if (!launch_ok()) return CURDKV_ERR_CUDA;
+    parts = umma::kPartsPerTile;
+    launched = true;
+  } else if (desc->use_projection && !g_per_head && desc->n_max >= kTileRows) {
     // tensor-core path: one G for all heads, TMA tiles of 128 rows.  A ragged batch goes in
     // slices of at most kMaxRaggedBatch sequences (the kernel keeps their tile prefix sums
     // in shared memory).

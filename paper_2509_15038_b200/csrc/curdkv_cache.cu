@@ -75,6 +75,7 @@ curdkv_status curdkv_cache_append(const curdkv_cache* cache, const void* K_new, 
   curdkv_desc d = *desc_new;
   d.raw_scores = 1;
   d.score_mode = 0;
+  d.whiten = 0;                       // a row's score must not depend on the rows it arrives with
   curdkv_status st = curdkv_score(K_new, V_new, G, g_per_head, &d, raw_new,
                                   reinterpret_cast<float*>(ws + L.sums), ws + L.score_ws,
                                   L.raw_new - L.score_ws, cuda_stream);
