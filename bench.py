@@ -149,7 +149,8 @@ def run_cuda(args):
     K, V, seqlens = synth.make_kv(w, dev)
     G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
     sl = None if seqlens is None else torch.as_tensor(seqlens, device=dev)
-    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads, seqlens=sl)
+    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads, seqlens=sl, whiten=int(args.whiten),
+                         ridge=1e-4 if args.whiten else 0.0)
     ws = cur.alloc_workspace(desc, w.budget, w.adaptive)
     P = w.folded_batch * w.kv_heads
     scores = torch.empty((w.folded_batch, w.kv_heads, w.n_max), dtype=torch.float32, device=dev)
@@ -222,11 +223,14 @@ def run_cuda(args):
     stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in ev]).mean(0)
 
     tokens, read_bytes, write_bytes = workload_bytes(w, seqlens)
+    pass_bytes = read_bytes                  # K + V once: what one streaming kernel reads
+    if args.whiten:
+        read_bytes *= 2                      # Gram pass + sketch pass
     value = job_throughput(tokens, world, ms_step * 1e-3)
     gbs = job_throughput(read_bytes + write_bytes, world, ms_step * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
     sketch_ms = float(np.mean([a.elapsed_time(b) for a, b in sk]))
-    sketch_gbs = read_bytes / (sketch_ms * 1e-3) / 1e9
+    sketch_gbs = pass_bytes / (sketch_ms * 1e-3) / 1e9
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -237,6 +241,7 @@ def run_cuda(args):
                         f"(GQA {w.q_heads}:{w.kv_heads}), n={w.n_max}, d={w.d}, r={w.r}, "
                         f"budget {w.budget} incl. window {w.window}, sinks {w.num_sink}, "
                         + ("AdaCurDKV alpha=%.2f" % w.alpha if w.adaptive else "fixed per-head budget")
+                        + (", whitened sketch (leverage scores, ridge 1e-4)" if args.whiten else "")
                         + (f", ragged lengths {w.ragged}" if w.ragged else ""),
             "head_tokens_per_step": tokens, "seq_tokens_per_step": tokens // (w.layers * w.kv_heads),
             "l2": "inputs (%.1f GB) exceed the 126 MB L2, no flush between steps" % (read_bytes / 1e9),
@@ -253,8 +258,9 @@ def run_cuda(args):
         "roofline": {
             "bound": "hbm", "kernel": "sketch_umma_kernel (inside curdkv_score)",
             "achieved": sketch_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
-            "unit": "GB/s", "frac": sketch_gbs / peak, "traffic": TRAFFIC_BYTES.get(w.name),
-            "algorithmic_bytes_per_launch": read_bytes, "ms_per_launch": sketch_ms,
+            "unit": "GB/s", "frac": sketch_gbs / peak,
+            "traffic": None if args.whiten else TRAFFIC_BYTES.get(w.name),
+            "algorithmic_bytes_per_launch": pass_bytes, "ms_per_launch": sketch_ms,
             "timer": "CUDA events recorded by the library around the kernel, mean over the timed steps",
         },
     }
@@ -480,6 +486,8 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--whiten", action="store_true",
+                    help="score with the whitened sketch (approximate leverage scores; reads K, V twice)")
     ap.add_argument("--e2e-steps", type=int, default=3,
                     help="steps of the host-buffer end-to-end leg (0 disables it)")
     args = ap.parse_args()

@@ -273,7 +273,7 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
     f.r = desc->r;
     f.ridge = desc->ridge;
     f.status = u.status;
-    const size_t fsm = ((size_t)kFactorD * (kFactorD + 1) + (size_t)kFactorD * desc->r) * sizeof(double);
+    const size_t fsm = kFactorSmemBytes;
     if (cudaFuncSetAttribute(whiten_factor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)fsm) != cudaSuccess)
       return CURDKV_ERR_CUDA;
