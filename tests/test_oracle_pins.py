@@ -564,3 +564,60 @@ def test_whitened_pipeline_normalises_and_respects_lengths():
     np.testing.assert_allclose(sc * S[..., None], lK * lV, rtol=1e-12)
     sc2, _, _, _ = wh.score_whitened(K[1:, :, :37], V[1:, :, :37], G, 1e-4)
     np.testing.assert_allclose(sc2[0], sc[1, :, :37], rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- eviction loss
+def test_attention_oracle_closed_forms():
+    from oracle import curdkv_eviction_oracle as ev
+
+    rng = np.random.default_rng(0)
+    m, n, d = 7, 50, 16
+    Q, K, V = rng.standard_normal((m, d)), rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    # all keys equal -> uniform weights -> every output row is the mean value row
+    O = ev.attention_out(Q, np.tile(K[:1], (n, 1)), V)
+    np.testing.assert_allclose(O, np.tile(V.mean(0), (m, 1)), rtol=1e-12)
+    # softmax rows sum to one: constant values come back unchanged
+    np.testing.assert_allclose(ev.attention_out(Q, K, np.ones((n, d))), 1.0, rtol=1e-12)
+    # one key aligned with a query and scaled up takes all the weight of that query
+    K2 = K.copy()
+    K2[13] = 40.0 * Q[3] / np.linalg.norm(Q[3])
+    np.testing.assert_allclose(ev.attention_out(Q, K2, V)[3], V[13], atol=1e-9)
+    # shifting every key by one vector shifts each row's logits by a constant: no change
+    np.testing.assert_allclose(ev.attention_out(Q, K + rng.standard_normal((1, d)), V),
+                               ev.attention_out(Q, K, V), rtol=1e-9)
+    # explicit two-key case
+    q, k0, k1 = np.array([[1.0, 0.0]]), np.array([2.0, 0.0]), np.array([0.0, 5.0])
+    w0 = np.exp(2.0) / (np.exp(2.0) + 1.0)
+    got = ev.attention_out(q, np.stack([k0, k1]), np.array([[1.0, 0.0], [0.0, 1.0]]))
+    np.testing.assert_allclose(got, [[w0, 1 - w0]], rtol=1e-13)
+    # scale multiplies the logits
+    np.testing.assert_allclose(ev.attention_out(Q, K, V, scale=0.25), ev.attention_out(0.25 * Q, K, V),
+                               rtol=1e-12)
+
+
+def test_eviction_loss_properties_and_lemma1():
+    """Lemma 1: ||softmax(QK^T)V - softmax(QK'^T)V'||_F <= sqrt(n)||V - V'||_F + 2 sqrt(n)||V'||_F with
+    zeroed rows; keeping everything loses nothing; zeroed rows are keys with logit 0 and value 0."""
+    from oracle import curdkv_eviction_oracle as ev
+
+    rng = np.random.default_rng(1)
+    n, d = 60, 16
+    Q, K, V = rng.standard_normal((n, d)), rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    assert ev.eviction_loss(Q, K, V, np.arange(n))[0] < 1e-12
+    assert ev.eviction_loss(Q, K, V, np.arange(n), zeroed=True)[0] < 1e-12
+    for k in (1, 5, 30, 59):
+        kept = np.sort(rng.choice(n, size=k, replace=False))
+        loss0, ref = ev.eviction_loss(Q, K, V, kept, zeroed=True)
+        assert loss0 <= ev.lemma1_bound(V, kept)
+        # the zeroed form is attention over the full-size K', V'
+        Kp, Vp = np.zeros_like(K), np.zeros_like(V)
+        Kp[kept], Vp[kept] = K[kept], V[kept]
+        direct = np.linalg.norm(ev.attention_out(Q, K, V) - ev.attention_out(Q, Kp, Vp))
+        np.testing.assert_allclose(loss0, direct, rtol=1e-10)
+        np.testing.assert_allclose(ref, np.linalg.norm(ev.attention_out(Q, K, V)), rtol=1e-13)
+    # evicting rows whose value is zero and whose key repels every query costs (almost) nothing
+    K3, V3 = K.copy(), V.copy()
+    K3[40:] = -50.0 * np.sign(Q.sum(0, keepdims=True))
+    Qpos = np.abs(Q) * np.sign(Q.sum(0, keepdims=True))
+    V3[40:] = 0.0
+    assert ev.eviction_loss(Qpos, K3, V3, np.arange(40))[0] < 1e-9
