@@ -241,6 +241,40 @@ curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* 
                                     int32_t window, void* workspace, size_t workspace_bytes,
                                     void* cuda_stream);
 
+/* ---- Eviction loss (Lemma 1; the reconstruction-loss figure of the introduction):
+ * how far the attention output moves when the cache is replaced by a selection,
+ *   loss[b][h] = || softmax(scale Q K^T) V - softmax(scale Q K'^T) V' ||_F .
+ * curdkv_attention_out computes O = softmax(scale * Q K^T) V for one cache (every
+ * query row sees every valid key row: the question-after-context setting); call it
+ * on the full cache and on the compacted one, then curdkv_eviction_loss.
+ *   Q            bf16 [batch][kv_heads][q_rows][128] with element strides q_stride_*
+ *                (the queries of a GQA group are stacked along q_rows)
+ *   K, V, desc   the cache, as in curdkv_score (d = 128), unless head_offsets != NULL:
+ *                then K and V are packed [packed_rows][128] arrays as curdkv_compact
+ *                writes them for AdaCurDKV, head p starting at row head_offsets[p]
+ *   head_rows    device int32 [batch*kv_heads] valid key rows per head, or NULL to use
+ *                desc->seqlens / n_max (required with head_offsets)
+ *   extra_zero_keys  NULL, or device int32 [batch*kv_heads]: that many further keys
+ *                with logit 0 and value 0 take part in each softmax -- Lemma 1's K', V'
+ *                keep the evicted rows as zero rows; NULL drops them, which is what a
+ *                compressed cache computes
+ *   scale        multiplies the logits (the paper writes softmax(QK^T): scale = 1)
+ *   O            fp32 [batch][kv_heads][q_rows][128]; a head with no key rows gets 0
+ * Exact two-pass softmax; the weights enter the second product as bf16 pairs
+ * (hi + lo), so O agrees with an fp64 evaluation to about 1e-5 relative. */
+size_t curdkv_attention_workspace_bytes(const curdkv_desc* desc);
+curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stride_b, int64_t q_stride_h,
+                                   int64_t q_stride_n, const void* K, const void* V,
+                                   const curdkv_desc* desc, const int32_t* head_rows,
+                                   const int32_t* head_offsets, int64_t packed_rows,
+                                   const int32_t* extra_zero_keys, float scale, float* O, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream);
+/* loss[p] = ||O_full[p] - O_compressed[p]||_F and (if not NULL) ref_norm[p] = ||O_full[p]||_F
+ * over elems_per_problem floats per problem; fixed summation order. */
+curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compressed, int32_t problems,
+                                   int64_t elems_per_problem, float* loss, float* ref_norm,
+                                   void* cuda_stream);
+
 /* GQA (Sec. 3.2): query head q uses KV head q / (q_heads / kv_heads).  Writes
  * kv_head_of_q int32 [q_heads] (device) so that attention consumers can index
  * the shared selection without replicating the compacted cache. */

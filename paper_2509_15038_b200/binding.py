@@ -25,7 +25,8 @@ EXPORTS = (
     "curdkv_gqa_map", "curdkv_device_status", "curdkv_launch_count", "curdkv_status_string",
     "curdkv_score_static", "curdkv_host_arena_bytes", "curdkv_compress_host",
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
-    "curdkv_cache_compress",
+    "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
+    "curdkv_eviction_loss",
 )
 
 
@@ -97,6 +98,13 @@ def load():
     lib.curdkv_cache_append.argtypes = [cp, vp, vp, vp, i32, dp, vp, ctypes.c_size_t, vp]
     lib.curdkv_cache_compress.restype = ctypes.c_int
     lib.curdkv_cache_compress.argtypes = [cp, cp, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
+    lib.curdkv_attention_workspace_bytes.restype = ctypes.c_size_t
+    lib.curdkv_attention_workspace_bytes.argtypes = [dp]
+    lib.curdkv_attention_out.restype = ctypes.c_int
+    lib.curdkv_attention_out.argtypes = [vp, i32, i64, i64, i64, vp, vp, dp, vp, vp, i64, vp,
+                                         ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
+    lib.curdkv_eviction_loss.restype = ctypes.c_int
+    lib.curdkv_eviction_loss.argtypes = [vp, vp, i32, i64, vp, vp, vp]
     lib.curdkv_profile_next_score.restype = ctypes.c_int
     lib.curdkv_profile_next_score.argtypes = [vp, vp]
     lib.curdkv_launch_count.restype = ctypes.c_uint64
@@ -326,6 +334,38 @@ def curdkv_cache_compress(src: DeviceCache, dst: DeviceCache, budget: int, works
                                         int(budget), int(num_sink), int(window), _ptr(workspace),
                                         workspace.numel(), _stream())
     _check(code, "curdkv_cache_compress")
+
+
+def curdkv_attention_out(Q, K, V, desc: Desc, *, scale: float = 1.0, head_rows=None, head_offsets=None,
+                         extra_zero_keys=None, O=None, workspace: Optional[torch.Tensor] = None):
+    """O = softmax(scale Q K^T) V per (b, h).  Q bf16 ``[B, Hkv, m, 128]``; K, V as described by
+    ``desc``, or packed ``[rows, 128]`` arrays when ``head_offsets`` is given."""
+    if Q.dtype != torch.bfloat16 or Q.dim() != 4 or Q.stride(3) != 1:
+        raise ValueError("Q must be bf16 [B, Hkv, m, d] with a contiguous last axis")
+    B, H, m, d = Q.shape
+    if O is None:
+        O = torch.empty((B, H, m, d), dtype=torch.float32, device=Q.device)
+    if workspace is None:
+        nbytes = int(load().curdkv_attention_workspace_bytes(ctypes.byref(desc)))
+        workspace = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=Q.device)
+    packed_rows = K.shape[0] if head_offsets is not None else 0
+    code = load().curdkv_attention_out(_ptr(Q), m, Q.stride(0), Q.stride(1), Q.stride(2), _ptr(K), _ptr(V),
+                                       ctypes.byref(desc), _ptr(head_rows), _ptr(head_offsets),
+                                       packed_rows, _ptr(extra_zero_keys), float(scale), _ptr(O),
+                                       _ptr(workspace), workspace.numel(), _stream())
+    _check(code, "curdkv_attention_out")
+    return O, workspace
+
+
+def curdkv_eviction_loss(O_full, O_comp):
+    """(||O - O'||_F, ||O||_F) per (b, h) for fp32 ``[B, Hkv, m, d]`` outputs."""
+    B, H = O_full.shape[:2]
+    loss = torch.empty((B, H), dtype=torch.float32, device=O_full.device)
+    ref = torch.empty_like(loss)
+    code = load().curdkv_eviction_loss(_ptr(O_full), _ptr(O_comp), B * H, O_full[0, 0].numel(), _ptr(loss),
+                                       _ptr(ref), _stream())
+    _check(code, "curdkv_eviction_loss")
+    return loss, ref
 
 
 def curdkv_profile_next_score(start: torch.cuda.Event, stop: torch.cuda.Event) -> None:

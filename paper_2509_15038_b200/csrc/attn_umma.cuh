@@ -1,0 +1,339 @@
+// Attention output O = softmax(scale * Q K^T) V of one cache (full or
+// compressed), the quantity whose change under eviction Lemma 1 bounds.  Used by
+// the eviction-loss evaluator; not a serving kernel (no causal mask: every
+// query sees the whole cache, as in the question-after-context setting).
+//
+// One CTA per (problem, block of 128 queries).  Exact two-pass softmax on the
+// tensor cores:
+//   pass 1   S = Q K_t^T per 128-key tile (tcgen05.mma, fp32 in TMEM), row maxima
+//   pass 2   S again, P = exp(S - max) split into bf16 P_hi + P_lo in shared
+//            memory, O += P_hi V_t + P_lo V_t (V tile read MN-major), row sums
+// Warp roles and bounded waits as in sketch_umma_kernel.  Keys at or beyond the
+// problem's row count are masked by index; the value rows among them are cleared
+// in shared memory so that padding can never leak NaNs through a zero weight.
+#pragma once
+#include "whiten_umma.cuh"
+
+namespace curdkv {
+namespace umma {
+
+struct AttnArgs {
+  const int32_t* rows;       // [problems] valid key rows of each problem
+  const int32_t* row_start;  // [problems] first row inside the packed array, or nullptr
+  const int32_t* extra_zero; // [problems] further keys with logit 0 and value 0 (Lemma 1), or nullptr
+  int heads, m, packed;      // query rows per problem; packed: K, V are one [rows, d] array
+  float scale;
+  float* O;                  // [problems][m][128]
+  uint32_t* status;
+};
+
+constexpr int kAttnRing = 3;
+constexpr int kAttnQ = 0;
+constexpr int kAttnPhi = kSlotBytes;
+constexpr int kAttnPlo = 2 * kSlotBytes;
+constexpr int kAttnSlot0 = 3 * kSlotBytes;
+constexpr int kAttnBar = kAttnSlot0 + kAttnRing * kSlotBytes;
+constexpr int kAttnDynamic = kAttnBar + 256 + 1024;
+constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O at 256
+
+// P V: A = P K-major, B = V tile MN-major (contraction over the keys)
+__host__ __device__ constexpr uint32_t instr_desc_pv() { return instr_desc_bf16(128) | (1u << 16); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                      const __grid_constant__ CUtensorMap map_v, const AttnArgs a) {
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t bar0 = base + kAttnBar;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kAttnRing + s); };
+  auto s_full_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + s); };
+  auto s_empty_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 2 + s); };
+  const uint32_t q_full_bar = bar0 + 8u * (2 * kAttnRing + 4);
+  const uint32_t p_ready_bar = bar0 + 8u * (2 * kAttnRing + 5);
+  const uint32_t p_empty_bar = bar0 + 8u * (2 * kAttnRing + 6);
+  const uint32_t o_full_bar = bar0 + 8u * (2 * kAttnRing + 7);
+  const uint32_t drain_bar = bar0 + 8u * (2 * kAttnRing + 8);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + kAttnBar + 8 * (2 * kAttnRing + 9));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const int q_blocks = (a.m + kTileRows - 1) / kTileRows;
+  const int p = blockIdx.x / q_blocks, qb = blockIdx.x % q_blocks;
+  const int b = p / a.heads, h = p % a.heads;
+  const int n = max(a.rows[p], 0);
+  const int T = (n + kTileRows - 1) / kTileRows;           // key tiles
+  const int key0 = a.row_start != nullptr ? a.row_start[p] : 0;
+  const int kh = a.packed ? 0 : h, kb = a.packed ? 0 : b;
+  const int extra = a.extra_zero != nullptr ? max(a.extra_zero[p], 0) : 0;
+
+  if (T == 0) {                                            // empty cache: define O = 0
+    for (int e = tid; e < kTileRows * 128; e += kThreads) {
+      const int row = qb * kTileRows + e / 128;
+      if (row < a.m) a.O[((size_t)p * a.m + row) * 128 + (e & 127)] = 0.f;
+    }
+    return;
+  }
+
+  if (tid == 0) {
+    for (int s = 0; s < kAttnRing; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(s_full_bar(s), 1); mbar_init(s_empty_bar(s), 128); }
+    mbar_init(q_full_bar, 1);
+    mbar_init(p_ready_bar, 128);
+    mbar_init(p_empty_bar, 1);
+    mbar_init(o_full_bar, 1);
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_holder)),
+                 "r"((uint32_t)kAttnTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  // Tiles go through the ring in the order the MMA issuer consumes them:
+  //   pass 1: K_0 .. K_{T-1};  pass 2: K_0, then for every t: K_{t+1} (if any), V_t.
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint64_t pol_keep;
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+      mbar_arrive_expect_tx(q_full_bar, kSlotBytes);
+      tma_load_4d(base + kAttnQ, &map_q, q_full_bar, 0, qb * kTileRows, h, b, pol_keep);
+      tma_load_4d(base + kAttnQ + kHalfBytes, &map_q, q_full_bar, 64, qb * kTileRows, h, b, pol_keep);
+      uint32_t it = 0;
+      bool ok = true;
+      auto load = [&](const CUtensorMap* map, int t) {
+        const int slot = it % kAttnRing;
+        const uint32_t phase = (it / kAttnRing) & 1u;
+        if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status))) return;
+        mbar_arrive_expect_tx(full_bar(slot), kSlotBytes);
+        const uint32_t dst = base + kAttnSlot0 + slot * kSlotBytes;
+        // the key tiles of a problem are read by all of its query blocks: no evict-first
+        tma_load_4d(dst, map, full_bar(slot), 0, key0 + t * kTileRows, kh, kb, pol_keep);
+        tma_load_4d(dst + kHalfBytes, map, full_bar(slot), 64, key0 + t * kTileRows, kh, kb, pol_keep);
+        ++it;
+      };
+      for (int t = 0; ok && t < T; ++t) load(&map_k, t);
+      if (ok) load(&map_k, 0);
+      for (int t = 0; ok && t < T; ++t) {
+        if (t + 1 < T) load(&map_k, t + 1);
+        if (ok) load(&map_v, t);
+      }
+      if (!ok) {
+        const uint32_t pending = it < (uint32_t)kAttnRing ? it : (uint32_t)kAttnRing;
+        for (uint32_t q = it - pending; q < it; ++q) {
+          unsigned long long t0 = global_ns();
+          while (!mbar_try_wait(full_bar(q % kAttnRing), (q / kAttnRing) & 1u) &&
+                 global_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = instr_desc_bf16(128);
+      constexpr uint32_t idesc_pv = instr_desc_pv();
+      uint32_t it = 0, job = 0;
+      bool ok = mbar_wait(q_full_bar, 0, abort_flag, a.status);
+      tc_fence_after();
+      auto issue_s = [&]() {                               // S[job & 1] = Q K^T for the next K tile
+        const uint32_t buf = job & 1u;
+        if (!(ok = mbar_wait(s_empty_bar(buf), ((job >> 1) & 1u) ^ 1u, abort_flag, a.status))) return;
+        const int slot = it % kAttnRing;
+        if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status))) return;
+        tc_fence_after();
+        const uint32_t k_base = base + kAttnSlot0 + slot * kSlotBytes;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
+          tc_mma_bf16(tmem_base + buf * 128u, smem_desc_sw128(base + kAttnQ + off),
+                      smem_desc_sw128(k_base + off), idesc_s, k > 0);
+        }
+        tc_commit(empty_bar(slot));
+        tc_commit(s_full_bar(buf));
+        ++it;
+        ++job;
+      };
+      for (int t = 0; ok && t < T; ++t) issue_s();         // pass 1
+      if (ok) issue_s();                                   // pass 2, tile 0
+      for (int t = 0; ok && t < T; ++t) {
+        if (t + 1 < T) issue_s();
+        if (!ok) break;
+        const int slot = it % kAttnRing;
+        if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status))) break;
+        const int rows = min(kTileRows, n - t * kTileRows);
+        const int groups = (rows + 15) >> 4;
+        if (rows < groups * 16) {                          // clear the padding rows the last MMA reads
+          for (int j = rows; j < groups * 16; ++j)
+            for (int half = 0; half < 2; ++half)
+              for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(base_ptr + kAttnSlot0 + slot * kSlotBytes + half * kHalfBytes +
+                                          j * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        if (!(ok = mbar_wait(p_ready_bar, (uint32_t)t & 1u, abort_flag, a.status))) break;
+        tc_fence_after();
+        const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
+        for (int part = 0; part < 2; ++part) {             // P_hi, then P_lo
+          const uint32_t p_base = base + (part ? kAttnPlo : kAttnPhi);
+          for (int g = 0; g < groups; ++g) {               // 16 keys per MMA
+            const uint32_t poff = (g >> 2) * kHalfBytes + (g & 3) * 32;
+            tc_mma_bf16(tmem_base + 256u, smem_desc_sw128(p_base + poff),
+                        smem_desc_mn_sw128(v_base + g * 2048), idesc_pv, (t > 0 || part > 0 || g > 0) ? 1u : 0u);
+          }
+        }
+        tc_commit(empty_bar(slot));
+        tc_commit(p_empty_bar);
+        ++it;
+      }
+      if (ok) tc_commit(o_full_bar);
+      if (!ok) {
+        tc_commit(drain_bar);
+        unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax + epilogue
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;                     // query row inside the block = TMEM lane
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    constexpr float kLog2e = 1.4426950408889634f;
+    const float sc = a.scale * kLog2e;                     // logits in units of log2
+    float top = extra > 0 ? 0.f : -INFINITY;
+    uint32_t job = 0;
+    bool ok = true;
+    for (int t = 0; ok && t < T; ++t, ++job) {             // pass 1: row maxima
+      const uint32_t buf = job & 1u;
+      ok = mbar_wait(s_full_bar(buf), (job >> 1) & 1u, abort_flag, a.status);
+      if (!(ok = __all_sync(0xffffffffu, ok))) break;
+      tc_fence_after();
+      const int valid = n - t * kTileRows;                 // keys of this tile that exist
+#pragma unroll 1
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        float v[32];
+        tmem_ld32(lane_addr + buf * 128u + c0, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (c0 + c < valid) top = fmaxf(top, v[c] * sc);
+      }
+      tc_fence_before();
+      mbar_arrive(s_empty_bar(buf));
+    }
+    float sum = extra > 0 ? (float)extra * exp2f(-top) : 0.f;
+    for (int t = 0; ok && t < T; ++t, ++job) {             // pass 2: P and row sums
+      const uint32_t buf = job & 1u;
+      ok = mbar_wait(s_full_bar(buf), (job >> 1) & 1u, abort_flag, a.status);
+      if (ok && t > 0) ok = mbar_wait(p_empty_bar, (uint32_t)(t - 1) & 1u, abort_flag, a.status);
+      if (!(ok = __all_sync(0xffffffffu, ok))) break;
+      tc_fence_after();
+      const int valid = n - t * kTileRows;
+#pragma unroll 1
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        float v[32];
+        tmem_ld32(lane_addr + buf * 128u + c0, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {                      // 8 keys -> one 16-byte chunk of P_hi, P_lo
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float w[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int c = g * 8 + e * 2 + q;
+              w[q] = c0 + c < valid ? exp2f(v[c] * sc - top) : 0.f;
+            }
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(w[0]), h1 = __float2bfloat16_rn(w[1]);
+            const __nv_bfloat16 l0 = __float2bfloat16_rn(w[0] - __bfloat162float(h0));
+            const __nv_bfloat16 l1 = __float2bfloat16_rn(w[1] - __bfloat162float(h1));
+            sum += (__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1));
+            hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+          }
+          const int key = c0 + g * 8;                      // first key of the chunk inside the tile
+          const uint32_t off = (uint32_t)(key >> 6) * kHalfBytes + (uint32_t)r * 128u +
+                               ((((uint32_t)(key & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4);
+          *reinterpret_cast<uint4*>(base_ptr + kAttnPhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(base_ptr + kAttnPlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(s_empty_bar(buf));
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(p_ready_bar);
+    }
+    if (ok) {
+      ok = mbar_wait(o_full_bar, 0, abort_flag, a.status);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      const int row = qb * kTileRows + r;
+      const float inv = sum > 0.f ? 1.f / sum : 0.f;
+      float* out = a.O + ((size_t)p * a.m + row) * 128;
+#pragma unroll 1
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        float v[32];
+        tmem_ld32(lane_addr + 256u + c0, v);
+        tmem_ld_wait();
+        if (row < a.m) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 4)
+            *reinterpret_cast<float4*>(out + c0 + c) =
+                make_float4(v[c] * inv, v[c + 1] * inv, v[c + 2] * inv, v[c + 3] * inv);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"((uint32_t)kAttnTmemCols)
+                 : "memory");
+  }
+}
+
+// ||O - O'||_F and ||O||_F per problem.  grid = problems, block = 256; fixed summation order.
+__global__ void __launch_bounds__(256) frob_diff_kernel(const float* O, const float* Oc, int elems,
+                                                        float* loss, float* ref_norm) {
+  __shared__ double red[2][8];
+  const int p = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* x = O + (size_t)p * elems;
+  const float* y = Oc + (size_t)p * elems;
+  double d2 = 0.0, r2 = 0.0;
+  for (int e = tid; e < elems; e += 256) {
+    const double u = x[e], w = (double)x[e] - (double)y[e];
+    d2 += w * w;
+    r2 += u * u;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    d2 += __shfl_xor_sync(0xffffffffu, d2, o);
+    r2 += __shfl_xor_sync(0xffffffffu, r2, o);
+  }
+  if (lane == 0) { red[0][warp] = d2; red[1][warp] = r2; }
+  __syncthreads();
+  if (tid == 0) {
+    double s0 = 0.0, s1 = 0.0;
+    for (int w = 0; w < 8; ++w) { s0 += red[0][w]; s1 += red[1][w]; }
+    loss[p] = (float)sqrt(s0);
+    if (ref_norm != nullptr) ref_norm[p] = (float)sqrt(s1);
+  }
+}
+
+}  // namespace umma
+}  // namespace curdkv

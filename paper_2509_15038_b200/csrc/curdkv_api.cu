@@ -11,6 +11,7 @@
 #include "select.cuh"
 #include "whiten_factor.cuh"
 #include "whiten_umma.cuh"
+#include "attn_umma.cuh"
 
 namespace {
 
@@ -168,6 +169,13 @@ WhitenLayout whiten_layout(const curdkv_desc* d, size_t after_tile_sums) {
   L.W = L.partials + round256(P * whiten_segments(d) * 2 * 128 * 128 * sizeof(float));
   L.total = L.W + round256(P * 2 * 128 * (size_t)(d->r > 0 ? d->r : 1) * sizeof(float));
   return L;
+}
+
+// valid key rows of every (sequence, head) when the caller gave none: the sequence lengths
+__global__ void rows_from_seqlens_kernel(const int32_t* seqlens, int heads, int n_max, int problems,
+                                         int32_t* rows) {
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p < problems) rows[p] = seq_len_of(seqlens, p / heads, n_max);
 }
 
 KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
@@ -496,6 +504,93 @@ curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, 
       cudaMemcpyAsync(status_flags, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice,
                       static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
     return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+size_t curdkv_attention_workspace_bytes(const curdkv_desc* desc) {
+  if (check_desc(desc) != CURDKV_OK) return 0;
+  return kStatusBytes + round256((size_t)desc->batch * desc->kv_heads * sizeof(int32_t));
+}
+
+curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stride_b, int64_t q_stride_h,
+                                   int64_t q_stride_n, const void* K, const void* V,
+                                   const curdkv_desc* desc, const int32_t* head_rows,
+                                   const int32_t* head_offsets, int64_t packed_rows,
+                                   const int32_t* extra_zero_keys, float scale, float* O, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if (Q == nullptr || K == nullptr || V == nullptr || O == nullptr || workspace == nullptr)
+    return CURDKV_ERR_INVALID_ARG;
+  if (desc->d != 128) return CURDKV_ERR_UNSUPPORTED;
+  if (q_rows < 1 || !(scale == scale)) return CURDKV_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return CURDKV_ERR_INVALID_ARG;
+  if (q_stride_b < 0 || q_stride_h < 0 || q_stride_n < 128 || q_stride_b % 8 || q_stride_h % 8 || q_stride_n % 8)
+    return CURDKV_ERR_INVALID_ARG;
+  const bool packed = head_offsets != nullptr;
+  if (packed && (head_rows == nullptr || packed_rows < 1)) return CURDKV_ERR_INVALID_ARG;
+  if (!packed && (st = check_kv(K, V, desc)) != CURDKV_OK) return st;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  if (workspace_bytes < curdkv_attention_workspace_bytes(desc)) return CURDKV_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  if (P == 0) return CURDKV_OK;
+  const int64_t q_blocks = ((int64_t)q_rows + kTileRows - 1) / kTileRows;
+  if (P * q_blocks > 0x7fffffffLL) return CURDKV_ERR_UNSUPPORTED;
+
+  const int32_t* rows = head_rows;
+  if (rows == nullptr) {
+    int32_t* mine = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
+    rows_from_seqlens_kernel<<<(unsigned)((P + 255) / 256), 256, 0, stream>>>(
+        desc->seqlens, desc->kv_heads, desc->n_max, (int)P, mine);
+    if (!launch_ok()) return CURDKV_ERR_CUDA;
+    rows = mine;
+  }
+  curdkv_desc qd = *desc;
+  qd.n_max = q_rows;
+  CUtensorMap mq, mk, mv;
+  if (!make_tile_map(&mq, Q, &qd, q_stride_b, q_stride_h, q_stride_n)) return CURDKV_ERR_CUDA;
+  if (packed) {
+    curdkv_desc pd = *desc;                                // one [packed_rows, 128] array
+    pd.batch = pd.kv_heads = 1;
+    if (packed_rows > 0x7fffffffLL) return CURDKV_ERR_UNSUPPORTED;
+    pd.n_max = (int32_t)packed_rows;
+    if (!make_tile_map(&mk, K, &pd, 0, 0, 128) || !make_tile_map(&mv, V, &pd, 0, 0, 128))
+      return CURDKV_ERR_CUDA;
+  } else if (!make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) ||
+             !make_tile_map(&mv, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n)) {
+    return CURDKV_ERR_CUDA;
+  }
+  umma::AttnArgs a;
+  a.rows = rows;
+  a.row_start = packed ? head_offsets : nullptr;
+  a.extra_zero = extra_zero_keys;
+  a.heads = desc->kv_heads;
+  a.m = q_rows;
+  a.packed = packed ? 1 : 0;
+  a.scale = scale;
+  a.O = O;
+  a.status = static_cast<uint32_t*>(workspace);
+  if (cudaFuncSetAttribute(umma::attention_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           umma::kAttnDynamic) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  umma::attention_umma_kernel<<<(unsigned)(P * q_blocks), umma::kThreads, umma::kAttnDynamic, stream>>>(
+      mq, mk, mv, a);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compressed, int32_t problems,
+                                   int64_t elems_per_problem, float* loss, float* ref_norm,
+                                   void* cuda_stream) {
+  if (O_full == nullptr || O_compressed == nullptr || loss == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (problems < 0 || elems_per_problem < 0 || elems_per_problem > 0x7fffffffLL)
+    return CURDKV_ERR_INVALID_ARG;
+  if (problems == 0) return CURDKV_OK;
+  umma::frob_diff_kernel<<<(unsigned)problems, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      O_full, O_compressed, (int)elems_per_problem, loss, ref_norm);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }
 

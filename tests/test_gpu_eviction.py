@@ -1,0 +1,132 @@
+"""Eviction-loss evaluator on the GPU (attention output of the full and the compressed cache,
+through the C ABI) against the fp64 oracle.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import curdkv_eviction_oracle as ev
+from paper_2509_15038_b200 import binding as cur
+from paper_2509_15038_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+# exp2 of fp32 logits and bf16 (hi + lo) weights: outputs agree with fp64 to ~1e-5 of the largest
+# entry; 2e-4 leaves room for logits of a few hundred
+OUT_TOL = 2e-4
+
+
+def _f64(t):
+    return synth.u16_to_f64(synth.to_u16(t))
+
+
+def _queries(B, H, m, d, seed, gain=1.0):
+    g = torch.Generator(device=DEV).manual_seed(seed)
+    return (gain * torch.randn((B, H, m, d), generator=g, device=DEV)).to(torch.bfloat16)
+
+
+def _check_out(O, Q, K, V, lens, scale, extra=None, what=""):
+    got = O.cpu().numpy().astype(np.float64)
+    Qf, Kf, Vf = _f64(Q), _f64(K), _f64(V)
+    B, H = Q.shape[:2]
+    for b in range(B):
+        for h in range(H):
+            n = int(lens[b, h])
+            if n == 0:
+                assert np.all(got[b, h] == 0)
+                continue
+            want = ev.attention_out(Qf[b, h], Kf[b, h, :n], Vf[b, h, :n], scale,
+                                    0 if extra is None else int(extra[b, h]))
+            err = np.abs(got[b, h] - want).max()
+            assert err <= OUT_TOL * np.abs(want).max(), f"{what} b={b} h={h}: err {err:.3e}"
+
+
+@pytest.mark.parametrize("scale", [1.0 / np.sqrt(128.0), 1.0])
+def test_attention_out_matches_oracle(scale):
+    """Ragged key counts incl. 0, 1 and non-multiples of the tile; query rows not a multiple of 128."""
+    B, H, n, d, m = 3, 2, 1000, 128, 200
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=B, n_max=n, kv_heads=H, q_heads=H)
+    K, V, _ = synth.make_kv(w, DEV)
+    Q = _queries(B, H, m, d, seed=5, gain=0.5 if scale == 1.0 else 1.0)
+    lens = np.array([1000, 333, 0], dtype=np.int32)
+    desc = cur.make_desc(K, V, 32, seqlens=torch.as_tensor(lens, device=DEV))
+    O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=scale)
+    assert cur.curdkv_device_status(ws) == 0
+    _check_out(O, Q, K, V, np.repeat(lens[:, None], H, 1), scale, what=f"scale={scale:.3f}")
+    # explicit per-head row counts override the sequence lengths
+    rows = np.array([[1, 129], [128, 999], [7, 0]], dtype=np.int32)
+    O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=scale,
+                                     head_rows=torch.as_tensor(rows.reshape(-1), device=DEV))
+    assert cur.curdkv_device_status(ws) == 0
+    _check_out(O, Q, K, V, rows, scale, what="head_rows")
+
+
+def test_constant_values_and_nan_padding():
+    """Softmax rows sum to one (V = 1 comes back as 1), and NaNs in the padding rows never leak."""
+    B, H, n, d, m = 1, 2, 300, 128, 64
+    g = torch.Generator(device=DEV).manual_seed(1)
+    K = torch.randn((B, H, n, d), generator=g, device=DEV).to(torch.bfloat16)
+    V = torch.ones((B, H, n, d), device=DEV).to(torch.bfloat16)
+    K[:, :, 200:] = float("nan")
+    V[:, :, 200:] = float("nan")
+    Q = _queries(B, H, m, d, seed=2)
+    desc = cur.make_desc(K, V, 32, seqlens=torch.tensor([200], dtype=torch.int32, device=DEV))
+    O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=0.1)
+    assert cur.curdkv_device_status(ws) == 0
+    np.testing.assert_allclose(O.cpu().numpy(), 1.0, rtol=1e-5)
+
+
+@pytest.mark.parametrize("adaptive", [False, True])
+def test_eviction_loss_of_a_curdkv_selection(adaptive):
+    """score -> select -> compact -> attention on both caches -> loss, against the oracle's loss for
+    the rows the GPU kept; also Lemma 1's zeroed form and its bound."""
+    B, H, n, d, m, k = 2, 4, 2048, 128, 256, 300
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=B, n_max=n, kv_heads=H, q_heads=H, data_seed=9)
+    K, V, _ = synth.make_kv(w, DEV)
+    Q = _queries(B, H, m, d, seed=3)
+    scale = 1.0 / np.sqrt(d)
+    G = torch.as_tensor(synth.make_G(d, 32, seed=0), device=DEV)
+    desc = cur.make_desc(K, V, 32)
+    ws = cur.alloc_workspace(desc, k, adaptive)
+    scores, _ = cur.curdkv_score(K, V, G, desc, ws)
+    idx, cnt, off = cur.curdkv_select(scores, desc, k, num_sink=4, window=32, adaptive=adaptive, workspace=ws)
+    Kc, Vc = cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=adaptive, workspace=ws)
+    O, _ = cur.curdkv_attention_out(Q, K, V, desc, scale=scale)
+    rows = cnt.reshape(-1).contiguous()
+    if adaptive:
+        Oc, aws = cur.curdkv_attention_out(Q, Kc, Vc, desc, scale=scale, head_rows=rows, head_offsets=off)
+    else:
+        cdesc = cur.make_desc(Kc, Vc, 32)
+        Oc, aws = cur.curdkv_attention_out(Q, Kc, Vc, cdesc, scale=scale, head_rows=rows)
+    assert cur.curdkv_device_status(aws) == 0
+    loss, ref = cur.curdkv_eviction_loss(O, Oc)
+    extra = (n - cnt).to(torch.int32).reshape(-1).contiguous()
+    if adaptive:
+        Oz, _ = cur.curdkv_attention_out(Q, Kc, Vc, desc, scale=scale, head_rows=rows, head_offsets=off,
+                                         extra_zero_keys=extra)
+    else:
+        Oz, _ = cur.curdkv_attention_out(Q, Kc, Vc, cdesc, scale=scale, head_rows=rows, extra_zero_keys=extra)
+    loss_z, _ = cur.curdkv_eviction_loss(O, Oz)
+
+    Qf, Kf, Vf = _f64(Q), _f64(K), _f64(V)
+    gi, gc, go = idx.cpu().numpy(), cnt.cpu().numpy(), off.cpu().numpy()
+    for b in range(B):
+        for h in range(H):
+            p = b * H + h
+            kept = gi[go[p]: go[p] + gc[b, h]] if adaptive else gi[b, h, : gc[b, h]]
+            want, want_ref = ev.eviction_loss(Qf[b, h], Kf[b, h], Vf[b, h], kept, scale)
+            assert abs(float(loss[b, h]) - want) <= 1e-3 * want_ref, (b, h, float(loss[b, h]), want)
+            assert abs(float(ref[b, h]) - want_ref) <= 1e-4 * want_ref
+            want_z, _ = ev.eviction_loss(Qf[b, h], Kf[b, h], Vf[b, h], kept, scale, zeroed=True)
+            assert abs(float(loss_z[b, h]) - want_z) <= 1e-3 * want_ref
+            assert float(loss_z[b, h]) <= ev.lemma1_bound(Vf[b, h], kept)          # Lemma 1
+    # keeping every row loses nothing
+    same, _ = cur.curdkv_eviction_loss(O, O)
+    assert float(same.max()) == 0.0
+
+
+def test_attention_rejects_bad_arguments():
+    K = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device=DEV)
+    Q = torch.zeros((1, 1, 16, 64), dtype=torch.bfloat16, device=DEV)
+    desc = cur.make_desc(K, K, 32)
+    with pytest.raises(cur.CurdkvError):
+        cur.curdkv_attention_out(Q, K, K, desc)
