@@ -397,6 +397,104 @@ def run_decode(args):
     }), flush=True)
 
 
+# --------------------------------------------------------------------------- eviction loss
+
+EVICT = dict(workload="cfg2", q_rows=512)
+
+
+def run_evict(args):
+    """Eviction-loss workload (Lemma 1): attention output of the full and of the compressed cache
+    for synthetic queries, and the relative loss of CurDKV against key-only, value-only and random
+    selections of the same size.  One step = attention over the full cache + over the CurDKV cache +
+    the Frobenius difference."""
+    from paper_2509_15038_b200 import binding as cur
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    w = synth.CONFIGS[EVICT["workload"]]
+    m = EVICT["q_rows"]
+    K, V, _ = synth.make_kv(w, dev)
+    LB, H, n, d = K.shape
+    g = torch.Generator(device=dev).manual_seed(99)
+    # queries that look like keys of the same head (same outlier channels), so that logits are not flat
+    Q = (K[:, :, torch.randint(0, n, (m,), generator=g, device=dev)].float()
+         + torch.randn((LB, H, m, d), generator=g, device=dev)).to(torch.bfloat16)
+    scale = 1.0 / float(np.sqrt(d))
+    G = torch.as_tensor(synth.make_G(d, w.r, seed=0), device=dev)
+    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads)
+    ws = cur.alloc_workspace(desc, w.budget)
+
+    def select(score_mode=0, use_projection=1, random=False):
+        dsc = cur.make_desc(K, V, w.r, q_heads=w.q_heads, score_mode=score_mode, use_projection=use_projection)
+        scores, _ = cur.curdkv_score(K, V, G, dsc, ws)
+        if random:
+            scores = torch.rand(scores.shape, generator=g, device=dev)
+        idx, cnt, off = cur.curdkv_select(scores, dsc, w.budget, num_sink=w.num_sink, window=w.window, workspace=ws)
+        Kc, Vc = cur.curdkv_compact(K, V, dsc, idx, cnt, off, workspace=ws)
+        return Kc, Vc, cnt.reshape(-1).contiguous()
+
+    O = torch.empty((LB, H, m, d), dtype=torch.float32, device=dev)
+    Oc = torch.empty_like(O)
+    Kc, Vc, rows = select()
+    cdesc = cur.make_desc(Kc, Vc, w.r)
+    aws = torch.empty((1 << 20,), dtype=torch.uint8, device=dev)
+
+    def step():
+        cur.curdkv_attention_out(Q, K, V, desc, scale=scale, O=O, workspace=aws)
+        cur.curdkv_attention_out(Q, Kc, Vc, cdesc, scale=scale, head_rows=rows, O=Oc, workspace=aws)
+        return cur.curdkv_eviction_loss(O, Oc)
+
+    for _ in range(max(args.warmup, 3)):
+        loss, ref = step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = cur.launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        loss, ref = step()
+    t1.record()
+    torch.cuda.synchronize()
+    launches = cur.launch_count() - launches0
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / args.steps
+    rel = {"curdkv": float((loss / ref).mean())}
+    for name, kw in (("key_only", dict(score_mode=1)), ("value_only", dict(score_mode=2)),
+                     ("key_norm", dict(score_mode=1, use_projection=0)), ("random", dict(random=True))):
+        Kx, Vx, rx = select(**kw)
+        cur.curdkv_attention_out(Q, Kx, Vx, cur.make_desc(Kx, Vx, w.r), scale=scale, head_rows=rx, O=Oc,
+                                 workspace=aws)
+        lx, _ = cur.curdkv_eviction_loss(O, Oc)
+        rel[name] = float((lx / ref).mean())
+    P = LB * H
+    kept = int(rows.sum())
+    flops = 4.0 * m * d * (P * n + kept)                 # one Q K^T and one P V per cache
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, peak_kind = float(json.load(f)["bf16_tflops_sustained"]), "measured sustained bf16 cuBLAS"
+    except Exception:
+        peak, peak_kind = 1400.0, "fallback sustained bf16"
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "attention_query_key_pairs_per_s", "value": m * (P * n + kept) / (ms * 1e-3),
+        "unit": "query-key pairs/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"evict: {w.name} cache ({w.layers} layers x {w.kv_heads} KV heads, n={n}, "
+                               f"budget {w.budget}), {m} synthetic query rows per KV head, scale 1/sqrt(d)"},
+        "relative_eviction_loss": rel, "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "attention_umma_kernel (full + compressed cache)",
+                     "achieved": tf, "peak": peak, "peak_kind": peak_kind, "unit": "TFLOP/s",
+                     "frac": tf / peak, "traffic": None,
+                     "note": "algorithmic flops = one QK^T and one PV; the kernel issues twice that "
+                             "(two-pass softmax, hi/lo weights)"},
+    }), flush=True)
+
+
 # --------------------------------------------------------------------------- oracle arm
 
 def oracle_sample(w, elements):
@@ -484,17 +582,17 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
-    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode", "evict"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--whiten", action="store_true",
                     help="score with the whitened sketch (approximate leverage scores; reads K, V twice)")
     ap.add_argument("--e2e-steps", type=int, default=3,
                     help="steps of the host-buffer end-to-end leg (0 disables it)")
     args = ap.parse_args()
-    if args.workload == "decode":
+    if args.workload in ("decode", "evict"):
         if args.impl == "reference":
             raise SystemExit("the reference arm times the prefill workloads only")
-        run_decode(args)
+        run_decode(args) if args.workload == "decode" else run_evict(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
