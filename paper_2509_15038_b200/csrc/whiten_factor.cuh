@@ -26,6 +26,86 @@ struct FactorArgs {
   uint32_t* status;
 };
 
+// Elimination steps k = 32*KU .. 32*KU + 31: only the blocks u, v >= KU still change, so the
+// phase is compiled for exactly those (no selects on the block index, no work on finished blocks).
+template <int KU>
+__device__ __forceinline__ void cholesky_phase(double (&m)[4][4], double* Lt, int ti, int tj, bool& bad) {
+  constexpr int D = kFactorD;
+#pragma unroll 1
+  for (int kt = 0; kt < 32; ++kt) {
+    const int k = 32 * KU + kt;
+    if (tj == kt) {                                        // owners publish column k, pivot included
+#pragma unroll
+      for (int u = KU; u < 4; ++u) Lt[k * D + ti + 32 * u] = m[u][KU];
+    }
+    __syncthreads();
+    double piv = Lt[k * D + k];
+    if (!(piv > 0.0)) { piv = 1e-300; bad = true; }
+    // 1 / piv: fp32 seed and two Newton steps; out-of-range pivots take the exact division
+    double inv;
+    if (piv > 1e-30 && piv < 1e30) {
+      inv = (double)(1.0f / (float)piv);
+      inv = inv * (2.0 - piv * inv);
+      inv = inv * (2.0 - piv * inv);
+    } else {
+      inv = 1.0 / piv;
+    }
+    double li[4], lj[4];
+#pragma unroll
+    for (int u = KU; u < 4; ++u) {
+      li[u] = Lt[k * D + ti + 32 * u] * inv;
+      lj[u] = Lt[k * D + tj + 32 * u];
+    }
+    if (ti <= kt) li[KU] = 0.0;                            // rows and columns up to k are finished
+    if (tj <= kt) lj[KU] = 0.0;
+#pragma unroll
+    for (int u = KU; u < 4; ++u)
+#pragma unroll
+      for (int v = KU; v < 4; ++v) m[u][v] -= li[u] * lj[v];
+  }
+}
+
+// Back-substitution steps i = 32*IU + 31 .. 32*IU: only rows of blocks u <= IU are still open.
+template <int IU, int WCOLS>
+__device__ __forceinline__ void backsub_phase(double (&x)[4][2], const double* Lt, double* wrow, int ti,
+                                              int tj) {
+  constexpr int D = kFactorD;
+#pragma unroll 1
+  for (int it = 31; it >= 0; --it) {
+    const int i = 32 * IU + it;
+    double* wr = wrow + (i & 1) * 64;
+    if (ti == it) {
+      const double inv = 1.0 / Lt[i * D + i];
+#pragma unroll
+      for (int w = 0; w < WCOLS; ++w) {
+        x[IU][w] *= inv;                                   // W[i][c]
+        wr[tj + 32 * w] = x[IU][w];
+      }
+    }
+    __syncthreads();
+    double wv[2];
+#pragma unroll
+    for (int w = 0; w < WCOLS; ++w) wv[w] = wr[tj + 32 * w];
+#pragma unroll
+    for (int u = 0; u <= IU; ++u) {
+      const int row = ti + 32 * u;
+      if (u < IU || ti < it) {
+        const double l = Lt[row * D + i];                  // L[i][row]
+#pragma unroll
+        for (int w = 0; w < WCOLS; ++w) x[u][w] -= l * wv[w];
+      }
+    }
+  }
+}
+
+template <int WCOLS>
+__device__ __forceinline__ void backsub_all(double (&x)[4][2], const double* Lt, double* wrow, int ti, int tj) {
+  backsub_phase<3, WCOLS>(x, Lt, wrow, ti, tj);
+  backsub_phase<2, WCOLS>(x, Lt, wrow, ti, tj);
+  backsub_phase<1, WCOLS>(x, Lt, wrow, ti, tj);
+  backsub_phase<0, WCOLS>(x, Lt, wrow, ti, tj);
+}
+
 // grid = batch*heads*2, block = 1024, dynamic shared memory = kFactorSmemBytes.
 __global__ void __launch_bounds__(kFactorThreads, 1) whiten_factor_kernel(const FactorArgs a) {
   extern __shared__ double fsm[];
@@ -78,43 +158,10 @@ __global__ void __launch_bounds__(kFactorThreads, 1) whiten_factor_kernel(const 
   // ---- Cholesky by outer products: step k publishes column k (unscaled, pivot included) and
   // every thread updates its elements below and right of it: m_ij -= m_ik m_jk / m_kk
   bool bad = false;
-#pragma unroll 1
-  for (int k = 0; k < D; ++k) {
-    const int ku = k >> 5, kt = k & 31;
-    if (tj == kt) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        double c = 0.0;
-#pragma unroll
-        for (int v = 0; v < 4; ++v)
-          if (v == ku) c = m[u][v];
-        Lt[k * D + ti + 32 * u] = c;
-      }
-    }
-    __syncthreads();
-    double piv = Lt[k * D + k];
-    if (!(piv > 0.0)) { piv = 1e-300; bad = true; }
-    // 1 / piv: fp32 seed and two Newton steps (an fp64 division in every thread and step would
-    // cost as much as the update itself); out-of-range pivots take the exact division
-    double inv;
-    if (piv > 1e-30 && piv < 1e30) {
-      inv = (double)(1.0f / (float)piv);
-      inv = inv * (2.0 - piv * inv);
-      inv = inv * (2.0 - piv * inv);
-    } else {
-      inv = 1.0 / piv;
-    }
-    double li[4], lj[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      li[u] = ti + 32 * u > k ? Lt[k * D + ti + 32 * u] * inv : 0.0;
-      lj[u] = tj + 32 * u > k ? Lt[k * D + tj + 32 * u] : 0.0;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-#pragma unroll
-      for (int v = 0; v < 4; ++v) m[u][v] -= li[u] * lj[v];
-  }
+  cholesky_phase<0>(m, Lt, ti, tj, bad);
+  cholesky_phase<1>(m, Lt, ti, tj, bad);
+  cholesky_phase<2>(m, Lt, ti, tj, bad);
+  cholesky_phase<3>(m, Lt, ti, tj, bad);
   if (bad && tid == 0) flag_status(a.status, CURDKV_DEV_NOT_SPD);
   __syncthreads();
   // scale the published columns: L[i][k] = m_ik / sqrt(m_kk), L[k][k] = sqrt(m_kk)
@@ -139,37 +186,8 @@ __global__ void __launch_bounds__(kFactorThreads, 1) whiten_factor_kernel(const 
       x[u][w] = c < r ? (double)__ldg(a.G + (size_t)(ti + 32 * u) * r + c) : 0.0;
     }
   __syncthreads();
-#pragma unroll 1
-  for (int i = D - 1; i >= 0; --i) {
-    const int iu = i >> 5, it = i & 31;
-    double* wr = wrow + (i & 1) * 64;
-    if (ti == it) {
-      const double inv = 1.0 / Lt[i * D + i];
-#pragma unroll
-      for (int w = 0; w < 2; ++w) {
-        double v = 0.0;
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (u == iu) v = x[u][w];
-        v *= inv;
-        wr[tj + 32 * w] = v;
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (u == iu) x[u][w] = v;                        // W[i][c]
-      }
-    }
-    __syncthreads();
-    const double w0 = wr[tj], w1 = wr[tj + 32];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int row = ti + 32 * u;
-      if (row < i) {
-        const double l = Lt[row * D + i];                  // L[i][row]
-        x[u][0] -= l * w0;
-        x[u][1] -= l * w1;
-      }
-    }
-  }
+  if (r > 32) backsub_all<2>(x, Lt, wrow, ti, tj);
+  else backsub_all<1>(x, Lt, wrow, ti, tj);
 #pragma unroll
   for (int u = 0; u < 4; ++u)
 #pragma unroll
