@@ -8,7 +8,10 @@
 //   pass 1   S = Q K_t^T per 128-key tile (tcgen05.mma, fp32 in TMEM), row maxima
 //   pass 2   S again, P = exp(S - max) split into bf16 P_hi + P_lo in shared
 //            memory, O += P_hi V_t + P_lo V_t (V tile read MN-major), row sums
-// Warp roles and bounded waits as in sketch_umma_kernel.  Keys at or beyond the
+// Warp 0 feeds the TMA ring, warp 1 issues the MMAs, and two groups of four
+// softmax warps take alternate key tiles (each group owns one S accumulator
+// and one P buffer), since the exponentials, not the tensor pipe, set the pace.
+// Bounded waits as in sketch_umma_kernel.  Keys at or beyond the
 // problem's row count are masked by index; the value rows among them are cleared
 // in shared memory so that padding can never leak NaNs through a zero weight.
 #pragma once
@@ -27,11 +30,12 @@ struct AttnArgs {
   uint32_t* status;
 };
 
-constexpr int kAttnRing = 3;
+constexpr int kAttnThreads = 320;                          // TMA, MMA, 2 x 4 softmax warps
+constexpr int kAttnRing = 2;
 constexpr int kAttnQ = 0;
-constexpr int kAttnPhi = kSlotBytes;
-constexpr int kAttnPlo = 2 * kSlotBytes;
-constexpr int kAttnSlot0 = 3 * kSlotBytes;
+constexpr int kAttnP = kSlotBytes;                         // P[buf]: hi at +0, lo at +kSlotBytes
+constexpr int kAttnPBytes = 2 * kSlotBytes;
+constexpr int kAttnSlot0 = kAttnP + 2 * kAttnPBytes;
 constexpr int kAttnBar = kAttnSlot0 + kAttnRing * kSlotBytes;
 constexpr int kAttnDynamic = kAttnBar + 256 + 1024;
 constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O at 256
@@ -39,7 +43,7 @@ constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O
 // P V: A = P K-major, B = V tile MN-major (contraction over the keys)
 __host__ __device__ constexpr uint32_t instr_desc_pv() { return instr_desc_bf16(128) | (1u << 16); }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v, const AttnArgs a) {
   extern __shared__ unsigned char smem_dyn[];
@@ -50,12 +54,13 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   auto empty_bar = [&](int s) { return bar0 + 8u * (kAttnRing + s); };
   auto s_full_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + s); };
   auto s_empty_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 2 + s); };
-  const uint32_t q_full_bar = bar0 + 8u * (2 * kAttnRing + 4);
-  const uint32_t p_ready_bar = bar0 + 8u * (2 * kAttnRing + 5);
-  const uint32_t p_empty_bar = bar0 + 8u * (2 * kAttnRing + 6);
-  const uint32_t o_full_bar = bar0 + 8u * (2 * kAttnRing + 7);
-  const uint32_t drain_bar = bar0 + 8u * (2 * kAttnRing + 8);
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + kAttnBar + 8 * (2 * kAttnRing + 9));
+  auto p_ready_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 4 + s); };
+  auto p_empty_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 6 + s); };
+  const uint32_t q_full_bar = bar0 + 8u * (2 * kAttnRing + 8);
+  const uint32_t o_full_bar = bar0 + 8u * (2 * kAttnRing + 9);
+  const uint32_t drain_bar = bar0 + 8u * (2 * kAttnRing + 10);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + kAttnBar + 8 * (2 * kAttnRing + 11));
+  __shared__ float xchg[2][kTileRows];                     // row maxima, then row sums, of the two groups
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -69,7 +74,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   const int extra = a.extra_zero != nullptr ? max(a.extra_zero[p], 0) : 0;
 
   if (T == 0) {                                            // empty cache: define O = 0
-    for (int e = tid; e < kTileRows * 128; e += kThreads) {
+    for (int e = tid; e < kTileRows * 128; e += kAttnThreads) {
       const int row = qb * kTileRows + e / 128;
       if (row < a.m) a.O[((size_t)p * a.m + row) * 128 + (e & 127)] = 0.f;
     }
@@ -78,10 +83,13 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
 
   if (tid == 0) {
     for (int s = 0; s < kAttnRing; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(s_full_bar(s), 1); mbar_init(s_empty_bar(s), 128); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(s_full_bar(s), 1);
+      mbar_init(s_empty_bar(s), 128);
+      mbar_init(p_ready_bar(s), 128);
+      mbar_init(p_empty_bar(s), 1);
+    }
     mbar_init(q_full_bar, 1);
-    mbar_init(p_ready_bar, 128);
-    mbar_init(p_empty_bar, 1);
     mbar_init(o_full_bar, 1);
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -180,11 +188,12 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                                           j * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        if (!(ok = mbar_wait(p_ready_bar, (uint32_t)t & 1u, abort_flag, a.status))) break;
+        const uint32_t pbuf = (uint32_t)(T + t) & 1u;      // the buffer of the group that owns this tile
+        if (!(ok = mbar_wait(p_ready_bar(pbuf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status))) break;
         tc_fence_after();
         const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
         for (int part = 0; part < 2; ++part) {             // P_hi, then P_lo
-          const uint32_t p_base = base + (part ? kAttnPlo : kAttnPhi);
+          const uint32_t p_base = base + kAttnP + pbuf * kAttnPBytes + part * kSlotBytes;
           for (int g = 0; g < groups; ++g) {               // 16 keys per MMA
             const uint32_t poff = (g >> 2) * kHalfBytes + (g & 3) * 32;
             tc_mma_bf16(tmem_base + 256u, smem_desc_sw128(p_base + poff),
@@ -192,7 +201,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           }
         }
         tc_commit(empty_bar(slot));
-        tc_commit(p_empty_bar);
+        tc_commit(p_empty_bar(pbuf));
         ++it;
       }
       if (ok) tc_commit(o_full_bar);
@@ -204,44 +213,52 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue
+    const int group = (warp - 2) >> 2;                     // takes the jobs of its parity
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;                     // query row inside the block = TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     constexpr float kLog2e = 1.4426950408889634f;
     const float sc = a.scale * kLog2e;                     // logits in units of log2
     float top = extra > 0 ? 0.f : -INFINITY;
-    uint32_t job = 0;
     bool ok = true;
-    for (int t = 0; ok && t < T; ++t, ++job) {             // pass 1: row maxima
-      const uint32_t buf = job & 1u;
-      ok = mbar_wait(s_full_bar(buf), (job >> 1) & 1u, abort_flag, a.status);
+    for (uint32_t job = (uint32_t)group; ok && job < (uint32_t)T; job += 2) {   // pass 1: row maxima
+      const int t = (int)job;
+      ok = mbar_wait(s_full_bar(group), (job >> 1) & 1u, abort_flag, a.status);
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const int valid = n - t * kTileRows;                 // keys of this tile that exist
 #pragma unroll 1
       for (int c0 = 0; c0 < 128; c0 += 32) {
         float v[32];
-        tmem_ld32(lane_addr + buf * 128u + c0, v);
+        tmem_ld32(lane_addr + group * 128u + c0, v);
         tmem_ld_wait();
 #pragma unroll
         for (int c = 0; c < 32; ++c)
           if (c0 + c < valid) top = fmaxf(top, v[c] * sc);
       }
       tc_fence_before();
-      mbar_arrive(s_empty_bar(buf));
+      mbar_arrive(s_empty_bar(group));
     }
-    float sum = extra > 0 ? (float)extra * exp2f(-top) : 0.f;
-    for (int t = 0; ok && t < T; ++t, ++job) {             // pass 2: P and row sums
-      const uint32_t buf = job & 1u;
-      ok = mbar_wait(s_full_bar(buf), (job >> 1) & 1u, abort_flag, a.status);
-      if (ok && t > 0) ok = mbar_wait(p_empty_bar, (uint32_t)(t - 1) & 1u, abort_flag, a.status);
+    // both groups need the maximum over all tiles (reached by all eight warps, aborted or not)
+    xchg[group][r] = top;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    top = fmaxf(xchg[0][r], xchg[1][r]);
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    float sum = (extra > 0 && group == 0) ? (float)extra * exp2f(-top) : 0.f;
+    uint32_t first2 = (uint32_t)T;                         // first pass-2 job of this group's parity
+    if ((first2 & 1u) != (uint32_t)group) ++first2;
+    unsigned char* Pbuf = base_ptr + kAttnP + group * kAttnPBytes;
+    for (uint32_t job = first2; ok && job < 2u * (uint32_t)T; job += 2) {       // pass 2: P and row sums
+      const int t = (int)job - T;
+      ok = mbar_wait(s_full_bar(group), (job >> 1) & 1u, abort_flag, a.status);
+      if (ok && t >= 2) ok = mbar_wait(p_empty_bar(group), (uint32_t)((t >> 1) - 1) & 1u, abort_flag, a.status);
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const int valid = n - t * kTileRows;
 #pragma unroll 1
       for (int c0 = 0; c0 < 128; c0 += 32) {
         float v[32];
-        tmem_ld32(lane_addr + buf * 128u + c0, v);
+        tmem_ld32(lane_addr + group * 128u + c0, v);
         tmem_ld_wait();
 #pragma unroll
         for (int g = 0; g < 4; ++g) {                      // 8 keys -> one 16-byte chunk of P_hi, P_lo
@@ -264,34 +281,40 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           const int key = c0 + g * 8;                      // first key of the chunk inside the tile
           const uint32_t off = (uint32_t)(key >> 6) * kHalfBytes + (uint32_t)r * 128u +
                                ((((uint32_t)(key & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4);
-          *reinterpret_cast<uint4*>(base_ptr + kAttnPhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(base_ptr + kAttnPlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(Pbuf + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(Pbuf + kSlotBytes + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
       }
       tc_fence_before();
-      mbar_arrive(s_empty_bar(buf));
+      mbar_arrive(s_empty_bar(group));
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(p_ready_bar);
+      mbar_arrive(p_ready_bar(group));
     }
-    if (ok) {
-      ok = mbar_wait(o_full_bar, 0, abort_flag, a.status);
-      ok = __all_sync(0xffffffffu, ok);
-    }
-    if (ok) {
-      tc_fence_after();
-      const int row = qb * kTileRows + r;
-      const float inv = sum > 0.f ? 1.f / sum : 0.f;
-      float* out = a.O + ((size_t)p * a.m + row) * 128;
+    // group 1 hands its row sums to group 0, which finishes the rows
+    if (group == 1) xchg[1][r] = sum;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (group == 0) {
+      sum += xchg[1][r];
+      if (ok) {
+        ok = mbar_wait(o_full_bar, 0, abort_flag, a.status);
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (ok) {
+        tc_fence_after();
+        const int row = qb * kTileRows + r;
+        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        float* out = a.O + ((size_t)p * a.m + row) * 128;
 #pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        float v[32];
-        tmem_ld32(lane_addr + 256u + c0, v);
-        tmem_ld_wait();
-        if (row < a.m) {
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          float v[32];
+          tmem_ld32(lane_addr + 256u + c0, v);
+          tmem_ld_wait();
+          if (row < a.m) {
 #pragma unroll
-          for (int c = 0; c < 32; c += 4)
-            *reinterpret_cast<float4*>(out + c0 + c) =
-                make_float4(v[c] * inv, v[c + 1] * inv, v[c + 2] * inv, v[c + 3] * inv);
+            for (int c = 0; c < 32; c += 4)
+              *reinterpret_cast<float4*>(out + c0 + c) =
+                  make_float4(v[c] * inv, v[c + 1] * inv, v[c + 2] * inv, v[c + 3] * inv);
+          }
         }
       }
     }

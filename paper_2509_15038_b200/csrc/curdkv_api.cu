@@ -575,7 +575,7 @@ curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stri
   if (cudaFuncSetAttribute(umma::attention_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            umma::kAttnDynamic) != cudaSuccess)
     return CURDKV_ERR_CUDA;
-  umma::attention_umma_kernel<<<(unsigned)(P * q_blocks), umma::kThreads, umma::kAttnDynamic, stream>>>(
+  umma::attention_umma_kernel<<<(unsigned)(P * q_blocks), umma::kAttnThreads, umma::kAttnDynamic, stream>>>(
       mq, mk, mv, a);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
