@@ -388,6 +388,9 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
     if (P * (int64_t)(budget < desc->n_max ? budget : desc->n_max) > 0x7fffffffLL)
       return CURDKV_ERR_UNSUPPORTED;
     const int min_protected = (int)floor(alpha * (double)budget);
+    if (cudaFuncSetAttribute(select_adaptive_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kAdaptiveDynamic) != cudaSuccess)
+      return CURDKV_ERR_CUDA;
     if (desc->kv_heads > 8 &&
         cudaFuncSetAttribute(select_adaptive_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
                              1) != cudaSuccess)
@@ -395,6 +398,7 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)P);
     cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = kAdaptiveDynamic;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -415,9 +419,9 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
   const size_t row_bytes = (((size_t)desc->n_max + 3) / 4) * sizeof(uint4);
   const size_t stage_bytes = row_bytes <= (size_t)kSelStageBytes ? row_bytes : 0;
   if (cudaFuncSetAttribute(select_fixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kSelStageBytes) != cudaSuccess)
+                           kSelStageBytes + kSelListBytes) != cudaSuccess)
     return CURDKV_ERR_CUDA;
-  select_fixed_kernel<<<(unsigned)P, kSelThreads, stage_bytes, stream>>>(
+  select_fixed_kernel<<<(unsigned)P, kSelThreads, stage_bytes + kSelListBytes, stream>>>(
       scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,
       (int)(stage_bytes / sizeof(uint4)), idx, head_counts, head_offsets);
   if (!launch_ok()) return CURDKV_ERR_CUDA;

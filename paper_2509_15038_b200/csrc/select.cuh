@@ -19,7 +19,13 @@ namespace curdkv {
 namespace cg = cooperative_groups;
 
 constexpr int kSelThreads = 1024;
-constexpr int kSelStageBytes = 192 * 1024;                 // largest row copy kept in shared memory
+constexpr int kSelStageBytes = 144 * 1024;                 // largest row copy kept in shared memory
+// After the leading digit of a cut is known, the keys that share it (a few per cent of a row)
+// are copied with their token index into a list in shared memory; the remaining digits, the
+// tie count and the per-warp totals of the compaction then come from the list instead of from
+// further sweeps over the row.  A list that overflows falls back to sweeping.
+constexpr int kSelListCap = 6144;                          // (key, index) pairs per list
+constexpr int kSelListBytes = kSelListCap * 8;
 constexpr int kMaxAdaptiveHeads = 16;                      // one CTA per head in a cluster
 constexpr uint32_t kForcedKey = 0xffffffffu;
 
@@ -63,7 +69,16 @@ __device__ __forceinline__ uint32_t pass_digit_mask(int pass) { return pass == 2
 struct SelectSmem {
   alignas(16) uint32_t hist[kSelBins];                     // read and cleared as 16-byte vectors
   uint32_t warp_def[32], warp_eq[32];
+  uint32_t seg_def[32], seg_eq[32];                        // per-segment totals of the compaction
   uint32_t digit, remaining, above;
+  uint32_t list_count[2];
+};
+
+struct KeyList {
+  uint2* items;            // (rank key, token index)
+  uint32_t* count;         // entries offered; more than kSelListCap means the list is incomplete
+  __device__ __forceinline__ bool complete() const { return *count <= (uint32_t)kSelListCap; }
+  __device__ __forceinline__ int size() const { return (int)min(*count, (uint32_t)kSelListCap); }
 };
 
 __device__ __forceinline__ void clear_hist(uint32_t* hist) {
@@ -239,49 +254,32 @@ __device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, ui
   run.flush(hist);
 }
 
-// Cut that keeps the `want` largest keys of a row (0 < want <= n).  Whole CTA.
-// With first_hist_ready the leading-digit histogram is already in sm.hist
-// (built by stage_keys).
-__device__ __forceinline__ Cut local_cut(const RowKeys& keys, int want, SelectSmem& sm,
-                                         bool first_hist_ready) {
-  uint32_t prefix = 0, mask = 0, remaining = (uint32_t)want;
-  for (int pass = 0; pass < kSelPasses; ++pass) {
-    if (!(first_hist_ready && pass == 0)) {
-      clear_hist(sm.hist);
-      __syncthreads();
-      digit_histogram(keys, 0xffffffffu, mask, prefix, pass, sm.hist);
-    }
-    __syncthreads();
-    pick_digit(sm.hist, remaining, sm);
-    prefix |= sm.digit << pass_shift(pass);
-    mask |= pass_digit_mask(pass) << pass_shift(pass);
-    remaining = sm.remaining;
-    __syncthreads();
+// Quads of a row are dealt to the 32 warps in contiguous runs ("segments"), so that the kept
+// tokens of warp w precede those of warp w + 1 in token order.
+struct Segments {
+  int per_warp, quads;
+  __device__ __forceinline__ explicit Segments(int quads_) : quads(quads_) {
+    per_warp = (((quads_ + 31) >> 5) + 31) & ~31;          // whole-warp sweeps
   }
-  return Cut{prefix, remaining};
+  __device__ __forceinline__ int begin(int warp) const { return min(warp * per_warp, quads); }
+  __device__ __forceinline__ int end(int warp) const { return min(begin(warp) + per_warp, quads); }
+  __device__ __forceinline__ int of_token(uint32_t j) const { return (int)(j >> 2) / per_warp; }
+};
+
+// flags of the four tokens of a quad: bits 0-3 key above T, bits 4-7 key equal to T
+__device__ __forceinline__ uint32_t classify(const uint4& v, uint32_t T) {
+  return (v.x > T ? 1u : 0u) | (v.y > T ? 2u : 0u) | (v.z > T ? 4u : 0u) | (v.w > T ? 8u : 0u) |
+         (v.x == T ? 16u : 0u) | (v.y == T ? 32u : 0u) | (v.z == T ? 64u : 0u) | (v.w == T ? 128u : 0u);
 }
 
-// Ordered compaction of one row: the tokens whose key is above cut.T and the
-// first cut.eq_take tokens whose key equals cut.T, written to `out` in
-// ascending token order.  Every warp owns a contiguous run of quads; a first
-// sweep counts what each warp keeps, one scan over the warp totals places the
-// warps, a second sweep writes.  Whole CTA, blockDim = 1024.
-__device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Cut& cut, int32_t* out,
-                                                SelectSmem& sm) {
+// Per-segment numbers of keys above / equal to the cut, by sweeping the row.  Whole CTA;
+// the totals land in sm.seg_def / sm.seg_eq (visible after the caller's next barrier).
+__device__ __forceinline__ void count_sweep(const RowKeys& keys, const Cut& cut, SelectSmem& sm) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int quads = keys.quads();
-  const int per_warp = (((quads + 31) >> 5) + 31) & ~31;   // quads per warp, whole warp sweeps
-  const int q_begin = min(warp * per_warp, quads), q_end = min(q_begin + per_warp, quads);
-  const uint32_t T = cut.T;
-
-  // flags of the four tokens of a quad: bits 0-3 key above the cut, bits 4-7 key equal to it
-  auto classify = [&](const uint4& v) -> uint32_t {
-    return (v.x > T ? 1u : 0u) | (v.y > T ? 2u : 0u) | (v.z > T ? 4u : 0u) | (v.w > T ? 8u : 0u) |
-           (v.x == T ? 16u : 0u) | (v.y == T ? 32u : 0u) | (v.z == T ? 64u : 0u) | (v.w == T ? 128u : 0u);
-  };
-
+  const Segments seg(keys.quads());
+  const int q_end = seg.end(warp);
   uint32_t def_cnt = 0, eq_cnt = 0;
-  for (int q0 = q_begin + lane; q0 < q_end; q0 += kSelUnroll * 32) {
+  for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += kSelUnroll * 32) {
     uint4 v[kSelUnroll];
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u)
@@ -289,7 +287,7 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Cut& 
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u) {
       if (q0 + u * 32 < q_end) {
-        const uint32_t f = classify(v[u]);
+        const uint32_t f = classify(v[u], cut.T);
         def_cnt += __popc(f & 15u);
         eq_cnt += __popc(f >> 4);
       }
@@ -300,11 +298,106 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Cut& 
     def_cnt += __shfl_xor_sync(0xffffffffu, def_cnt, o);
     eq_cnt += __shfl_xor_sync(0xffffffffu, eq_cnt, o);
   }
-  if (lane == 0) { sm.warp_def[warp] = def_cnt; sm.warp_eq[warp] = eq_cnt; }
+  if (lane == 0) { sm.seg_def[warp] = def_cnt; sm.seg_eq[warp] = eq_cnt; }
+}
+
+// One sweep over the row once the leading digits are known: counts, per segment, the keys whose
+// leading digit is above `d_cut` (they are kept whatever the rest of the cut turns out to be) and
+// copies the keys with leading digit d_a (and d_b, if use_b) into the lists.  Whole CTA; totals in
+// sm.seg_def (sm.seg_eq is cleared); list counters must be zero on entry.
+__device__ __forceinline__ void collect_sweep(const RowKeys& keys, uint32_t d_cut, uint32_t d_a,
+                                              const KeyList& list_a, bool use_b, uint32_t d_b,
+                                              const KeyList& list_b, SelectSmem& sm) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const Segments seg(keys.quads());
+  const int q_end = seg.end(warp);
+  uint32_t def_cnt = 0;
+  for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += kSelUnroll * 32) {
+    uint4 v[kSelUnroll];
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u)
+      if (q0 + u * 32 < q_end) v[u] = keys.load4(q0 + u * 32);
+#pragma unroll
+    for (int u = 0; u < kSelUnroll; ++u) {
+      if (q0 + u * 32 < q_end) {
+        const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t dgt = k4[i] >> 20;
+          def_cnt += dgt > d_cut ? 1u : 0u;
+          if (dgt == d_a) {
+            const uint32_t at = atomicAdd(list_a.count, 1u);
+            if (at < (uint32_t)kSelListCap) list_a.items[at] = make_uint2(k4[i], 4u * (q0 + u * 32) + i);
+          }
+          if (use_b && dgt == d_b) {
+            const uint32_t at = atomicAdd(list_b.count, 1u);
+            if (at < (uint32_t)kSelListCap) list_b.items[at] = make_uint2(k4[i], 4u * (q0 + u * 32) + i);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) def_cnt += __shfl_xor_sync(0xffffffffu, def_cnt, o);
+  if (lane == 0) { sm.seg_def[warp] = def_cnt; sm.seg_eq[warp] = 0; }
+}
+
+// digit_histogram over a (complete) list instead of the row.
+__device__ __forceinline__ void list_histogram(const KeyList& list, uint32_t ceiling, uint32_t mask,
+                                               uint32_t prefix, int pass, uint32_t* hist) {
+  const int shift = pass_shift(pass), n = list.size();
+  const uint32_t dmask = pass_digit_mask(pass);
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const uint32_t key = list.items[e].x;
+    if ((key & mask) == prefix && key <= ceiling) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+  }
+}
+
+// Adds the list's keys above / equal to the cut to the per-segment totals (the list holds every
+// key whose leading digit equals the cut's; keys with a higher digit were counted by collect_sweep).
+__device__ __forceinline__ void count_from_list(const KeyList& list, const Cut& cut, const Segments& seg,
+                                                SelectSmem& sm) {
+  const int n = list.size();
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const uint2 it = list.items[e];
+    if (it.x > cut.T) atomicAdd(&sm.seg_def[seg.of_token(it.y)], 1u);
+    else if (it.x == cut.T) atomicAdd(&sm.seg_eq[seg.of_token(it.y)], 1u);
+  }
+}
+
+// Remaining digits of a cut whose leading digit `d0` is known: the `rank`-th largest key (1-based)
+// among the keys of leading digit d0.  Uses the list if it is complete, else sweeps the row.  Whole CTA.
+__device__ __forceinline__ Cut finish_cut(const RowKeys& keys, const KeyList& list, uint32_t d0,
+                                          uint32_t rank, SelectSmem& sm) {
+  uint32_t prefix = d0 << 20, mask = 0xfffu << 20, remaining = rank;
+  const bool from_list = list.complete();
+  for (int pass = 1; pass < kSelPasses; ++pass) {
+    clear_hist(sm.hist);
+    __syncthreads();
+    if (from_list) list_histogram(list, 0xffffffffu, mask, prefix, pass, sm.hist);
+    else digit_histogram(keys, 0xffffffffu, mask, prefix, pass, sm.hist);
+    __syncthreads();
+    pick_digit(sm.hist, remaining, sm);
+    prefix |= sm.digit << pass_shift(pass);
+    mask |= pass_digit_mask(pass) << pass_shift(pass);
+    remaining = sm.remaining;
+    __syncthreads();
+  }
+  return Cut{prefix, remaining};
+}
+
+// Ordered write of one row: the tokens whose key is above cut.T and the first cut.eq_take tokens
+// whose key equals cut.T go to `out` in ascending token order.  The per-segment totals must be in
+// sm.seg_def / sm.seg_eq (from count_sweep, or collect_sweep + count_from_list).  Whole CTA.
+__device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut, int32_t* out,
+                                            SelectSmem& sm) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const Segments seg(keys.quads());
+  const int q_begin = seg.begin(warp), q_end = seg.end(warp);
   __syncthreads();
   uint32_t def_before = 0, eq_before = 0;                  // kept / equal tokens of earlier warps
   {
-    const uint32_t d = sm.warp_def[lane], e = sm.warp_eq[lane];
+    const uint32_t d = sm.seg_def[lane], e = sm.seg_eq[lane];
     uint32_t di = d, ei = e;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -314,11 +407,10 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Cut& 
     def_before = __shfl_sync(0xffffffffu, di - d, warp);
     eq_before = __shfl_sync(0xffffffffu, ei - e, warp);
   }
-
   for (int q0 = q_begin; q0 < q_end; q0 += 32) {           // uniform trip count across the warp
     const int q = q0 + lane;
     uint32_t f = 0;
-    if (q < q_end) f = classify(keys.load4(q));
+    if (q < q_end) f = classify(keys.load4(q), cut.T);
     const uint32_t mine = (uint32_t)__popc(f & 15u) | ((uint32_t)__popc(f >> 4) << 16);
     uint32_t inc = mine;
 #pragma unroll
@@ -348,7 +440,8 @@ __device__ __forceinline__ void ordered_compact(const RowKeys& keys, const Cut& 
 
 // ---------------------------------------------------------------------------
 // Fixed per-head budget.  grid = batch*heads, block = 1024, dynamic shared
-// memory = 16 * stage_quads bytes (0: rows are read from global memory).
+// memory = 16 * stage_quads bytes (0: rows are read from global memory) followed
+// by one candidate list (kSelListBytes).
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
@@ -366,6 +459,7 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
   int32_t* out = idx + (size_t)p * budget;
 
   Cut cut;
+  bool counted = false;                                    // per-segment totals already in sm.warp_*
   if (k_eff == 0) {
     cut = keep_nothing();
   } else if (k_eff == n) {
@@ -373,17 +467,32 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
   } else if (F.free_slots == 0) {
     cut = keep_forced_only();
   } else {
-    const bool stage = keys.quads() <= stage_quads;        // the row fits in shared memory
-    if (stage) {
-      clear_hist(sm.hist);
-      __syncthreads();
+    // sweep 1: leading-digit histogram (staging the keys on the way if the row fits)
+    clear_hist(sm.hist);
+    if (tid == 0) sm.list_count[0] = 0;
+    __syncthreads();
+    if (keys.quads() <= stage_quads) {
       stage_keys(keys, staged_keys, sm.hist);
       keys.staged = staged_keys;
+    } else {
+      digit_histogram(keys, 0xffffffffu, 0u, 0u, 0, sm.hist);
     }
-    cut = local_cut(keys, k_eff, sm, stage);
+    __syncthreads();
+    pick_digit(sm.hist, (uint32_t)k_eff, sm);
+    const uint32_t d0 = sm.digit, rank = sm.remaining;
+    __syncthreads();
+    // sweep 2: keys above the digit are counted per segment, keys of the digit go to the list
+    const KeyList list{reinterpret_cast<uint2*>(staged_keys + stage_quads), &sm.list_count[0]};
+    collect_sweep(keys, d0, d0, list, false, 0u, list, sm);
+    __syncthreads();
+    cut = finish_cut(keys, list, d0, rank, sm);
+    if (list.complete()) {
+      count_from_list(list, cut, Segments(keys.quads()), sm);
+      counted = true;
+    }
   }
-
-  ordered_compact(keys, cut, out, sm);
+  if (!counted) count_sweep(keys, cut, sm);
+  write_sweep(keys, cut, out, sm);
   for (int t = k_eff + tid; t < budget; t += kSelThreads) out[t] = -1;
   if (tid == 0) {
     counts[p] = k_eff;
@@ -409,12 +518,17 @@ struct AdaptiveSmem {
   uint32_t pub_eq;                                         // unprotected keys equal to the global cut
   uint32_t pub_count;                                      // rows this head keeps
 };
+constexpr int kAdaptiveDynamic = kSelBins * 4 + 2 * kSelListBytes;   // leading-digit histogram + two lists
 
 __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
     const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
     int budget, int num_sink, int window, int min_protected, int32_t* __restrict__ idx,
     int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   __shared__ AdaptiveSmem sm;
+  extern __shared__ uint4 adaptive_dyn[];
+  uint32_t* hist_all = reinterpret_cast<uint32_t*>(adaptive_dyn);          // leading digits of all keys
+  const KeyList list_a{reinterpret_cast<uint2*>(hist_all + kSelBins), &sm.s.list_count[0]};
+  const KeyList list_b{list_a.items + kSelListCap, &sm.s.list_count[1]};
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x;
   const int h = (int)cluster.block_rank();
@@ -425,31 +539,95 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   const RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
   const int forced = k_eff - F.free_slots;
   const int prot = min(max(min_protected, forced), k_eff);  // protected rows per head, forced included
+  const bool none = prot == 0, all = prot >= n;             // nothing / everything is protected
+  const uint32_t pool = (uint32_t)heads * (uint32_t)(k_eff - prot);   // same for every head of b
 
-  // ---- this head's safeguard share: its `prot` largest keys
+  // ---- sweep 1: leading-digit histogram of the row; leading digit of this head's safeguard cut
+  // (its `prot` largest keys) and how many keys of that digit the cut takes
+  clear_hist(hist_all);
+  if (tid == 0) sm.s.list_count[0] = sm.s.list_count[1] = 0;
+  __syncthreads();
+  if (!all) digit_histogram(keys, 0xffffffffu, 0u, 0u, 0, hist_all);
+  __syncthreads();
+  uint32_t d0 = 0xffffffffu, rank_own = 0;
+  if (!none && !all) {
+    pick_digit(hist_all, (uint32_t)prot, sm.s);
+    d0 = sm.s.digit;
+    rank_own = sm.s.remaining;
+    __syncthreads();
+  }
+
+  // ---- leading digit of the layer-wide cut over the unprotected keys of all heads.  Their
+  // leading-digit histogram follows from the row's: bins below d0 whole, bin d0 minus the
+  // protected keys in it, nothing above.
+  uint32_t dg = 0, remaining = pool, local_gt = 0, local_eq = 0;
+  if (pool > 0) {
+    {
+      const uint4 v = reinterpret_cast<const uint4*>(hist_all)[tid];
+      uint32_t c[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t bin = (uint32_t)(4 * tid + u);
+        if (all) c[u] = 0;
+        else if (!none && bin > d0) c[u] = 0;
+        else if (!none && bin == d0) c[u] -= rank_own;
+      }
+      reinterpret_cast<uint4*>(sm.hist_local)[tid] = make_uint4(c[0], c[1], c[2], c[3]);
+    }
+    cluster.sync();
+    {
+      uint4 acc = make_uint4(0u, 0u, 0u, 0u);              // this thread's four bins over all heads
+      for (int r = 0; r < heads; ++r) {
+        const uint4 v = reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      reinterpret_cast<uint4*>(sm.s.hist)[tid] = acc;
+    }
+    __syncthreads();
+    pick_digit(sm.s.hist, remaining, sm.s);
+    dg = sm.s.digit;
+    remaining = sm.s.remaining;
+    local_gt = count_above(sm.hist_local, dg, sm.s);
+    cluster.sync();                                        // peers are done reading hist_local
+  }
+
+  // ---- sweep 2: keys with a leading digit above the final cut's are kept for sure (counted per
+  // segment); keys with the digits d0 and dg go to the lists
+  // (the layer-wide cut can lie above this head's own cut when other heads score higher: then
+  // this head keeps its protected keys only and its final cut is its own)
+  const bool global_lower = pool > 0 && (none || dg < d0); // the final cut has leading digit dg
+  const uint32_t d_cut = global_lower ? dg : d0;
+  const bool share = !none && dg == d0;                    // one list serves both cuts
+  const bool swept = !all && (pool > 0 || !none);
+  if (swept) collect_sweep(keys, d_cut, d0, list_a, pool > 0 && !share, dg, list_b, sm.s);
+  __syncthreads();
+
+  // ---- this head's safeguard cut
   Cut own = keep_nothing();
-  if (prot >= n) own = keep_every_token();
-  else if (prot > 0 && prot == forced) own = Cut{kForcedKey, (uint32_t)forced};
-  else if (prot > 0) own = local_cut(keys, prot, sm.s, false);
+  if (all) own = keep_every_token();
+  else if (!none) own = finish_cut(keys, list_a, d0, rank_own, sm.s);
   // unprotected keys: those <= own.T, minus the first own.eq_take equal to it
   const uint32_t ceiling = own.T;
 
-  // ---- layer-wide cut over the unprotected keys of all heads
-  const uint32_t pool = (uint32_t)heads * (uint32_t)(k_eff - prot);
-  uint32_t Tg = 0, eq_g = 0, local_gt = 0, local_eq = 0;
+  // ---- remaining digits of the layer-wide cut
+  const KeyList& list_g = share ? list_a : list_b;
+  uint32_t Tg = 0, eq_g = 0;
   if (pool > 0) {
-    uint32_t prefix = 0, mask = 0, remaining = pool;
-    for (int pass = 0; pass < kSelPasses; ++pass) {
+    uint32_t prefix = dg << 20, mask = 0xfffu << 20;
+    for (int pass = 1; pass < kSelPasses; ++pass) {
       const int shift = pass_shift(pass);
       clear_hist(sm.hist_local);
       __syncthreads();
-      digit_histogram(keys, ceiling, mask, prefix, pass, sm.hist_local);
+      if (!all) {
+        if (list_g.complete()) list_histogram(list_g, ceiling, mask, prefix, pass, sm.hist_local);
+        else digit_histogram(keys, ceiling, mask, prefix, pass, sm.hist_local);
+      }
       __syncthreads();
       if (tid == 0 && own.eq_take > 0 && (own.T & mask) == prefix)
         sm.hist_local[(own.T >> shift) & pass_digit_mask(pass)] -= own.eq_take;   // those are protected
       cluster.sync();
       {
-        uint4 acc = make_uint4(0u, 0u, 0u, 0u);            // this thread's four bins over all heads
+        uint4 acc = make_uint4(0u, 0u, 0u, 0u);
         for (int r = 0; r < heads; ++r) {
           const uint4 v = reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid];
           acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
@@ -499,7 +677,11 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   for (int r = 0; r < h; ++r) off += *cluster.map_shared_rank(&sm.pub_count, r);
   __syncthreads();
 
-  ordered_compact(keys, cut, idx + off, sm.s);
+  // ---- per-segment totals, then the ordered write (sweep 3)
+  const KeyList& list_c = global_lower ? list_b : list_a;  // holds the keys of the cut's leading digit
+  if (swept && list_c.complete()) count_from_list(list_c, cut, Segments(keys.quads()), sm.s);
+  else count_sweep(keys, cut, sm.s);
+  write_sweep(keys, cut, idx + off, sm.s);
   if (tid == 0) {
     counts[p] = (int32_t)kept;
     offsets[p] = (int32_t)off;
