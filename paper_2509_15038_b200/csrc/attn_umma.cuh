@@ -43,6 +43,21 @@ constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O
 // P V: A = P K-major, B = V tile MN-major (contraction over the keys)
 __host__ __device__ constexpr uint32_t instr_desc_pv() { return instr_desc_bf16(128) | (1u << 16); }
 
+// 2^x, relative error ~2^-22 (the weights are rounded to bf16 pairs afterwards)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Two weights -> packed bf16 (hi) and packed bf16 of the remainders (lo).
+__device__ __forceinline__ void split_bf16x2(float w0, float w1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  const float r0 = w0 - __uint_as_float(hi << 16), r1 = w1 - __uint_as_float(hi & 0xffff0000u);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(r0, r1);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v, const AttnArgs a) {
@@ -232,9 +247,14 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         float v[32];
         tmem_ld32(lane_addr + group * 128u + c0, v);
         tmem_ld_wait();
+        if (valid >= kTileRows) {                          // full tile: no masking
 #pragma unroll
-        for (int c = 0; c < 32; ++c)
-          if (c0 + c < valid) top = fmaxf(top, v[c] * sc);
+          for (int c = 0; c < 32; ++c) top = fmaxf(top, v[c] * sc);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (c0 + c < valid) top = fmaxf(top, v[c] * sc);
+        }
       }
       tc_fence_before();
       mbar_arrive(s_empty_bar(group));
@@ -265,18 +285,14 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           uint32_t hi[4], lo[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float w[2];
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              const int c = g * 8 + e * 2 + q;
-              w[q] = c0 + c < valid ? exp2f(v[c] * sc - top) : 0.f;
+            const int c = g * 8 + e * 2;
+            float w0 = fast_exp2(fmaf(v[c], sc, -top)), w1 = fast_exp2(fmaf(v[c + 1], sc, -top));
+            if (valid < kTileRows) {                       // last tile of the cache: mask by index
+              if (c0 + c >= valid) w0 = 0.f;
+              if (c0 + c + 1 >= valid) w1 = 0.f;
             }
-            const __nv_bfloat16 h0 = __float2bfloat16_rn(w[0]), h1 = __float2bfloat16_rn(w[1]);
-            const __nv_bfloat16 l0 = __float2bfloat16_rn(w[0] - __bfloat162float(h0));
-            const __nv_bfloat16 l1 = __float2bfloat16_rn(w[1] - __bfloat162float(h1));
-            sum += (__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1));
-            hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-            lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            sum += w0 + w1;                                // equals the bf16 pairs to 2^-17
+            split_bf16x2(w0, w1, hi[e], lo[e]);
           }
           const int key = c0 + g * 8;                      // first key of the chunk inside the tile
           const uint32_t off = (uint32_t)(key >> 6) * kHalfBytes + (uint32_t)r * 128u +
