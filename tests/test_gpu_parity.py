@@ -193,6 +193,25 @@ def test_select_long_rows():
     _select_case(sc, 6681, 4, 0)
 
 
+def test_select_candidate_list_overflow_falls_back_to_sweeps():
+    """Scores that share their leading 12 bits put more keys into the cut's digit than the
+    shared-memory candidate list holds: fixed and adaptive selection must still be exact, ties included."""
+    rng = np.random.default_rng(12)
+    B, H, n = 2, 4, 20000
+    near = (1.0 + rng.random((B, H, n)) * 2.0 ** -13).astype(np.float32)       # one leading digit for all
+    _select_case(near, 3000, 4, 64)
+    _select_case(near, 19000, 0, 0)
+    coarse = (1.0 + np.floor(rng.random((B, H, n)) * 4) * 2.0 ** -20).astype(np.float32)   # four values: ties
+    _select_case(coarse, 7000, 2, 10)
+    _adaptive_case(near, 3000, 4, 64, 0.2)
+    _adaptive_case(coarse, 7000, 2, 10, 0.5)
+    mixed = near.copy()
+    mixed[:, ::2] *= 3.0                                    # heads on different leading digits
+    _adaptive_case(mixed, 5000, 0, 32, 0.1)
+    long_rows = (1.0 + rng.random((1, 2, 60000)) * 2.0 ** -13).astype(np.float32)  # beyond the staged size
+    _select_case(long_rows, 9000, 4, 128)
+
+
 def test_compact_flags_bad_index_without_faulting():
     B, H, n, d = 1, 2, 64, 128
     K = torch.randn((B, H, n, d), device=DEV).to(torch.bfloat16)
