@@ -407,19 +407,28 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
     def_before = __shfl_sync(0xffffffffu, di - d, warp);
     eq_before = __shfl_sync(0xffffffffu, ei - e, warp);
   }
+  const uint32_t lt = (1u << lane) - 1u;                   // lanes before this one
   for (int q0 = q_begin; q0 < q_end; q0 += 32) {           // uniform trip count across the warp
     const int q = q0 + lane;
     uint32_t f = 0;
     if (q < q_end) f = classify(keys.load4(q), cut.T);
-    const uint32_t mine = (uint32_t)__popc(f & 15u) | ((uint32_t)__popc(f >> 4) << 16);
-    uint32_t inc = mine;
+    // tokens run lane-major, then by position in the quad: ranks from one ballot per flag bit
+    uint32_t d = def_before, dtot = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t bal = __ballot_sync(0xffffffffu, f & (1u << i));
+      d += __popc(bal & lt);
+      dtot += __popc(bal);
     }
-    const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
-    uint32_t d = def_before + ((inc - mine) & 0xffffu), e = eq_before + ((inc - mine) >> 16);
+    uint32_t e = eq_before, etot = 0;
+    if (__any_sync(0xffffffffu, f >> 4)) {                 // ties at the cut are rare
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t bal = __ballot_sync(0xffffffffu, f & (16u << i));
+        e += __popc(bal & lt);
+        etot += __popc(bal);
+      }
+    }
     if (f) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -432,8 +441,8 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
         }
       }
     }
-    def_before += total & 0xffffu;
-    eq_before += total >> 16;
+    def_before += dtot;
+    eq_before += etot;
   }
   __syncthreads();                                         // sm.warp_* may be reused
 }
