@@ -290,8 +290,8 @@ curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, 
  * handles (passed as void*, either may be NULL) on its stream immediately
  * before and after its sketch kernel -- the kernel that streams K and V -- so
  * that a benchmark can time that kernel alone without a profiler.  The request
- * is cleared by that call.  With projection off, per-head G or n_max < 128 the
- * sketch runs on another kernel and nothing is recorded. */
+ * is cleared by that call.  With projection off or n_max < 128 the scores come
+ * from a plain streaming kernel and nothing is recorded. */
 curdkv_status curdkv_profile_next_score(void* start_event, void* stop_event);
 
 /* Number of kernels this library has launched in this process so far. */

@@ -259,6 +259,7 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
     u.status = static_cast<uint32_t*>(workspace);
     u.partials = reinterpret_cast<float*>(ws + L.partials);
     u.W = reinterpret_cast<const float*>(ws + L.W);
+    u.w_per_problem = u.w_per_tensor = 1;
     u.r = desc->r;
     u.tiles_per_head = tiles;
     u.score_mode = desc->score_mode;
@@ -305,6 +306,50 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
     if (!launch_ok()) return CURDKV_ERR_CUDA;
     parts = umma::kPartsPerTile;
     launched = true;
+  } else if (desc->use_projection && g_per_head && desc->n_max >= kTileRows) {
+    // one G per KV head: the item-walking sketch kernel with the head's G staged per item
+    CUtensorMap mk, mv;
+    if (make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) &&
+        make_tile_map(&mv, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n)) {
+      umma::ItemArgs u;
+      u.seqlens = desc->seqlens;
+      u.batch = desc->batch;
+      u.heads = desc->kv_heads;
+      u.n_max = desc->n_max;
+      u.segments = whiten_segments(desc);
+      u.status = static_cast<uint32_t*>(workspace);
+      u.partials = nullptr;
+      u.W = G;
+      u.w_per_problem = u.w_per_tensor = 0;
+      u.r = desc->r;
+      u.tiles_per_head = tiles;
+      u.score_mode = desc->score_mode;
+      u.scores = scores;
+      u.tile_sums = a.tile_sums;
+      const int sms = sm_count();
+      if (sms <= 0) return CURDKV_ERR_CUDA;
+      const int64_t items = P * u.segments;
+      const unsigned grid_items = (unsigned)(items < sms ? items : sms);
+      if (g_profile_start != nullptr) cudaEventRecord(g_profile_start, stream);
+      if (desc->r <= 32) {
+        using S = umma::ItemSmem<32>;
+        if (cudaFuncSetAttribute(umma::sketch_items_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 S::kDynamic) != cudaSuccess)
+          return CURDKV_ERR_CUDA;
+        umma::sketch_items_kernel<32><<<grid_items, umma::kThreads, S::kDynamic, stream>>>(mk, mv, u);
+      } else {
+        using S = umma::ItemSmem<64>;
+        if (cudaFuncSetAttribute(umma::sketch_items_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 S::kDynamic) != cudaSuccess)
+          return CURDKV_ERR_CUDA;
+        umma::sketch_items_kernel<64><<<grid_items, umma::kThreads, S::kDynamic, stream>>>(mk, mv, u);
+      }
+      if (g_profile_stop != nullptr) cudaEventRecord(g_profile_stop, stream);
+      if (!launch_ok()) return CURDKV_ERR_CUDA;
+      parts = umma::kPartsPerTile;
+      launched = true;
+    }
+    g_profile_start = g_profile_stop = nullptr;
   } else if (desc->use_projection && !g_per_head && desc->n_max >= kTileRows) {
     // tensor-core path: one G for all heads, TMA tiles of 128 rows.  A ragged batch goes in
     // slices of at most kMaxRaggedBatch sequences (the kernel keeps their tile prefix sums

@@ -24,7 +24,10 @@ struct ItemArgs {
   // gram kernel
   float* partials;         // [batch*heads*segments][2][128][128]
   // sketch kernel
-  const float* W;          // [batch*heads][2][128][r]
+  const float* W;          // projections, fp32 [128][r] each:
+                           //   whitened: [batch*heads][2 tensors]   (w_per_problem = 1, w_per_tensor = 1)
+                           //   per-head G: [heads], shared by K, V  (w_per_problem = 0, w_per_tensor = 0)
+  int w_per_problem, w_per_tensor;
   int r, tiles_per_head, score_mode;
   float* scores;
   float* tile_sums;        // [batch*heads][tiles_per_head][kPartsPerTile]
@@ -230,8 +233,9 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------
-// Sketch + norms + combine (Alg. 1 lines 2-5) with a per-head, per-tensor
-// projection W instead of the shared G.  Same pipeline as sketch_umma_kernel;
+// Sketch + norms + combine (Alg. 1 lines 2-5) with a projection that changes
+// from head to head (the whitened W of each head and tensor, or a caller's
+// per-head G) instead of one shared G.  Same pipeline as sketch_umma_kernel;
 // the epilogue warps restage [W_hi | W_lo] for K and for V at the start of
 // every item and release the MMA issuer through g_ready.
 // ---------------------------------------------------------------------------
@@ -378,7 +382,9 @@ sketch_items_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       // every MMA of the previous item has retired (its last accumulator was handed over), so
       // the staged projections can be replaced: W^T = [W_hi | W_lo], swizzled K-major, per tensor
       for (int tensor = 0; tensor < 2; ++tensor) {
-        const float* Wp = a.W + ((size_t)w.p * 2 + tensor) * 128 * a.r;
+        const size_t which = (size_t)(a.w_per_problem ? w.p : w.p % a.heads) * (a.w_per_tensor ? 2 : 1) +
+                             (a.w_per_tensor ? tensor : 0);
+        const float* Wp = a.W + which * 128 * a.r;
         unsigned char* dstG = base_ptr + (tensor ? L::kGV : L::kGK);
         for (int i = etid; i < 128 * R; i += 128) {
           const int t = i / R, c = i % R;
