@@ -124,6 +124,26 @@ def test_eviction_loss_of_a_curdkv_selection(adaptive):
     assert float(same.max()) == 0.0
 
 
+def test_attention_tiny_and_odd_shapes():
+    """One query, one key; 129 queries (two blocks, the second almost empty) over 257 keys."""
+    g = torch.Generator(device=DEV).manual_seed(8)
+    for m, n in ((1, 1), (129, 257), (128, 128)):
+        K = torch.randn((1, 1, n, 128), generator=g, device=DEV).to(torch.bfloat16)
+        V = torch.randn((1, 1, n, 128), generator=g, device=DEV).to(torch.bfloat16)
+        Q = _queries(1, 1, m, 128, seed=m)
+        if n < 128:                       # the tiled loads want at least one full tile of allocation
+            Kp = torch.zeros((1, 1, 128, 128), dtype=torch.bfloat16, device=DEV)
+            Vp = torch.zeros_like(Kp)
+            Kp[:, :, :n], Vp[:, :, :n] = K, V
+            desc = cur.make_desc(Kp, Vp, 32, seqlens=torch.tensor([n], dtype=torch.int32, device=DEV))
+            O, ws = cur.curdkv_attention_out(Q, Kp, Vp, desc, scale=0.2)
+        else:
+            desc = cur.make_desc(K, V, 32)
+            O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=0.2)
+        assert cur.curdkv_device_status(ws) == 0
+        _check_out(O, Q, K, V, np.full((1, 1), n), 0.2, what=f"m={m} n={n}")
+
+
 def test_attention_rejects_bad_arguments():
     K = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device=DEV)
     Q = torch.zeros((1, 1, 16, 64), dtype=torch.bfloat16, device=DEV)

@@ -65,6 +65,13 @@ def test_whitened_long_rows_and_selection():
     assert (i0 != idx).any()
 
 
+def test_whitened_full_length_rows_r64():
+    """Rows as long as the benchmark's (32768 tokens: many tiles per segment), 64 sketch columns."""
+    w = synth.shrink(synth.CONFIGS["cfg3"], layers=1, batch=1, kv_heads=2, q_heads=2)
+    K, V, _ = synth.make_kv(w, DEV)
+    _check(K, V, synth.make_G(w.d, 64, seed=2), 1e-4, what="n=32768 r=64")
+
+
 def test_whitened_ragged_and_odd_lengths():
     w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=5, n_max=1000, kv_heads=2, q_heads=2)
     K, V, _ = synth.make_kv(w, DEV)
