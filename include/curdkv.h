@@ -280,6 +280,14 @@ curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compresse
  * the shared selection without replicating the compacted cache. */
 curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, void* cuda_stream);
 
+/* Optional expansion of a fixed-layout selection to the query heads (Sec. 3.2: the heads of a
+ * GQA group share the keys and values of their group, hence its selection):
+ *   idx_q[b][q][:] = idx[b][q / (q_heads / kv_heads)][:], counts_q[b][q] likewise.
+ * idx int32 [batch][kv_heads][budget], idx_q int32 [batch][q_heads][budget],
+ * counts_q int32 [batch][q_heads].  The compacted cache itself is never replicated. */
+curdkv_status curdkv_gqa_expand(const curdkv_desc* desc, const int32_t* idx, const int32_t* head_counts,
+                                int32_t budget, int32_t* idx_q, int32_t* counts_q, void* cuda_stream);
+
 /* Copies the device status word to *host_flags (host pointer) after
  * synchronising the stream.  Returns CURDKV_ERR_TIMEOUT if the timeout bit is
  * set, CURDKV_OK otherwise (other bits are reported through *host_flags). */

@@ -26,7 +26,7 @@ EXPORTS = (
     "curdkv_score_static", "curdkv_host_arena_bytes", "curdkv_compress_host",
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
     "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
-    "curdkv_eviction_loss",
+    "curdkv_eviction_loss", "curdkv_gqa_expand",
 )
 
 
@@ -89,6 +89,8 @@ def load():
                                          ctypes.POINTER(ctypes.c_uint32)]
     lib.curdkv_gqa_map.restype = ctypes.c_int
     lib.curdkv_gqa_map.argtypes = [dp, vp, vp]
+    lib.curdkv_gqa_expand.restype = ctypes.c_int
+    lib.curdkv_gqa_expand.argtypes = [dp, vp, vp, i32, vp, vp, vp]
     lib.curdkv_device_status.restype = ctypes.c_int
     lib.curdkv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     cp = ctypes.POINTER(Cache)
@@ -380,6 +382,16 @@ def curdkv_gqa_map(desc: Desc, device="cuda") -> torch.Tensor:
     out = torch.empty((desc.q_heads,), dtype=torch.int32, device=device)
     _check(load().curdkv_gqa_map(ctypes.byref(desc), _ptr(out), _stream()), "curdkv_gqa_map")
     return out
+
+
+def curdkv_gqa_expand(desc: Desc, idx: torch.Tensor, head_counts: torch.Tensor):
+    """Per-query-head copies of a fixed-layout selection: (idx_q [B, Hq, budget], counts_q [B, Hq])."""
+    budget = idx.shape[-1]
+    idx_q = torch.empty((desc.batch, desc.q_heads, budget), dtype=torch.int32, device=idx.device)
+    counts_q = torch.empty((desc.batch, desc.q_heads), dtype=torch.int32, device=idx.device)
+    _check(load().curdkv_gqa_expand(ctypes.byref(desc), _ptr(idx), _ptr(head_counts), budget, _ptr(idx_q),
+                                    _ptr(counts_q), _stream()), "curdkv_gqa_expand")
+    return idx_q, counts_q
 
 
 def curdkv_device_status(workspace: torch.Tensor) -> int:

@@ -69,4 +69,18 @@ __global__ void gqa_map_kernel(int32_t* kv_head_of_q, int q_heads, int kv_heads)
   if (q < q_heads) kv_head_of_q[q] = q / (q_heads / kv_heads);
 }
 
+// Per-query-head copy of a fixed-layout selection: query head q of sequence b gets the indices
+// and the count of its KV head (for attention code that wants one index list per query head).
+// grid = batch*q_heads, block = 256.
+__global__ void __launch_bounds__(256) gqa_expand_kernel(const int32_t* idx, const int32_t* counts,
+                                                         int q_heads, int kv_heads, int budget,
+                                                         int32_t* idx_q, int32_t* counts_q) {
+  const int b = blockIdx.x / q_heads, q = blockIdx.x % q_heads;
+  const int h = q / (q_heads / kv_heads);
+  const int32_t* src = idx + ((size_t)b * kv_heads + h) * budget;
+  int32_t* dst = idx_q + (size_t)blockIdx.x * budget;
+  for (int t = threadIdx.x; t < budget; t += blockDim.x) dst[t] = src[t];
+  if (threadIdx.x == 0) counts_q[blockIdx.x] = counts[b * kv_heads + h];
+}
+
 }  // namespace curdkv

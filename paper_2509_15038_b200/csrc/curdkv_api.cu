@@ -527,6 +527,21 @@ curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, voi
   return CURDKV_OK;
 }
 
+curdkv_status curdkv_gqa_expand(const curdkv_desc* desc, const int32_t* idx, const int32_t* head_counts,
+                                int32_t budget, int32_t* idx_q, int32_t* counts_q, void* cuda_stream) {
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if (idx == nullptr || head_counts == nullptr || idx_q == nullptr || counts_q == nullptr || budget < 0)
+    return CURDKV_ERR_INVALID_ARG;
+  const int64_t blocks = (int64_t)desc->batch * desc->q_heads;
+  if (blocks == 0) return CURDKV_OK;
+  if (blocks > 0x7fffffffLL) return CURDKV_ERR_UNSUPPORTED;
+  gqa_expand_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      idx, head_counts, desc->q_heads, desc->kv_heads, budget, idx_q, counts_q);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
 curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, void* cuda_stream) {
   if (workspace == nullptr || host_flags == nullptr) return CURDKV_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -266,6 +266,12 @@ def test_determinism_and_gqa_map():
         assert torch.equal(a, b)
     m = cur.curdkv_gqa_map(desc).cpu().tolist()
     assert m == [orc.kv_head_of_query(q, w.q_heads, w.kv_heads) for q in range(w.q_heads)]
+    idx_q, cnt_q = cur.curdkv_gqa_expand(desc, idx, cnt)
+    gi, gq = idx.cpu().numpy(), idx_q.cpu().numpy()
+    for q in range(w.q_heads):
+        h = orc.kv_head_of_query(q, w.q_heads, w.kv_heads)
+        np.testing.assert_array_equal(gq[:, q], gi[:, h])
+        np.testing.assert_array_equal(cnt_q.cpu().numpy()[:, q], cnt.cpu().numpy()[:, h])
 
 
 # ---------------------------------------------------------------- AdaCurDKV
