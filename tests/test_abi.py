@@ -34,3 +34,32 @@ def test_host_only_calls_work_without_a_device():
     bad = binding.Desc(4, 8, 12, 1000, 128, 32, 0, 0, 128, 0, 0, 128, None, 0, 1)
     assert binding.workspace_bytes(bad) == 0
     assert lib.curdkv_score(None, None, None, 0, None, None, None, None, 0, None) == 1
+
+
+def test_workspace_sizes_of_the_added_modes_without_a_device():
+    lib = binding.load()
+    plain = binding.Desc(4, 8, 32, 1000, 128, 32, 0, 0, 128, 0, 0, 128, None, 0, 1)
+    white = binding.Desc(4, 8, 32, 1000, 128, 32, 0, 0, 128, 0, 0, 128, None, 0, 1, 0, 1, 1e-4)
+    base = binding.workspace_bytes(plain)
+    # whitened: + one partial Gram pair (2 x 128 x 128 fp32) per (head, segment) + W (2 x 128 x r fp32) per head
+    extra = binding.workspace_bytes(white) - base
+    heads = 4 * 8
+    assert extra >= heads * 2 * 128 * 128 * 4 + heads * 2 * 128 * 32 * 4
+    assert extra % (2 * 128 * 128 * 4) % 256 == 0
+    bad_ridge = binding.Desc(4, 8, 32, 1000, 128, 32, 0, 0, 128, 0, 0, 128, None, 0, 1, 0, 1, -1.0)
+    assert binding.workspace_bytes(bad_ridge) == 0
+    # generation-phase cache: grows with rows appended per call and with the budget
+    small = lib.curdkv_cache_workspace_bytes(4, 8, 16, 512, 256)
+    assert small > 0
+    assert lib.curdkv_cache_workspace_bytes(4, 8, 256, 512, 256) > small
+    assert lib.curdkv_cache_workspace_bytes(4, 8, 16, 512, 400) > small
+    assert lib.curdkv_cache_workspace_bytes(4, 0, 16, 512, 256) == 0
+    # evaluator: status words + one int32 per head
+    import ctypes as ct
+    assert lib.curdkv_attention_workspace_bytes(ct.byref(plain)) == 256 + 256
+    # calls with NULL arguments are refused on the host, nothing is launched
+    before = binding.launch_count()
+    assert lib.curdkv_cache_compress(None, None, None, 1, 0, 0, None, 0, None) == 1
+    assert lib.curdkv_eviction_loss(None, None, 1, 1, None, None, None) == 1
+    assert lib.curdkv_gqa_expand(None, None, None, 1, None, None, None) == 1
+    assert binding.launch_count() == before
