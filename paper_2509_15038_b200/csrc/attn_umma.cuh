@@ -3,17 +3,20 @@
 // the eviction-loss evaluator; not a serving kernel (no causal mask: every
 // query sees the whole cache, as in the question-after-context setting).
 //
-// One CTA per (problem, block of 128 queries).  Exact two-pass softmax on the
-// tensor cores:
-//   pass 1   S = Q K_t^T per 128-key tile (tcgen05.mma, fp32 in TMEM), row maxima
-//   pass 2   S again, P = exp(S - max) split into bf16 P_hi + P_lo in shared
-//            memory, O += P_hi V_t + P_lo V_t (V tile read MN-major), row sums
+// One CTA per (problem, block of 128 queries), one pass over the keys with an
+// online softmax on the tensor cores:
+//   S = Q K_t^T per 128-key tile (tcgen05.mma, fp32 in TMEM, double-buffered);
+//   P = exp2(S - m) split into bf16 P_hi + P_lo in shared memory;
+//   O_g += P_hi V_t + P_lo V_t (V tile read MN-major), row sums l_g.
 // Warp 0 feeds the TMA ring, warp 1 issues the MMAs, and two groups of four
-// softmax warps take alternate key tiles (each group owns one S accumulator
-// and one P buffer), since the exponentials, not the tensor pipe, set the pace.
-// Bounded waits as in sketch_umma_kernel.  Keys at or beyond the
-// problem's row count are masked by index; the value rows among them are cleared
-// in shared memory so that padding can never leak NaNs through a zero weight.
+// softmax warps take alternate key tiles.  Each group runs its own online
+// softmax (running maximum m_g, sum l_g, accumulator O_g in TMEM); the running
+// maximum only moves when a tile exceeds it by more than 2^8, and then the group
+// rescales its accumulator in TMEM, which after the first tiles is rare.  The
+// two halves are merged at the end: O = (2^(m_0-m) O_0 + 2^(m_1-m) O_1) / (...).
+// Bounded waits as in sketch_umma_kernel.  Keys at or beyond the problem's row
+// count are masked by index; the value rows among them are cleared in shared
+// memory so that padding can never leak NaNs through a zero weight.
 #pragma once
 #include "whiten_umma.cuh"
 
@@ -38,12 +41,30 @@ constexpr int kAttnPBytes = 2 * kSlotBytes;
 constexpr int kAttnSlot0 = kAttnP + 2 * kAttnPBytes;
 constexpr int kAttnBar = kAttnSlot0 + kAttnRing * kSlotBytes;
 constexpr int kAttnDynamic = kAttnBar + 256 + 1024;
-constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O at 256
+constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O[2] at 256 / 384
+constexpr float kAttnMaxSlack = 8.f;                       // log2 units a tile may exceed the running maximum
 
 // P V: A = P K-major, B = V tile MN-major (contraction over the keys)
 __host__ __device__ constexpr uint32_t instr_desc_pv() { return instr_desc_bf16(128) | (1u << 16); }
 
 // 2^x, relative error ~2^-22 (the weights are rounded to bf16 pairs afterwards)
+// 32 consecutive fp32 columns of this thread's TMEM lane, written back.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  const uint32_t* u = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), "r"(u[8]),
+      "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]), "r"(u[16]),
+      "r"(u[17]), "r"(u[18]), "r"(u[19]), "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]), "r"(u[24]),
+      "r"(u[25]), "r"(u[26]), "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -75,7 +96,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   const uint32_t o_full_bar = bar0 + 8u * (2 * kAttnRing + 9);
   const uint32_t drain_bar = bar0 + 8u * (2 * kAttnRing + 10);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + kAttnBar + 8 * (2 * kAttnRing + 11));
-  __shared__ float xchg[2][kTileRows];                     // row maxima, then row sums, of the two groups
+  __shared__ float xchg[2][kTileRows];                     // running maximum and row sum of the second group
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -123,7 +144,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   const uint32_t tmem_base = *tmem_holder;
 
   // Tiles go through the ring in the order the MMA issuer consumes them:
-  //   pass 1: K_0 .. K_{T-1};  pass 2: K_0, then for every t: K_{t+1} (if any), V_t.
+  //   K_0, then for every t: K_{t+1} (if any), V_t.
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -145,8 +166,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         tma_load_4d(dst + kHalfBytes, map, full_bar(slot), 64, key0 + t * kTileRows, kh, kb, pol_keep);
         ++it;
       };
-      for (int t = 0; ok && t < T; ++t) load(&map_k, t);
-      if (ok) load(&map_k, 0);
+      load(&map_k, 0);
       for (int t = 0; ok && t < T; ++t) {
         if (t + 1 < T) load(&map_k, t + 1);
         if (ok) load(&map_v, t);
@@ -186,8 +206,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         ++it;
         ++job;
       };
-      for (int t = 0; ok && t < T; ++t) issue_s();         // pass 1
-      if (ok) issue_s();                                   // pass 2, tile 0
+      if (ok) issue_s();                                   // tile 0
       for (int t = 0; ok && t < T; ++t) {
         if (t + 1 < T) issue_s();
         if (!ok) break;
@@ -203,7 +222,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                                           j * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        const uint32_t pbuf = (uint32_t)(T + t) & 1u;      // the buffer of the group that owns this tile
+        const uint32_t pbuf = (uint32_t)t & 1u;            // the group that owns this tile, its P and O
         if (!(ok = mbar_wait(p_ready_bar(pbuf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status))) break;
         tc_fence_after();
         const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
@@ -211,8 +230,8 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           const uint32_t p_base = base + kAttnP + pbuf * kAttnPBytes + part * kSlotBytes;
           for (int g = 0; g < groups; ++g) {               // 16 keys per MMA
             const uint32_t poff = (g >> 2) * kHalfBytes + (g & 3) * 32;
-            tc_mma_bf16(tmem_base + 256u, smem_desc_sw128(p_base + poff),
-                        smem_desc_mn_sw128(v_base + g * 2048), idesc_pv, (t > 0 || part > 0 || g > 0) ? 1u : 0u);
+            tc_mma_bf16(tmem_base + 256u + pbuf * 128u, smem_desc_sw128(p_base + poff),
+                        smem_desc_mn_sw128(v_base + g * 2048), idesc_pv, (t > 1 || part > 0 || g > 0) ? 1u : 0u);
           }
         }
         tc_commit(empty_bar(slot));
@@ -234,51 +253,60 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     constexpr float kLog2e = 1.4426950408889634f;
     const float sc = a.scale * kLog2e;                     // logits in units of log2
-    float top = extra > 0 ? 0.f : -INFINITY;
-    bool ok = true;
-    for (uint32_t job = (uint32_t)group; ok && job < (uint32_t)T; job += 2) {   // pass 1: row maxima
-      const int t = (int)job;
-      ok = mbar_wait(s_full_bar(group), (job >> 1) & 1u, abort_flag, a.status);
+    // running maximum (log2 units) and row sum of this group's tiles; Lemma 1's zero keys (logit 0,
+    // weight 2^0 each) are booked by the first group
+    float top = (extra > 0 && group == 0) ? 0.f : -INFINITY;
+    float sum = (extra > 0 && group == 0) ? (float)extra : 0.f;
+    bool has_o = false, ok = true;                         // has_o: O_group holds at least one product
+    unsigned char* Pbuf = base_ptr + kAttnP + group * kAttnPBytes;
+    const uint32_t s_addr = lane_addr + group * 128u, o_addr = lane_addr + 256u + group * 128u;
+    for (int t = group; ok && t < T; t += 2) {
+      ok = mbar_wait(s_full_bar(group), (uint32_t)(t >> 1) & 1u, abort_flag, a.status);
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const int valid = n - t * kTileRows;                 // keys of this tile that exist
+      float tile_top = -INFINITY;
 #pragma unroll 1
       for (int c0 = 0; c0 < 128; c0 += 32) {
         float v[32];
-        tmem_ld32(lane_addr + group * 128u + c0, v);
+        tmem_ld32(s_addr + c0, v);
         tmem_ld_wait();
-        if (valid >= kTileRows) {                          // full tile: no masking
+        if (valid >= kTileRows) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) top = fmaxf(top, v[c] * sc);
+          for (int c = 0; c < 32; ++c) tile_top = fmaxf(tile_top, v[c] * sc);
         } else {
 #pragma unroll
           for (int c = 0; c < 32; ++c)
-            if (c0 + c < valid) top = fmaxf(top, v[c] * sc);
+            if (c0 + c < valid) tile_top = fmaxf(tile_top, v[c] * sc);
         }
       }
-      tc_fence_before();
-      mbar_arrive(s_empty_bar(group));
-    }
-    // both groups need the maximum over all tiles (reached by all eight warps, aborted or not)
-    xchg[group][r] = top;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    top = fmaxf(xchg[0][r], xchg[1][r]);
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    float sum = (extra > 0 && group == 0) ? (float)extra * exp2f(-top) : 0.f;
-    uint32_t first2 = (uint32_t)T;                         // first pass-2 job of this group's parity
-    if ((first2 & 1u) != (uint32_t)group) ++first2;
-    unsigned char* Pbuf = base_ptr + kAttnP + group * kAttnPBytes;
-    for (uint32_t job = first2; ok && job < 2u * (uint32_t)T; job += 2) {       // pass 2: P and row sums
-      const int t = (int)job - T;
-      ok = mbar_wait(s_full_bar(group), (job >> 1) & 1u, abort_flag, a.status);
-      if (ok && t >= 2) ok = mbar_wait(p_empty_bar(group), (uint32_t)((t >> 1) - 1) & 1u, abort_flag, a.status);
-      if (!(ok = __all_sync(0xffffffffu, ok))) break;
-      tc_fence_after();
-      const int valid = n - t * kTileRows;
+      // move the running maximum only when the tile exceeds it by more than the slack
+      const bool move = tile_top > top + kAttnMaxSlack || top == -INFINITY;
+      const float new_top = move ? fmaxf(top, tile_top) : top;
+      const float alpha = move ? fast_exp2(top - new_top) : 1.f;      // 0 when top was -inf
+      if (t >= 2) {                                        // this group's previous product has retired
+        ok = mbar_wait(p_empty_bar(group), (uint32_t)((t >> 1) - 1) & 1u, abort_flag, a.status);
+        if (!(ok = __all_sync(0xffffffffu, ok))) break;
+        tc_fence_after();
+      }
+      if (has_o && __any_sync(0xffffffffu, move)) {        // rescale O_group in TMEM
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          float v[32];
+          tmem_ld32(o_addr + c0, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) v[c] *= alpha;
+          tmem_st32(o_addr + c0, v);
+        }
+        tmem_st_wait();
+      }
+      sum *= alpha;
+      top = new_top;
 #pragma unroll 1
       for (int c0 = 0; c0 < 128; c0 += 32) {
         float v[32];
-        tmem_ld32(lane_addr + group * 128u + c0, v);
+        tmem_ld32(s_addr + c0, v);
         tmem_ld_wait();
 #pragma unroll
         for (int g = 0; g < 4; ++g) {                      // 8 keys -> one 16-byte chunk of P_hi, P_lo
@@ -305,12 +333,19 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       mbar_arrive(s_empty_bar(group));
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(p_ready_bar(group));
+      has_o = true;
     }
-    // group 1 hands its row sums to group 0, which finishes the rows
-    if (group == 1) xchg[1][r] = sum;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
+    // the second group hands its statistics to the first, which merges the two accumulators
+    if (group == 1) {
+      xchg[0][r] = has_o ? top : -INFINITY;
+      xchg[1][r] = has_o ? sum : 0.f;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");         // reached by all eight warps, aborted or not
     if (group == 0) {
-      sum += xchg[1][r];
+      const float top1 = xchg[0][r], sum1 = xchg[1][r];
+      const float m = fmaxf(top, top1);                    // group 0 always owns tile 0: m is finite
+      const float w0 = fast_exp2(top - m), w1 = top1 == -INFINITY ? 0.f : fast_exp2(top1 - m);
+      const float denom = w0 * sum + w1 * sum1;
       if (ok) {
         ok = mbar_wait(o_full_bar, 0, abort_flag, a.status);
         ok = __all_sync(0xffffffffu, ok);
@@ -318,18 +353,25 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       if (ok) {
         tc_fence_after();
         const int row = qb * kTileRows + r;
-        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        const float i0 = denom > 0.f ? w0 / denom : 0.f, i1 = denom > 0.f ? w1 / denom : 0.f;
+        const bool both = T > 1;                           // O_1 exists only if the second group had a tile
         float* out = a.O + ((size_t)p * a.m + row) * 128;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
-          float v[32];
+          float v[32], u[32];
           tmem_ld32(lane_addr + 256u + c0, v);
+          if (both) tmem_ld32(lane_addr + 384u + c0, u);
           tmem_ld_wait();
           if (row < a.m) {
 #pragma unroll
-            for (int c = 0; c < 32; c += 4)
-              *reinterpret_cast<float4*>(out + c0 + c) =
-                  make_float4(v[c] * inv, v[c + 1] * inv, v[c + 2] * inv, v[c + 3] * inv);
+            for (int c = 0; c < 32; c += 4) {
+              float4 o;
+              o.x = v[c] * i0 + (both ? u[c] * i1 : 0.f);
+              o.y = v[c + 1] * i0 + (both ? u[c + 1] * i1 : 0.f);
+              o.z = v[c + 2] * i0 + (both ? u[c + 2] * i1 : 0.f);
+              o.w = v[c + 3] * i0 + (both ? u[c + 3] * i1 : 0.f);
+              *reinterpret_cast<float4*>(out + c0 + c) = o;
+            }
           }
         }
       }

@@ -144,6 +144,26 @@ def test_attention_tiny_and_odd_shapes():
         _check_out(O, Q, K, V, np.full((1, 1), n), 0.2, what=f"m={m} n={n}")
 
 
+def test_attention_running_maximum_moves_every_tile():
+    """Logits that grow along the sequence force every tile to raise the running maximum (and each
+    warp group to rescale its accumulator); logits that shrink never do.  Both must match the oracle."""
+    B, H, n, d, m = 1, 2, 1500, 128, 130
+    g = torch.Generator(device=DEV).manual_seed(4)
+    ramp = torch.linspace(0.0, 1.0, n, device=DEV).view(1, 1, n, 1)
+    for direction in (1.0, -1.0):
+        K = torch.randn((B, H, n, d), generator=g, device=DEV) * 0.3
+        K[..., 0] += (40.0 * (ramp if direction > 0 else 1.0 - ramp)).squeeze(-1)
+        K = K.to(torch.bfloat16)
+        V = torch.randn((B, H, n, d), generator=g, device=DEV).to(torch.bfloat16)
+        Q = torch.randn((B, H, m, d), generator=g, device=DEV) * 0.3
+        Q[..., 0] += 3.0
+        Q = Q.to(torch.bfloat16)
+        desc = cur.make_desc(K, V, 32)
+        O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=1.0)
+        assert cur.curdkv_device_status(ws) == 0
+        _check_out(O, Q, K, V, np.full((B, H), n), 1.0, what=f"ramp {direction:+.0f}")
+
+
 def test_attention_rejects_bad_arguments():
     K = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device=DEV)
     Q = torch.zeros((1, 1, 16, 64), dtype=torch.bfloat16, device=DEV)
