@@ -502,8 +502,8 @@ def run_evict(args):
         "roofline": {"bound": "tensor", "kernel": "attention_umma_kernel (full + compressed cache)",
                      "achieved": tf, "peak": peak, "peak_kind": peak_kind, "unit": "TFLOP/s",
                      "frac": tf / peak, "traffic": None,
-                     "note": "algorithmic flops = one QK^T and one PV; the kernel issues twice that "
-                             "(two-pass softmax, hi/lo weights)"},
+                     "note": "algorithmic flops = one QK^T and one PV; the kernel issues 1.5x that "
+                             "(PV for the hi and the lo half of the weights)"},
     }), flush=True)
 
 
