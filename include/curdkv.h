@@ -260,8 +260,9 @@ curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* 
  *                compressed cache computes
  *   scale        multiplies the logits (the paper writes softmax(QK^T): scale = 1)
  *   O            fp32 [batch][kv_heads][q_rows][128]; a head with no key rows gets 0
- * Exact two-pass softmax; the weights enter the second product as bf16 pairs
- * (hi + lo), so O agrees with an fp64 evaluation to about 1e-5 relative. */
+ * Online softmax in fp32 (exact up to rounding: no approximation of the maximum's
+ * effect); the weights enter the second product as bf16 pairs (hi + lo), so O agrees
+ * with an fp64 evaluation to about 1e-5 relative. */
 size_t curdkv_attention_workspace_bytes(const curdkv_desc* desc);
 curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stride_b, int64_t q_stride_h,
                                    int64_t q_stride_n, const void* K, const void* V,
