@@ -59,14 +59,20 @@ class Cache(ctypes.Structure):
 
 
 def load():
-    """Load the CUDA library (built by ``python -m paper_2509_15038_b200.build``)."""
+    """Load the CUDA library, compiling it first with nvcc if it is missing or older than its
+    sources (a fresh checkout has no binary).  There is no other implementation to fall back to:
+    if the build fails, this raises."""
     global _lib
     if _lib is not None:
         return _lib
-    if not _LIB_PATH.exists():
-        raise RuntimeError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2509_15038_b200.build` "
-            "(there is no fallback path)")
+    from . import build as _build
+
+    try:
+        _build.build_library()
+    except Exception as exc:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing and could not be built: {exc} "
+                               "(there is no fallback path)") from exc
     lib = ctypes.CDLL(str(_LIB_PATH))
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     dp = ctypes.POINTER(Desc)
