@@ -106,6 +106,16 @@ def test_ragged_batch_larger_than_one_kernel_slice():
     np.testing.assert_array_equal(idx.cpu().numpy(), eidx)
 
 
+def test_odd_row_count_misaligned_score_rows():
+    """n_max = 1001: score rows of odd heads start off 16-byte boundaries (scalar paths of the
+    normaliser and the selection), and the last tile holds a single row."""
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=2, n_max=1001, kv_heads=3, q_heads=3)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = synth.make_G(w.d, 32, seed=0)
+    full_pipeline_check(K, V, G, 150, 4, 16, what="n_max=1001")
+    full_pipeline_check(K, V, G, 150, 0, 8, seqlens=np.array([1001, 897], dtype=np.int32), what="n_max=1001 ragged")
+
+
 def test_strided_token_major_layout():
     """K, V stored [B, n, H, d] (token-major) and viewed as [B, H, n, d]."""
     B, H, n, d = 2, 4, 640, 128
