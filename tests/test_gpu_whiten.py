@@ -103,6 +103,30 @@ def test_whitened_identity_G_gives_svd_leverage():
     np.testing.assert_allclose(full, np.sum(U * U, axis=1), rtol=1e-8)
 
 
+def test_whitened_and_attention_on_token_major_views():
+    """K, V stored [B, n, H, d] and viewed as [B, H, n, d]: strides reach the Gram, the per-item
+    sketch and the attention kernels through their tensor maps."""
+    from oracle import curdkv_eviction_oracle as ev
+
+    B, H, n, d = 2, 3, 700, 128
+    g = torch.Generator(device=DEV).manual_seed(17)
+    Kb = torch.randn((B, n, H, d), generator=g, device=DEV).to(torch.bfloat16)
+    Vb = torch.randn((B, n, H, d), generator=g, device=DEV).to(torch.bfloat16)
+    K, V = Kb.permute(0, 2, 1, 3), Vb.permute(0, 2, 1, 3)
+    _check(K, V, synth.make_G(d, 32, seed=4), 1e-4, what="token-major whitened")
+    Q = torch.randn((B, H, 96, d), generator=g, device=DEV).to(torch.bfloat16)
+    desc = cur.make_desc(K, V, 32)
+    O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=0.1)
+    assert cur.curdkv_device_status(ws) == 0
+    got = O.cpu().numpy().astype(np.float64)
+    f = lambda t: synth.u16_to_f64(synth.to_u16(t))
+    Qf, Kf, Vf = f(Q), f(K), f(V)
+    for b in range(B):
+        for h in range(H):
+            want = ev.attention_out(Qf[b, h], Kf[b, h], Vf[b, h], 0.1)
+            assert np.abs(got[b, h] - want).max() <= 2e-4 * np.abs(want).max()
+
+
 def test_whitened_rejects_unsupported_shapes():
     K = torch.zeros((1, 1, 64, 128), dtype=torch.bfloat16, device=DEV)
     G = torch.zeros((128, 32), dtype=torch.float32, device=DEV)
