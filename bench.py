@@ -360,12 +360,17 @@ def run_decode(args):
     cur.curdkv_cache_compress(caches[0], caches[1], k, ws, num_sink=c["num_sink"], window=c["window"])
     live = 1
 
+    inplace = args.decode_mode == "inplace"
+
     def step():
         nonlocal live
         cur.curdkv_cache_append(caches[live], K_new, V_new, G, ws)
-        cur.curdkv_cache_compress(caches[live], caches[1 - live], k, ws, num_sink=c["num_sink"],
-                                  window=c["window"])
-        live = 1 - live
+        if inplace:       # survivors stay put, at most `chunk` rows per head move into the holes
+            cur.curdkv_cache_compress_inplace(caches[live], k, ws, num_sink=c["num_sink"], window=c["window"])
+        else:             # ordered copy of all survivors into the other cache
+            cur.curdkv_cache_compress(caches[live], caches[1 - live], k, ws, num_sink=c["num_sink"],
+                                      window=c["window"])
+            live = 1 - live
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -388,8 +393,9 @@ def run_decode(args):
     ms = t0.elapsed_time(t1) / args.steps
     P = LB * H
     rows = P * (k + t)                       # rows the compression looks at per step
-    # new rows read and stored, their scores; held scores read; survivors read and written
-    counted = P * (t * 512 * 2 + (k + t) * 4 + k * 512 * 2)
+    # new rows read and stored, their scores; held scores read; then either every survivor read and
+    # written (ordered) or at most `chunk` moved rows per head read and written (in place)
+    counted = P * (t * 512 * 2 + (k + t) * 4 + (t if inplace else k) * 512 * 2)
     peak, peak_kind = measured_peak()
     gbs = counted / (ms * 1e-3) / 1e9
     print(json.dumps({
@@ -398,7 +404,8 @@ def run_decode(args):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "decode: %(layers)d layers x batch %(batch)d x %(kv_heads)d KV heads, cache "
                                "budget %(budget)d (sinks %(num_sink)d, window %(window)d), %(chunk)d new rows "
-                               "per head and step, r=%(r)d" % c,
+                               "per head and step, r=%(r)d" % c
+                               + (", in-place compression" if inplace else ", ordered compression into a second cache"),
                    "head_tokens_per_step": rows,
                    "l2": "caches (%.1f GB) exceed the 126 MB L2" % (2 * 2 * P * cap * d * 2 / 1e9)},
         "gb_per_s": gbs, "counted_bytes_per_step": counted,
@@ -596,6 +603,8 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode", "evict"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
+                    help="--workload decode: compress inside the cache (unordered) or copy in order")
     ap.add_argument("--whiten", action="store_true",
                     help="score with the whitened sketch (approximate leverage scores; reads K, V twice)")
     ap.add_argument("--e2e-steps", type=int, default=3,

@@ -276,6 +276,18 @@ curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compresse
                                    int64_t elems_per_problem, float* loss, float* ref_norm,
                                    void* cuda_stream);
 
+/* The same compression inside one cache, for steady-state generation: the rows that are
+ * kept stay where they are, and only survivors stored at or beyond slot min(budget, held)
+ * move, into the slots the evicted rows leave below it (at most as many rows as were
+ * evicted, instead of a copy of the whole cache).  Afterwards the cache holds its rows in no
+ * particular order: `pos` tells which token each slot holds, and attention over the cache
+ * does not depend on the order.  The kept SET is that of curdkv_cache_compress, except that
+ * ties between equal scores go to the lower slot rather than the lower position.
+ * Requires num_sink + window <= budget and capacity <= 204800. */
+curdkv_status curdkv_cache_compress_inplace(const curdkv_cache* cache, const curdkv_desc* desc,
+                                            int32_t budget, int32_t num_sink, int32_t window,
+                                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* GQA (Sec. 3.2): query head q uses KV head q / (q_heads / kv_heads).  Writes
  * kv_head_of_q int32 [q_heads] (device) so that attention consumers can index
  * the shared selection without replicating the compacted cache. */

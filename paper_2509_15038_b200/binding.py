@@ -26,7 +26,7 @@ EXPORTS = (
     "curdkv_score_static", "curdkv_host_arena_bytes", "curdkv_compress_host",
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
     "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
-    "curdkv_eviction_loss", "curdkv_gqa_expand",
+    "curdkv_eviction_loss", "curdkv_gqa_expand", "curdkv_cache_compress_inplace",
 )
 
 
@@ -106,6 +106,8 @@ def load():
     lib.curdkv_cache_append.argtypes = [cp, vp, vp, vp, i32, dp, vp, ctypes.c_size_t, vp]
     lib.curdkv_cache_compress.restype = ctypes.c_int
     lib.curdkv_cache_compress.argtypes = [cp, cp, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
+    lib.curdkv_cache_compress_inplace.restype = ctypes.c_int
+    lib.curdkv_cache_compress_inplace.argtypes = [cp, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
     lib.curdkv_attention_workspace_bytes.restype = ctypes.c_size_t
     lib.curdkv_attention_workspace_bytes.argtypes = [dp]
     lib.curdkv_attention_out.restype = ctypes.c_int
@@ -342,6 +344,17 @@ def curdkv_cache_compress(src: DeviceCache, dst: DeviceCache, budget: int, works
                                         int(budget), int(num_sink), int(window), _ptr(workspace),
                                         workspace.numel(), _stream())
     _check(code, "curdkv_cache_compress")
+
+
+def curdkv_cache_compress_inplace(cache: DeviceCache, budget: int, workspace: torch.Tensor, *,
+                                  num_sink: int = 0, window: int = 0) -> None:
+    """Alg. 1 lines 6-10 on the rows held in ``cache``, in place (the row order is given up)."""
+    desc = Desc(cache.batch, cache.kv_heads, cache.kv_heads, cache.capacity, cache.d, 1)
+    desc.use_projection = 1
+    code = load().curdkv_cache_compress_inplace(ctypes.byref(cache.c), ctypes.byref(desc), int(budget),
+                                                int(num_sink), int(window), _ptr(workspace),
+                                                workspace.numel(), _stream())
+    _check(code, "curdkv_cache_compress_inplace")
 
 
 def curdkv_attention_out(Q, K, V, desc: Desc, *, scale: float = 1.0, head_rows=None, head_offsets=None,

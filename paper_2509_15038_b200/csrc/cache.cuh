@@ -94,4 +94,90 @@ __global__ void __launch_bounds__(256) cache_gather_meta_kernel(const CacheView 
   }
 }
 
+// ---- in-place compression: the cache keeps no particular row order ----------
+
+// Selection keys of the held rows: +inf for forced rows (positions < num_sink or among the most
+// recent `window`), otherwise the row's l^KV, lifted to the smallest positive float if it is 0 so
+// that a real row always outranks an unused slot.  grid = batch*heads, block = 256.
+__global__ void __launch_bounds__(256) cache_keyed_scores_kernel(const CacheView c, int heads, int num_sink,
+                                                                 int window, float* keyed) {
+  const int p = blockIdx.x, b = p / heads;
+  const int held = min(max(c.count[b], 0), c.capacity);
+  const int recent = c.total[b] - window;
+  for (int s = threadIdx.x; s < held; s += blockDim.x) {
+    const int pos = c.pos[(size_t)p * c.capacity + s];
+    const float raw = c.raw[(size_t)p * c.capacity + s];
+    keyed[(size_t)p * c.capacity + s] =
+        (pos < num_sink || pos >= recent) ? __int_as_float(0x7f800000) : fmaxf(raw, 1.17549435e-38f);
+  }
+}
+
+// After the selection: rows kept at slots >= kept ("movers", the tail of the ascending idx list)
+// are copied into the slots < kept that were not kept ("holes"), so that the survivors occupy
+// slots [0, kept) again.  At most min(kept, held - kept) rows move.  grid = batch*heads,
+// block = 256, dynamic shared memory = capacity bytes (slot flags); holes: int32 [problems][capacity].
+__global__ void __launch_bounds__(256) cache_fill_holes_kernel(const CacheView c, const int32_t* idx,
+                                                               int budget, const int32_t* counts, int heads,
+                                                               int d, int32_t* holes, uint32_t* status) {
+  extern __shared__ unsigned char slot_kept[];
+  __shared__ int s_first_mover, s_base, s_warp_tot[8];
+  const int p = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kept = min(counts[p], c.capacity);
+  const int32_t* ix = idx + (size_t)p * budget;
+  int32_t* my_holes = holes + (size_t)p * c.capacity;
+  for (int s = tid; s < kept; s += 256) slot_kept[s] = 0;
+  if (tid == 0) {                                          // idx is ascending: first entry >= kept
+    int lo = 0, hi = kept;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (ix[mid] < kept) lo = mid + 1; else hi = mid;
+    }
+    s_first_mover = lo;
+    s_base = 0;
+  }
+  __syncthreads();
+  const int first_mover = s_first_mover, movers = kept - first_mover;
+  for (int t = tid; t < first_mover; t += 256) slot_kept[ix[t]] = 1;
+  __syncthreads();
+  // holes in ascending slot order, 256 slots per sweep
+  for (int s0 = 0; s0 < kept; s0 += 256) {
+    const int s = s0 + tid;
+    const bool hole = s < kept && slot_kept[s] == 0;
+    const uint32_t bal = __ballot_sync(0xffffffffu, hole);
+    if (lane == 0) s_warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int before = s_base;
+    for (int w = 0; w < warp; ++w) before += s_warp_tot[w];
+    if (hole) my_holes[before + __popc(bal & ((1u << lane) - 1u))] = s;
+    __syncthreads();
+    if (tid == 0) {
+      int tot = 0;
+      for (int w = 0; w < 8; ++w) tot += s_warp_tot[w];
+      s_base += tot;
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && s_base != movers) flag_status(status, CURDKV_DEV_BAD_INDEX);   // idx was not a valid selection
+  const int moves = min(s_base, movers);
+  // copy mover i into hole i: a half-warp per tensor row (K in lanes 0-15, V in lanes 16-31)
+  const int half = lane >> 4, l16 = lane & 15, chunks = d >> 3;
+  __nv_bfloat16* rows = (half ? c.V : c.K) + (size_t)p * c.capacity * d;
+  for (int i = warp; i < moves; i += 8) {
+    const int src = ix[first_mover + i], dst = my_holes[i];
+    for (int ch = l16; ch < chunks; ch += 16)
+      reinterpret_cast<uint4*>(rows + (size_t)dst * d)[ch] =
+          *reinterpret_cast<const uint4*>(rows + (size_t)src * d + ch * 8);
+    if (lane == 0) {
+      c.raw[(size_t)p * c.capacity + dst] = c.raw[(size_t)p * c.capacity + src];
+      c.pos[(size_t)p * c.capacity + dst] = c.pos[(size_t)p * c.capacity + src];
+    }
+  }
+}
+
+// count[b] = rows kept (the same for every head of a sequence).  grid = ceil(batch / 256).
+__global__ void cache_set_count_kernel(CacheView cache, const int32_t* counts, int heads, int batch) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < batch) cache.count[b] = min(counts[b * heads], cache.capacity);
+}
+
 }  // namespace curdkv

@@ -13,7 +13,7 @@ using namespace curdkv;
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct CacheWorkspace {     // byte offsets from the workspace base
-  size_t score_ws, raw_new, sums, idx, counts, total;
+  size_t score_ws, raw_new, sums, idx, counts, keyed, holes, total;
 };
 
 bool layout(int32_t batch, int32_t heads, int32_t t_max, int32_t capacity, int32_t budget,
@@ -36,6 +36,8 @@ bool layout(int32_t batch, int32_t heads, int32_t t_max, int32_t capacity, int32
   L->sums = take(P * 4);
   L->idx = take(P * (size_t)budget * 4);
   L->counts = take(P * 4);
+  L->keyed = take(P * (size_t)capacity * 4);    // in-place compression only
+  L->holes = take(P * (size_t)capacity * 4);
   L->total = o;
   return true;
 }
@@ -148,6 +150,57 @@ curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* 
   }
   cache_gather_meta_kernel<<<(unsigned)P, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       view_of(in), view_of(out), idx, budget, counts, d.kv_heads);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_cache_compress_inplace(const curdkv_cache* cache, const curdkv_desc* desc,
+                                            int32_t budget, int32_t num_sink, int32_t window,
+                                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!cache_ok(cache) || desc == nullptr || workspace == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (budget < 0 || num_sink < 0 || window < 0) return CURDKV_ERR_INVALID_ARG;
+  if ((int64_t)num_sink + window > budget) return CURDKV_ERR_INVALID_ARG;   // forced rows must fit
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  if (cache->capacity > 200 * 1024) return CURDKV_ERR_UNSUPPORTED;          // slot flags live in shared memory
+  CacheWorkspace L;
+  if (!layout(desc->batch, desc->kv_heads, 0, cache->capacity, budget, &L)) return CURDKV_ERR_INVALID_ARG;
+  if (workspace_bytes < L.total) return CURDKV_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  float* keyed = reinterpret_cast<float*>(ws + L.keyed);
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  if (P == 0 || budget == 0) return budget == 0 && P > 0 ? CURDKV_ERR_INVALID_ARG : CURDKV_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const CacheView view = view_of(cache);
+
+  cache_keyed_scores_kernel<<<(unsigned)P, 256, 0, stream>>>(view, desc->kv_heads, num_sink, window, keyed);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+
+  curdkv_desc d = *desc;
+  d.q_heads = d.kv_heads;
+  d.n_max = cache->capacity;
+  d.seqlens = cache->count;
+  d.score_mode = 0;
+  d.use_projection = 1;
+  d.raw_scores = 0;
+  d.whiten = 0;
+  // forced rows carry +inf keys, so the selection itself needs no sinks or window
+  curdkv_status st = curdkv_select(keyed, &d, budget, nullptr, 0, 0, 0, 0.0, idx, counts, nullptr,
+                                   ws + L.score_ws, L.raw_new - L.score_ws, cuda_stream);
+  if (st != CURDKV_OK) return st;
+  if (cudaFuncSetAttribute(cache_fill_holes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           200 * 1024) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  cache_fill_holes_kernel<<<(unsigned)P, 256, (size_t)cache->capacity, stream>>>(
+      view, idx, budget, counts, d.kv_heads, d.d, reinterpret_cast<int32_t*>(ws + L.holes),
+      reinterpret_cast<uint32_t*>(ws + L.score_ws));
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  cache_set_count_kernel<<<(unsigned)((d.batch + 255) / 256), 256, 0, stream>>>(view, counts, d.kv_heads,
+                                                                                d.batch);
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
   return CURDKV_OK;

@@ -103,6 +103,52 @@ def test_decode_token_by_token_and_ragged_appends():
     _compare(cache, ref, 24, 2, 4)
 
 
+@pytest.mark.parametrize("k,s,w", [(64, 4, 0), (64, 0, 16), (100, 4, 8)])
+def test_decode_in_place_keeps_the_same_rows(k, s, w):
+    """In-place compression (rows stay put, survivors from the tail fill the holes): the cache ends
+    up unordered but holds exactly the rows the ordered procedure and one-shot Alg. 1 keep."""
+    B, H, N, d, r = 3, 2, 700, 128, 32
+    K, V = _history(B, H, N, d, seed=31)
+    G = synth.make_G(d, r, seed=0)
+    Gd = torch.as_tensor(G, device=DEV)
+    schedule = [256, 1, 1, 130, 7, 200, 64, 41]
+    capacity = k + 256
+    cache = cur.DeviceCache(B, H, capacity, d, DEV)
+    ws = cur.cache_workspace(B, H, max(schedule), capacity, k, DEV)
+    ref = dec.CacheOracle(B, H, d)
+    Ku, Vu = synth.to_u16(K), synth.to_u16(V)
+    at = held = 0
+    for t in schedule:
+        if held + t > capacity:
+            cur.curdkv_cache_compress_inplace(cache, k, ws, num_sink=s, window=w)
+            ref.compress(k, s, w)
+            held = min(held, k)
+        cur.curdkv_cache_append(cache, K[:, :, at:at + t], V[:, :, at:at + t], Gd, ws)
+        ref.append(Ku[:, :, at:at + t], Vu[:, :, at:at + t], G)
+        at += t
+        held += t
+    cur.curdkv_cache_compress_inplace(cache, k, ws, num_sink=s, window=w)
+    ref.compress(k, s, w)
+    assert cur.curdkv_device_status(ws) == 0
+    cnt = cache.count.cpu().numpy()
+    pos, raw = cache.pos.cpu().numpy(), cache.raw.cpu().numpy()
+    Ko, Vo = synth.to_u16(cache.K), synth.to_u16(cache.V)
+    for b in range(B):
+        for h in range(H):
+            c = int(cnt[b])
+            assert c == len(ref.pos[b][h])
+            got = pos[b, h, :c]
+            assert len(set(got.tolist())) == c                      # no slot twice
+            # fp32 vs fp64 scores can only disagree on a near-tie at the cut
+            assert len(set(got.tolist()) ^ set(ref.pos[b][h].tolist())) <= 2
+            for slot in range(c):                                   # every slot holds its token's rows
+                np.testing.assert_array_equal(Ko[b, h, slot], Ku[b, h, got[slot]])
+                np.testing.assert_array_equal(Vo[b, h, slot], Vu[b, h, got[slot]])
+            order = np.argsort(got)
+            both, gi, ri = np.intersect1d(got[order], ref.pos[b][h], return_indices=True)
+            np.testing.assert_allclose(raw[b, h, :c][order][gi], ref.raw[b][h][ri], rtol=1e-3)
+
+
 def test_decode_overflow_is_flagged_not_written():
     B, H, d = 1, 1, 128
     K, V = _history(B, H, 64, d, seed=23)
