@@ -47,7 +47,6 @@ constexpr float kAttnMaxSlack = 8.f;                       // log2 units a tile 
 // P V: A = P K-major, B = V tile MN-major (contraction over the keys)
 __host__ __device__ constexpr uint32_t instr_desc_pv() { return instr_desc_bf16(128) | (1u << 16); }
 
-// 2^x, relative error ~2^-22 (the weights are rounded to bf16 pairs afterwards)
 // 32 consecutive fp32 columns of this thread's TMEM lane, written back.
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
   const uint32_t* u = reinterpret_cast<const uint32_t*>(v);
@@ -65,6 +64,7 @@ __device__ __forceinline__ void tmem_st_wait() {
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+// 2^x, relative error ~2^-22 (the weights are rounded to bf16 pairs afterwards)
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
