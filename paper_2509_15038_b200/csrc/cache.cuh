@@ -50,14 +50,29 @@ __global__ void __launch_bounds__(kAppendWarps * 32) cache_append_kernel(const A
   const __nv_bfloat16* src = T.base + b * T.stride_b + h * T.stride_h;
   __nv_bfloat16* dst = (half ? a.cache.V : a.cache.K) + ((size_t)p * a.cache.capacity + held) * a.d;
   const int chunks = a.d >> 3;
-  for (int i = chunk * kAppendRowsPerCta + warp; i < min((chunk + 1) * kAppendRowsPerCta, tb);
-       i += kAppendWarps) {
-    for (int c = l16; c < chunks; c += 16)
-      reinterpret_cast<uint4*>(dst + (size_t)i * a.d)[c] =
-          __ldg(reinterpret_cast<const uint4*>(src + i * T.stride_n) + c);
-    if (lane == 0) {
-      a.cache.raw[(size_t)p * a.cache.capacity + held + i] = a.raw_new[(size_t)p * a.t + i];
-      a.cache.pos[(size_t)p * a.cache.capacity + held + i] = first_pos + i;
+  // four rows per warp in flight (rows warp, warp + 8, warp + 16, warp + 24 of the chunk)
+  const int row0 = chunk * kAppendRowsPerCta + warp;
+  for (int c = l16; c < chunks; c += 16) {
+    uint4 v[kAppendRowsPerCta / kAppendWarps];
+#pragma unroll
+    for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
+      const int i = row0 + j * kAppendWarps;
+      if (i < tb) v[j] = __ldg(reinterpret_cast<const uint4*>(src + i * T.stride_n) + c);
+    }
+#pragma unroll
+    for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
+      const int i = row0 + j * kAppendWarps;
+      if (i < tb) reinterpret_cast<uint4*>(dst + (size_t)i * a.d)[c] = v[j];
+    }
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
+      const int i = row0 + j * kAppendWarps;
+      if (i < tb) {
+        a.cache.raw[(size_t)p * a.cache.capacity + held + i] = a.raw_new[(size_t)p * a.t + i];
+        a.cache.pos[(size_t)p * a.cache.capacity + held + i] = first_pos + i;
+      }
     }
   }
 }
