@@ -231,6 +231,7 @@ def run_cuda(args):
     else:
         ms_step = max_over_ranks(t0.elapsed_time(t1), dev, world) / args.steps
     stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in ev]).mean(0)
+    per_step = np.array([e[0].elapsed_time(e[3]) for e in ev])      # this rank's steps, one by one
 
     tokens, read_bytes, write_bytes = workload_bytes(w, seqlens)
     pass_bytes = read_bytes                  # K + V once: what one streaming kernel reads
@@ -265,6 +266,7 @@ def run_cuda(args):
         "seq_tokens_per_s": value / (w.layers * w.kv_heads),
         "stage_ms": {"score": float(stage_ms[0]), "select": float(stage_ms[1]),
                      "compact": float(stage_ms[2])},
+        "ms_per_step_median": float(np.median(per_step)), "ms_per_step_best": float(per_step.min()),
         "clocks": clocks,
         "gpu_launches": int(launches),
         "roofline": {
