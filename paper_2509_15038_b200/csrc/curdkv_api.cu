@@ -466,9 +466,13 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
   if (cudaFuncSetAttribute(select_fixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSelStageBytes + kSelListBytes) != cudaSuccess)
     return CURDKV_ERR_CUDA;
-  select_fixed_kernel<<<(unsigned)P, kSelThreads, stage_bytes + kSelListBytes, stream>>>(
+  // rows of up to 16384 tokens run as CTAs of 512 threads with a smaller list, two per SM
+  const bool small_rows = desc->n_max <= 16384;
+  const int sel_threads = small_rows ? 512 : kSelThreads;
+  const int list_cap = small_rows ? kSelListCap / 2 : kSelListCap;
+  select_fixed_kernel<<<(unsigned)P, sel_threads, stage_bytes + (size_t)list_cap * 8, stream>>>(
       scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,
-      (int)(stage_bytes / sizeof(uint4)), idx, head_counts, head_offsets);
+      (int)(stage_bytes / sizeof(uint4)), list_cap, idx, head_counts, head_offsets);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }

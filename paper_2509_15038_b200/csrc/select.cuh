@@ -76,25 +76,38 @@ struct SelectSmem {
 
 struct KeyList {
   uint2* items;            // (rank key, token index)
-  uint32_t* count;         // entries offered; more than kSelListCap means the list is incomplete
-  __device__ __forceinline__ bool complete() const { return *count <= (uint32_t)kSelListCap; }
-  __device__ __forceinline__ int size() const { return (int)min(*count, (uint32_t)kSelListCap); }
+  uint32_t* count;         // entries offered; more than cap means the list is incomplete
+  uint32_t cap;
+  __device__ __forceinline__ bool complete() const { return *count <= cap; }
+  __device__ __forceinline__ int size() const { return (int)min(*count, cap); }
 };
 
+// The CTA-wide helpers below work for CTAs of 1024 threads (four histogram bins per thread) and
+// of 512 threads (eight): short rows run as two 512-thread CTAs per SM, which hides more of the
+// latency of their many short phases.
 __device__ __forceinline__ void clear_hist(uint32_t* hist) {
-  reinterpret_cast<uint4*>(hist)[threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);   // 1024 threads x 4 bins
+  for (int i = threadIdx.x; i < kSelBins / 4; i += blockDim.x)
+    reinterpret_cast<uint4*>(hist)[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // One radix-select step over the kSelBins-bin histogram `hist`: finds the digit
 // holding the `remaining`-th largest key and leaves it in sm.digit, the rank
 // inside that digit's bucket in sm.remaining and the number of keys in higher
-// bins in sm.above.  Whole CTA (1024 threads, four bins each); the results are
+// bins in sm.above.  Whole CTA (B consecutive bins per thread); the results are
 // readable after the call.
-__device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
+template <int B>
+__device__ __forceinline__ void pick_digit_impl(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
+  constexpr int kWarps = kSelBins / (32 * B);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint4 c4 = reinterpret_cast<const uint4*>(hist)[tid];
-  const uint32_t c[4] = {c4.x, c4.y, c4.z, c4.w};
-  const uint32_t mine = c[0] + c[1] + c[2] + c[3];
+  uint32_t c[B];
+#pragma unroll
+  for (int q = 0; q < B / 4; ++q) {
+    const uint4 c4 = reinterpret_cast<const uint4*>(hist)[tid * (B / 4) + q];
+    c[4 * q] = c4.x; c[4 * q + 1] = c4.y; c[4 * q + 2] = c4.z; c[4 * q + 3] = c4.w;
+  }
+  uint32_t mine = 0;
+#pragma unroll
+  for (int u = 0; u < B; ++u) mine += c[u];
   uint32_t suffix = mine;                                  // inclusive suffix sum over the warp
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -104,7 +117,7 @@ __device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remain
   if (lane == 0) sm.warp_def[warp] = suffix;
   if (tid == 0) { sm.digit = 0; sm.remaining = 0; sm.above = 0; }
   __syncthreads();
-  uint32_t w = sm.warp_def[lane], wsuf = w;                // inclusive suffix sum over the warps
+  uint32_t w = lane < kWarps ? sm.warp_def[lane] : 0u, wsuf = w;   // inclusive suffix sum over the warps
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const uint32_t v = __shfl_down_sync(0xffffffffu, wsuf, o);
@@ -112,9 +125,9 @@ __device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remain
   }
   uint32_t above = __shfl_sync(0xffffffffu, wsuf - w, warp) + (suffix - mine);
 #pragma unroll
-  for (int u = 3; u >= 0; --u) {
+  for (int u = B - 1; u >= 0; --u) {
     if (above < remaining && above + c[u] >= remaining) {
-      sm.digit = (uint32_t)(tid * 4 + u);
+      sm.digit = (uint32_t)(tid * B + u);
       sm.remaining = remaining - above;
       sm.above = above;
     }
@@ -122,25 +135,32 @@ __device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remain
   }
   __syncthreads();
 }
+__device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
+  if (blockDim.x == 1024) pick_digit_impl<4>(hist, remaining, sm);
+  else pick_digit_impl<8>(hist, remaining, sm);
+}
 
 // Number of keys of `hist` in bins above `digit`.  Whole CTA; every thread gets the sum.
-__device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
+template <int B>
+__device__ __forceinline__ uint32_t count_above_impl(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
+  constexpr int kWarps = kSelBins / (32 * B);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint4 c4 = reinterpret_cast<const uint4*>(hist)[tid];
-  const uint32_t c[4] = {c4.x, c4.y, c4.z, c4.w};
   uint32_t v = 0;
 #pragma unroll
-  for (int u = 0; u < 4; ++u)
-    if ((uint32_t)(tid * 4 + u) > digit) v += c[u];
+  for (int u = 0; u < B; ++u)
+    if ((uint32_t)(tid * B + u) > digit) v += hist[tid * B + u];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   if (lane == 0) sm.warp_eq[warp] = v;
   __syncthreads();
-  uint32_t t = sm.warp_eq[lane];
+  uint32_t t = lane < kWarps ? sm.warp_eq[lane] : 0u;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
   __syncthreads();
   return t;
+}
+__device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
+  return blockDim.x == 1024 ? count_above_impl<4>(hist, digit, sm) : count_above_impl<8>(hist, digit, sm);
 }
 
 // Rank keys of one row, four tokens at a time ("quad" q holds tokens
@@ -254,12 +274,13 @@ __device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, ui
   run.flush(hist);
 }
 
-// Quads of a row are dealt to the 32 warps in contiguous runs ("segments"), so that the kept
+// Quads of a row are dealt to the CTA's warps in contiguous runs ("segments"), so that the kept
 // tokens of warp w precede those of warp w + 1 in token order.
 struct Segments {
   int per_warp, quads;
   __device__ __forceinline__ explicit Segments(int quads_) : quads(quads_) {
-    per_warp = (((quads_ + 31) >> 5) + 31) & ~31;          // whole-warp sweeps
+    const int warps = (int)blockDim.x >> 5;
+    per_warp = ((quads_ + warps - 1) / warps + 31) & ~31;  // whole-warp sweeps
   }
   __device__ __forceinline__ int begin(int warp) const { return min(warp * per_warp, quads); }
   __device__ __forceinline__ int end(int warp) const { return min(begin(warp) + per_warp, quads); }
@@ -327,11 +348,11 @@ __device__ __forceinline__ void collect_sweep(const RowKeys& keys, uint32_t d_cu
           def_cnt += dgt > d_cut ? 1u : 0u;
           if (dgt == d_a) {
             const uint32_t at = atomicAdd(list_a.count, 1u);
-            if (at < (uint32_t)kSelListCap) list_a.items[at] = make_uint2(k4[i], 4u * (q0 + u * 32) + i);
+            if (at < list_a.cap) list_a.items[at] = make_uint2(k4[i], 4u * (q0 + u * 32) + i);
           }
           if (use_b && dgt == d_b) {
             const uint32_t at = atomicAdd(list_b.count, 1u);
-            if (at < (uint32_t)kSelListCap) list_b.items[at] = make_uint2(k4[i], 4u * (q0 + u * 32) + i);
+            if (at < list_b.cap) list_b.items[at] = make_uint2(k4[i], 4u * (q0 + u * 32) + i);
           }
         }
       }
@@ -397,7 +418,8 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
   __syncthreads();
   uint32_t def_before = 0, eq_before = 0;                  // kept / equal tokens of earlier warps
   {
-    const uint32_t d = sm.seg_def[lane], e = sm.seg_eq[lane];
+    const bool live = lane < ((int)blockDim.x >> 5);       // one segment per warp of the CTA
+    const uint32_t d = live ? sm.seg_def[lane] : 0u, e = live ? sm.seg_eq[lane] : 0u;
     uint32_t di = d, ei = e;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -448,14 +470,14 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
 }
 
 // ---------------------------------------------------------------------------
-// Fixed per-head budget.  grid = batch*heads, block = 1024, dynamic shared
+// Fixed per-head budget.  grid = batch*heads, block = 1024 or 512, dynamic shared
 // memory = 16 * stage_quads bytes (0: rows are read from global memory) followed
-// by one candidate list (kSelListBytes).
+// by one candidate list of list_cap entries.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
     int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window, int stage_quads,
-    int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+    int list_cap, int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   __shared__ SelectSmem sm;
   extern __shared__ uint4 staged_keys[];                   // stage_quads quads, or nothing
   const int p = blockIdx.x, b = p / heads, tid = threadIdx.x;
@@ -491,7 +513,8 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     const uint32_t d0 = sm.digit, rank = sm.remaining;
     __syncthreads();
     // sweep 2: keys above the digit are counted per segment, keys of the digit go to the list
-    const KeyList list{reinterpret_cast<uint2*>(staged_keys + stage_quads), &sm.list_count[0]};
+    const KeyList list{reinterpret_cast<uint2*>(staged_keys + stage_quads), &sm.list_count[0],
+                       (uint32_t)list_cap};
     collect_sweep(keys, d0, d0, list, false, 0u, list, sm);
     __syncthreads();
     cut = finish_cut(keys, list, d0, rank, sm);
@@ -502,7 +525,7 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
   }
   if (!counted) count_sweep(keys, cut, sm);
   write_sweep(keys, cut, out, sm);
-  for (int t = k_eff + tid; t < budget; t += kSelThreads) out[t] = -1;
+  for (int t = k_eff + tid; t < budget; t += (int)blockDim.x) out[t] = -1;
   if (tid == 0) {
     counts[p] = k_eff;
     if (offsets != nullptr) {                              // heads sit at multiples of `budget` rows
@@ -536,8 +559,9 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   __shared__ AdaptiveSmem sm;
   extern __shared__ uint4 adaptive_dyn[];
   uint32_t* hist_all = reinterpret_cast<uint32_t*>(adaptive_dyn);          // leading digits of all keys
-  const KeyList list_a{reinterpret_cast<uint2*>(hist_all + kSelBins), &sm.s.list_count[0]};
-  const KeyList list_b{list_a.items + kSelListCap, &sm.s.list_count[1]};
+  const KeyList list_a{reinterpret_cast<uint2*>(hist_all + kSelBins), &sm.s.list_count[0],
+                       (uint32_t)kSelListCap};
+  const KeyList list_b{list_a.items + kSelListCap, &sm.s.list_count[1], (uint32_t)kSelListCap};
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x;
   const int h = (int)cluster.block_rank();
@@ -560,7 +584,7 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   __syncthreads();
   uint32_t d0 = 0xffffffffu, rank_own = 0;
   if (!none && !all) {
-    pick_digit(hist_all, (uint32_t)prot, sm.s);
+    pick_digit_impl<4>(hist_all, (uint32_t)prot, sm.s);
     d0 = sm.s.digit;
     rank_own = sm.s.remaining;
     __syncthreads();
@@ -593,10 +617,10 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
       reinterpret_cast<uint4*>(sm.s.hist)[tid] = acc;
     }
     __syncthreads();
-    pick_digit(sm.s.hist, remaining, sm.s);
+    pick_digit_impl<4>(sm.s.hist, remaining, sm.s);
     dg = sm.s.digit;
     remaining = sm.s.remaining;
-    local_gt = count_above(sm.hist_local, dg, sm.s);
+    local_gt = count_above_impl<4>(sm.hist_local, dg, sm.s);
     cluster.sync();                                        // peers are done reading hist_local
   }
 
@@ -644,12 +668,12 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
         reinterpret_cast<uint4*>(sm.s.hist)[tid] = acc;
       }
       __syncthreads();
-      pick_digit(sm.s.hist, remaining, sm.s);
+      pick_digit_impl<4>(sm.s.hist, remaining, sm.s);
       const uint32_t dgt = sm.s.digit;
       remaining = sm.s.remaining;
       prefix |= dgt << shift;
       mask |= pass_digit_mask(pass) << shift;
-      local_gt += count_above(sm.hist_local, dgt, sm.s);
+      local_gt += count_above_impl<4>(sm.hist_local, dgt, sm.s);
       if (pass == kSelPasses - 1) local_eq = sm.hist_local[dgt];
       cluster.sync();                                      // peers are done reading hist_local
     }
