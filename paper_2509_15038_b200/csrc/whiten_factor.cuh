@@ -5,27 +5,23 @@
 //
 // One CTA of 256 threads per matrix, two CTAs per SM.  The kernel is bound by
 // instruction issue and by the chain of 2 x 128 dependent steps, so each thread
-// holds a large register tile (few warps repeat the per-step bookkeeping) and no
-// CTA-wide barrier sits inside the two sequential loops: both run as a dataflow
-// over shared memory.
+// holds a large register tile (few warps repeat the per-step bookkeeping) and
+// the steps are chained as tightly as the hardware allows.
 //  * Factorisation.  Warp w owns the columns w, w + 8, ... of the lower triangle;
 //    lane l holds their rows l + 32u in registers (40 values per thread: the
 //    32 x 8 blocks on or below the diagonal).  Column k of L is written to shared
-//    memory (packed lower triangle) by its warp, which then arrives on the
-//    column's own mbarrier; every warp waits for that mbarrier before it applies
-//    column k to its columns.  The warp that owns column k + 1 updates and
-//    publishes that column first and its other columns afterwards, so the chain
-//    column k -> column k + 1 is one warp's short path and the bulk of the
-//    rank-1 update runs behind it.
+//    memory (packed lower triangle) by its warp, which then arrives, without
+//    waiting, on a named barrier; the other warps wait on that barrier before
+//    they apply column k to their columns.  The warp that owns column k + 1
+//    updates and publishes that column first and its other columns afterwards,
+//    so the chain column k -> column k + 1 is one warp's short path and the bulk
+//    of the rank-1 update runs behind it.  (Measured on B200: a hand-over through
+//    a hardware barrier costs about 90 cycles, through an mbarrier about 220.)
 //  * Back substitution, 32 right-hand sides at a time.  Lane l holds the rows
-//    l + 32u of the solution, warp w their columns 4w .. 4w + 3.  Row i is
-//    published through shared memory and a per-row mbarrier in the same way: the
-//    lane that holds row i - 1 finishes it first, in every warp.
-// Every wait is bounded: on expiry the CTA stops waiting, finishes (with a wrong
-// result) and raises the time-out bit of the device status word.
+//    l + 32u of the solution, warp w their columns 4w .. 4w + 3, so a warp solves
+//    its columns without the others: the finished row i is broadcast by shuffles.
 #pragma once
 #include "common.cuh"
-#include "score_umma.cuh"
 
 namespace curdkv {
 
@@ -33,14 +29,10 @@ constexpr int kFactorThreads = 256;
 constexpr int kFactorWarps = kFactorThreads / 32;
 constexpr int kFactorD = 128;
 constexpr int kFactorPass = 32;                            // right-hand sides per back-substitution pass
-// dynamic shared memory: L (packed lower triangle, by columns), one pass of solved rows, 1 / L[i][i],
-// one mbarrier per column and per row, abort flag
+// dynamic shared memory: L (packed lower triangle, by columns), one pass of solved rows, 1 / L[i][i]
 constexpr size_t kFactorOffW = (size_t)kFactorD * (kFactorD + 1) / 2 * sizeof(double);
 constexpr size_t kFactorOffInv = kFactorOffW + (size_t)kFactorD * kFactorPass * sizeof(double);
-constexpr size_t kFactorOffColBar = kFactorOffInv + kFactorD * sizeof(double);
-constexpr size_t kFactorOffRowBar = kFactorOffColBar + kFactorD * sizeof(uint64_t);
-constexpr size_t kFactorOffAbort = kFactorOffRowBar + kFactorD * sizeof(uint64_t);
-constexpr size_t kFactorSmemBytes = kFactorOffAbort + 16;
+constexpr size_t kFactorSmemBytes = kFactorOffInv + kFactorD * sizeof(double);   // >= two staging areas
 
 struct FactorArgs {
   const float* partials;   // [batch*heads*segments][2][128][128]
@@ -51,39 +43,37 @@ struct FactorArgs {
   uint32_t* status;
 };
 
-struct FactorSync {
-  uint32_t col_bar, row_bar;                               // shared-memory addresses of the mbarrier arrays
-  volatile int* abort_flag;
-  uint32_t* status;
-  __device__ __forceinline__ void wait_col(int k) const {
-    umma::mbar_wait(col_bar + 8u * (uint32_t)k, 0u, abort_flag, status);
+// Copies what the factorisation reads of one stored 128 x 128 fp32 matrix into shared memory: rows
+// 0 .. 63 (32 KB), then columns 64 .. 127 of rows 64 .. 127 (16 KB).  Whole CTA; one cp.async group.
+constexpr int kFactorStageBytes = 48 * 1024;
+static_assert(2 * kFactorStageBytes <= kFactorSmemBytes, "two staging areas must fit");
+__device__ __forceinline__ void stage_partial(const float* src, unsigned char* stage, int tid) {
+  const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+  const unsigned char* g = reinterpret_cast<const unsigned char*>(src);
+  for (int q = tid; q < 2048; q += kFactorThreads)
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * q), "l"(g + 16 * q) : "memory");
+  for (int q = tid; q < 1024; q += kFactorThreads) {
+    const int row = 64 + (q >> 4), chunk = q & 15;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 32768u + 16u * q),
+                 "l"(g + (row * kFactorD + 64) * 4 + 16 * chunk)
+                 : "memory");
   }
-  // called by a whole warp after its stores: one arrival per warp
-  __device__ __forceinline__ void publish_col(int k) const {
-    __syncwarp();
-    if ((threadIdx.x & 31) == 0) umma::mbar_arrive(col_bar + 8u * (uint32_t)k);
-  }
-  __device__ __forceinline__ void wait_row(int i, uint32_t pass) const {
-    umma::mbar_wait(row_bar + 8u * (uint32_t)i, pass, abort_flag, status);
-  }
-  // called by the one lane of a warp that holds row i, after it has stored its part of the row
-  __device__ __forceinline__ void publish_row_part(int i) const { umma::mbar_arrive(row_bar + 8u * (uint32_t)i); }
-};
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// "Column k is in shared memory": hardware barrier 1 + k mod 8, on which the column's warp only
+// arrives and the seven others wait.  Every warp executes exactly one of the two per column, in
+// column order, so a barrier is never reused before its previous round has completed.
+__device__ __forceinline__ void column_arrive(int k) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(1 + (k & 7)), "r"(kFactorThreads) : "memory");
+}
+__device__ __forceinline__ void column_wait(int k) {
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + (k & 7)), "r"(kFactorThreads) : "memory");
+}
 
 // Column k of the packed triangle holds rows k .. 127; the returned offset already has k
 // subtracted, so that row i of column k is element tri_base(k) + i.
 __device__ __forceinline__ int tri_base(int k) { return k * (kFactorD - 1) - ((k * (k - 1)) >> 1); }
-
-// piv^(-1/2): fp32 seed and two Newton steps; out-of-range pivots take the library routine.
-__device__ __forceinline__ double pivot_rsqrt(double piv) {
-  if (piv > 1e-30 && piv < 1e30) {
-    double y = (double)rsqrtf((float)piv);
-    const double h = 0.5 * piv;
-    y = y * fma(-(h * y), y, 1.5);
-    return y * fma(-(h * y), y, 1.5);
-  }
-  return rsqrt(piv);
-}
 
 // m[u][v] is the element (l + 32u, w + 8v) of the matrix being eliminated; only the blocks on or
 // below the diagonal (u >= v / 4) are held.
@@ -92,11 +82,11 @@ __device__ __forceinline__ double pivot_rsqrt(double piv) {
 // rows k .. 127 (column k of L) to shared memory.
 template <int V>
 __device__ __forceinline__ void publish_column(const double (&m)[4][16], int k, double* Lt, double* invd,
-                                               const FactorSync& sync, int l, bool& bad) {
+                                               int l, bool& bad) {
   constexpr int U = V / 4;
   double piv = __shfl_sync(0xffffffffu, m[U][V], k & 31);
   if (!(piv > 0.0)) { piv = 1e-300; bad = true; }
-  const double rs = pivot_rsqrt(piv);
+  const double rs = rsqrt(piv);
   double* col = Lt + tri_base(k);
 #pragma unroll
   for (int u = U; u < 4; ++u) {
@@ -104,7 +94,7 @@ __device__ __forceinline__ void publish_column(const double (&m)[4][16], int k, 
     if (i >= k) col[i] = m[u][V] * rs;
   }
   if (l == (k & 31)) invd[k] = rs;                         // 1 / L[k][k]
-  sync.publish_col(k);
+  column_arrive(k);
 }
 
 // m[.][V] -= L[.][k] L[j][k] for this warp's column j = w + 8V.  MASK: the column may be finished
@@ -130,13 +120,13 @@ __device__ __forceinline__ void apply_from(double (&m)[4][16], const double (&li
 // Elimination steps k = 16*KH .. 16*KH + 15: only the columns v >= 2*KH and the row blocks
 // u >= KH / 2 still change, so the steps are compiled for exactly those.
 template <int KH>
-__device__ __forceinline__ void cholesky_steps(double (&m)[4][16], double* Lt, double* invd,
-                                               const FactorSync& sync, int w, int l, bool& bad) {
+__device__ __forceinline__ void cholesky_steps(double (&m)[4][16], double* Lt, double* invd, int w, int l,
+                                               bool& bad) {
   constexpr int D = kFactorD, V0 = 2 * KH, U0 = KH / 2;
 #pragma unroll 1
   for (int kt = 0; kt < 16; ++kt) {
     const int k = 16 * KH + kt;
-    sync.wait_col(k);
+    if ((k & 7) != w) column_wait(k);                      // its own column needs no waiting for
     const double* col = Lt + tri_base(k);
     double li[4];
 #pragma unroll
@@ -148,13 +138,13 @@ __device__ __forceinline__ void cholesky_steps(double (&m)[4][16], double* Lt, d
     if (owner_next) {
       if (vn == V0) {
         apply_column<V0, true>(m, li, col, k, w);
-        publish_column<V0>(m, kn, Lt, invd, sync, l, bad);
+        publish_column<V0>(m, kn, Lt, invd, l, bad);
       } else if (vn == V0 + 1) {
         apply_column<V0 + 1, true>(m, li, col, k, w);
-        publish_column<V0 + 1>(m, kn, Lt, invd, sync, l, bad);
+        publish_column<V0 + 1>(m, kn, Lt, invd, l, bad);
       } else if constexpr (V0 + 2 < 16) {
         apply_column<V0 + 2, false>(m, li, col, k, w);
-        publish_column<V0 + 2>(m, kn, Lt, invd, sync, l, bad);
+        publish_column<V0 + 2>(m, kn, Lt, invd, l, bad);
       }
     }
     // (the owner applies column k to the column it has just published once more: those registers are dead)
@@ -166,42 +156,31 @@ __device__ __forceinline__ void cholesky_steps(double (&m)[4][16], double* Lt, d
 
 // Back-substitution steps i = 32*IU + 31 .. 32*IU of one pass: only the rows of the blocks
 // u <= IU are still open.  x[u][c] is the element (l + 32u, column 4w + c of the pass) of the
-// right-hand side / solution; tb[u] = tri_base(l + 32u).  Row i - 1 sits in one lane of every
-// warp: that lane finishes and publishes its four columns before the warp does anything else.
+// right-hand side / solution; tb[u] = tri_base(l + 32u).  A warp solves its four columns on its
+// own: the finished row i is broadcast from the lane that holds it by shuffles, so the chain of
+// 128 dependent steps never leaves the warp.
 template <int IU>
-__device__ __forceinline__ void backsub_steps(double (&x)[4][4], const int (&tb)[4], const double* Lt,
-                                              double* Wt, const double* invd, const FactorSync& sync,
-                                              uint32_t pass, int w, int l) {
-#pragma unroll 1
+__device__ __forceinline__ void backsub_steps(double (&x)[4][4], const int (&tb)[4],
+                                              const double* __restrict__ Lt, double* __restrict__ Wt,
+                                              const double* __restrict__ invd, int w, int l) {
+#pragma unroll 2
   for (int it = 31; it >= 0; --it) {
     const int i = 32 * IU + it;
-    sync.wait_row(i, pass);
-    const double2 w01 = *reinterpret_cast<const double2*>(Wt + i * kFactorPass + 4 * w);
-    const double2 w23 = *reinterpret_cast<const double2*>(Wt + i * kFactorPass + 4 * w + 2);
-    const double wv[4] = {w01.x, w01.y, w23.x, w23.y};
-    const int in = i - 1;
-    if (in >= 0 && l == (in & 31)) {
-      const double lv = Lt[tri_base(in) + i], dinv = invd[in];   // L[i][i-1], 1 / L[i-1][i-1]
-      double o[4];
-      if (it > 0) {
+    const double dinv = invd[i];                           // 1 / L[i][i]
+    double wv[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) o[c] = (x[IU][c] - lv * wv[c]) * dinv;
-      } else if constexpr (IU > 0) {
+    for (int c = 0; c < 4; ++c) wv[c] = __shfl_sync(0xffffffffu, x[IU][c] * dinv, it);   // W[i][4w + c]
 #pragma unroll
-        for (int c = 0; c < 4; ++c) o[c] = (x[IU - 1][c] - lv * wv[c]) * dinv;
-      }
-      double* dst = Wt + in * kFactorPass + 4 * w;
-      *reinterpret_cast<double2*>(dst) = make_double2(o[0], o[1]);
-      *reinterpret_cast<double2*>(dst + 2) = make_double2(o[2], o[3]);
-      sync.publish_row_part(in);
+    for (int u = 0; u <= IU; ++u) {
+      double lv = Lt[tb[u] + i];                           // L[i][row]; finished rows read a neighbour: masked
+      if (u == IU && l >= it) lv = 0.0;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) x[u][c] -= lv * wv[c];
     }
-#pragma unroll
-    for (int u = 0; u <= IU; ++u) {                        // (a row just published is dead in x)
-      if (u < IU || l < it) {
-        const double lv = Lt[tb[u] + i];                   // L[i][row]
-#pragma unroll
-        for (int c = 0; c < 4; ++c) x[u][c] -= lv * wv[c];
-      }
+    if (l == it) {
+      double* dst = Wt + i * kFactorPass + 4 * w;
+      *reinterpret_cast<double2*>(dst) = make_double2(wv[0], wv[1]);
+      *reinterpret_cast<double2*>(dst + 2) = make_double2(wv[2], wv[3]);
     }
   }
 }
@@ -213,38 +192,42 @@ __global__ void __launch_bounds__(kFactorThreads, 2) whiten_factor_kernel(const 
   double* Lt = reinterpret_cast<double*>(fsm);                       // packed: L[i][k] at tri_base(k) + i
   double* Wt = reinterpret_cast<double*>(fsm + kFactorOffW);         // Wt[i*32 + c] = W[i][32*pass + c]
   double* invd = reinterpret_cast<double*>(fsm + kFactorOffInv);     // 1 / L[i][i]
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(fsm + kFactorOffAbort);
   __shared__ double red[kFactorWarps];
   const int tid = threadIdx.x, w = tid >> 5, l = tid & 31;
   const int p = blockIdx.x >> 1, tensor = blockIdx.x & 1;
   const int r = a.r;
-  const FactorSync sync{umma::smem_u32(fsm + kFactorOffColBar), umma::smem_u32(fsm + kFactorOffRowBar),
-                        abort_flag, a.status};
-  if (tid < D) {                                           // one arrival: the owning warp's
-    umma::mbar_init(sync.col_bar + 8u * (uint32_t)tid, 1);
-    umma::mbar_init(sync.row_bar + 8u * (uint32_t)tid, kFactorWarps);   // a row is spread over all warps
-  }
-  if (tid == 0) *abort_flag = 0;
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 
   // ---- M = sum of the segments' partial Gram matrices (segment order).  Element (i, j), i >= j,
   // is taken from row j of the stored matrix, so that a warp reads along a row; the part of a
-  // diagonal block above the diagonal mirrors the part below it.
+  // diagonal block above the diagonal mirrors the part below it.  The rows 0 .. 63 and the lower
+  // right quadrant of a stored matrix (all that this needs) are staged in shared memory by
+  // asynchronous copies, two segments in flight.
   double m[4][16];
 #pragma unroll
   for (int v = 0; v < 16; ++v)
 #pragma unroll
     for (int u = v / 4; u < 4; ++u) m[u][v] = 0.0;
+  const float* first = a.partials + (((size_t)p * a.segments) * 2 + tensor) * D * D;
+  stage_partial(first, fsm, tid);
+  if (a.segments > 1) stage_partial(first + 2 * D * D, fsm + kFactorStageBytes, tid);
   for (int g = 0; g < a.segments; ++g) {
-    const float* src = a.partials + (((size_t)p * a.segments + g) * 2 + tensor) * D * D;
+    if (g + 1 < a.segments) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    const float* top = reinterpret_cast<const float*>(fsm + (g & 1) * kFactorStageBytes);
+    const float* quad = top + 64 * D;
 #pragma unroll
     for (int v = 0; v < 16; ++v) {
 #pragma unroll
       for (int u = v / 4; u < 4; ++u) {
         const int i = l + 32 * u, j = w + 8 * v;
-        m[u][v] += (double)__ldg(src + min(i, j) * D + max(i, j));
+        const int lo = min(i, j), hi = max(i, j);
+        m[u][v] += (double)(v < 8 ? top[lo * D + hi] : quad[(lo - 64) * 64 + (hi - 64)]);
       }
     }
+    __syncthreads();
+    if (g + 2 < a.segments)
+      stage_partial(first + (size_t)(g + 2) * 2 * D * D, fsm + (g & 1) * kFactorStageBytes, tid);
   }
   double tr = 0.0;
 #pragma unroll
@@ -270,15 +253,15 @@ __global__ void __launch_bounds__(kFactorThreads, 2) whiten_factor_kernel(const 
   // ---- Cholesky by outer products: column k of L is published as soon as columns 0 .. k-1 have
   // been applied to it, and every thread subtracts L_ik L_jk from its elements right of it
   bool bad = false;
-  if (w == 0) publish_column<0>(m, 0, Lt, invd, sync, l, bad);
-  cholesky_steps<0>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<1>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<2>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<3>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<4>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<5>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<6>(m, Lt, invd, sync, w, l, bad);
-  cholesky_steps<7>(m, Lt, invd, sync, w, l, bad);
+  if (w == 0) publish_column<0>(m, 0, Lt, invd, l, bad);
+  cholesky_steps<0>(m, Lt, invd, w, l, bad);
+  cholesky_steps<1>(m, Lt, invd, w, l, bad);
+  cholesky_steps<2>(m, Lt, invd, w, l, bad);
+  cholesky_steps<3>(m, Lt, invd, w, l, bad);
+  cholesky_steps<4>(m, Lt, invd, w, l, bad);
+  cholesky_steps<5>(m, Lt, invd, w, l, bad);
+  cholesky_steps<6>(m, Lt, invd, w, l, bad);
+  cholesky_steps<7>(m, Lt, invd, w, l, bad);
   if (bad && l == 0) flag_status(a.status, CURDKV_DEV_NOT_SPD);
 
   // ---- back substitution L^T W = G, last row first, 32 columns of G per pass
@@ -296,17 +279,10 @@ __global__ void __launch_bounds__(kFactorThreads, 2) whiten_factor_kernel(const 
         x[u][c] = col < r ? (double)__ldg(a.G + (size_t)(l + 32 * u) * r + col) : 0.0;
       }
     __syncthreads();                                       // L complete; Wt of the previous pass stored
-    if (l == 31) {                                         // row 127 has nothing to subtract
-      const double dinv = invd[D - 1];
-      double* dst = Wt + (D - 1) * kFactorPass + 4 * w;
-      *reinterpret_cast<double2*>(dst) = make_double2(x[3][0] * dinv, x[3][1] * dinv);
-      *reinterpret_cast<double2*>(dst + 2) = make_double2(x[3][2] * dinv, x[3][3] * dinv);
-      sync.publish_row_part(D - 1);
-    }
-    backsub_steps<3>(x, tb, Lt, Wt, invd, sync, (uint32_t)pass, w, l);
-    backsub_steps<2>(x, tb, Lt, Wt, invd, sync, (uint32_t)pass, w, l);
-    backsub_steps<1>(x, tb, Lt, Wt, invd, sync, (uint32_t)pass, w, l);
-    backsub_steps<0>(x, tb, Lt, Wt, invd, sync, (uint32_t)pass, w, l);
+    backsub_steps<3>(x, tb, Lt, Wt, invd, w, l);
+    backsub_steps<2>(x, tb, Lt, Wt, invd, w, l);
+    backsub_steps<1>(x, tb, Lt, Wt, invd, w, l);
+    backsub_steps<0>(x, tb, Lt, Wt, invd, w, l);
     __syncthreads();
     const int width = min(kFactorPass, r - kFactorPass * pass);
     for (int e = tid; e < D * width; e += kFactorThreads) {
