@@ -3,23 +3,24 @@
 // adds the ridge, factors M = L L^T and solves L^T W = G, all in fp64 (the Gram
 // matrix squares the conditioning of K or V).  Writes W as fp32 [128][r].
 //
-// One CTA of 256 threads per matrix, two CTAs per SM.  The kernel is bound by
-// instruction issue and by the chain of 2 x 128 dependent steps, so each thread
-// holds a large register tile (few warps repeat the per-step bookkeeping) and
-// the steps are chained as tightly as the hardware allows.
-//  * Factorisation.  Warp w owns the columns w, w + 8, ... of the lower triangle;
-//    lane l holds their rows l + 32u in registers (40 values per thread: the
-//    32 x 8 blocks on or below the diagonal).  Column k of L is written to shared
-//    memory (packed lower triangle) by its warp, which then arrives, without
-//    waiting, on a named barrier; the other warps wait on that barrier before
-//    they apply column k to their columns.  The warp that owns column k + 1
-//    updates and publishes that column first and its other columns afterwards,
-//    so the chain column k -> column k + 1 is one warp's short path and the bulk
-//    of the rank-1 update runs behind it.  (Measured on B200: a hand-over through
-//    a hardware barrier costs about 90 cycles, through an mbarrier about 220.)
-//  * Back substitution, 32 right-hand sides at a time.  Lane l holds the rows
-//    l + 32u of the solution, warp w their columns 4w .. 4w + 3, so a warp solves
-//    its columns without the others: the finished row i is broadcast by shuffles.
+// One CTA of 256 threads per matrix, two CTAs per SM.  Three things of similar size bound the
+// kernel (measured on B200 by leaving each out in turn): the chain of dependent steps, the
+// shared-memory loads of the published columns and the fp64 pipe.  So each thread holds a large
+// register tile (few warps repeat the per-step loads and bookkeeping), the steps are chained as
+// tightly as the hardware allows, and two matrices per SM fill each other's gaps.
+//  * Factorisation.  Warp w owns two adjacent columns out of every 16 of the lower triangle; lane
+//    l holds their rows l + 32u in registers (40 values per thread: the blocks on or below the
+//    diagonal).  A finished pair of columns of L is written to shared memory (packed lower
+//    triangle) by its warp, which then arrives, without waiting, on a named barrier; the other
+//    warps wait on that barrier before they apply the pair to their columns.  The warp that owns
+//    the next pair updates, factors (inside the warp, by shuffles) and publishes it first and
+//    updates its other columns afterwards, so the chain pair -> next pair is one warp's short path
+//    and the bulk of the rank-2 update runs behind it.  (A hand-over through a hardware barrier
+//    costs about 90 cycles here, through an mbarrier about 220, which is why columns go in pairs
+//    and over barriers.)
+//  * Back substitution, 32 right-hand sides at a time.  Lane l holds the rows l + 32u of the
+//    solution, warp w their columns 4w .. 4w + 3, so a warp solves its columns without the
+//    others: the finished row i is broadcast by shuffles.
 #pragma once
 #include "common.cuh"
 
@@ -61,96 +62,113 @@ __device__ __forceinline__ void stage_partial(const float* src, unsigned char* s
   asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-// "Column k is in shared memory": hardware barrier 1 + k mod 8, on which the column's warp only
-// arrives and the seven others wait.  Every warp executes exactly one of the two per column, in
-// column order, so a barrier is never reused before its previous round has completed.
-__device__ __forceinline__ void column_arrive(int k) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(1 + (k & 7)), "r"(kFactorThreads) : "memory");
+// "Column pair p is in shared memory": hardware barrier 1 + p mod 8, on which the pair's warp only
+// arrives and the seven others wait.  Every warp executes exactly one of the two per pair, in
+// pair order, so a barrier is never reused before its previous round has completed.
+__device__ __forceinline__ void pair_arrive(int p) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(1 + (p & 7)), "r"(kFactorThreads) : "memory");
 }
-__device__ __forceinline__ void column_wait(int k) {
-  asm volatile("bar.sync %0, %1;" ::"r"(1 + (k & 7)), "r"(kFactorThreads) : "memory");
+__device__ __forceinline__ void pair_wait(int p) {
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + (p & 7)), "r"(kFactorThreads) : "memory");
 }
 
 // Column k of the packed triangle holds rows k .. 127; the returned offset already has k
 // subtracted, so that row i of column k is element tri_base(k) + i.
 __device__ __forceinline__ int tri_base(int k) { return k * (kFactorD - 1) - ((k * (k - 1)) >> 1); }
 
-// m[u][v] is the element (l + 32u, w + 8v) of the matrix being eliminated; only the blocks on or
-// below the diagonal (u >= v / 4) are held.
-//
-// The warp that owns column k = w + 8V scales it by the inverse root of its pivot and writes the
-// rows k .. 127 (column k of L) to shared memory.
-template <int V>
-__device__ __forceinline__ void publish_column(const double (&m)[4][16], int k, double* Lt, double* invd,
-                                               int l, bool& bad) {
-  constexpr int U = V / 4;
-  double piv = __shfl_sync(0xffffffffu, m[U][V], k & 31);
-  if (!(piv > 0.0)) { piv = 1e-300; bad = true; }
-  const double rs = rsqrt(piv);
-  double* col = Lt + tri_base(k);
+// m[u][c] is the element (l + 32u, column_of(w, c)) of the matrix being eliminated: a warp owns
+// the two adjacent columns 2w, 2w + 1 of every group of 16, and only the blocks on or below the
+// diagonal (u >= c / 4) are held.  Elements above the diagonal (inside the diagonal blocks) and
+// columns that have already been published are dead: they are updated along with the rest, with
+// whatever the loads return for them, and never read.
+__device__ __forceinline__ int column_of(int w, int c) { return 16 * (c >> 1) + 2 * w + (c & 1); }
+
+// The warp that owns the columns kA = 2p and kB = kA + 1 (its register columns 2P and 2P + 1)
+// finishes both and writes them to shared memory: column kA is scaled by the inverse root of its
+// pivot, applied to column kB, and column kB scaled in turn; all of it stays inside the warp.
+template <int P>
+__device__ __forceinline__ void publish_pair(const double (&m)[4][16], int p, double* Lt, double* invd, int l,
+                                             bool& bad) {
+  constexpr int U = P / 2, CA = 2 * P, CB = 2 * P + 1;
+  const int kA = 2 * p, kB = kA + 1;
+  double pivA = __shfl_sync(0xffffffffu, m[U][CA], kA & 31);
+  if (!(pivA > 0.0)) { pivA = 1e-300; bad = true; }
+  const double rsA = rsqrt(pivA);
+  double la[4], lb[4];
+#pragma unroll
+  for (int u = U; u < 4; ++u) la[u] = m[u][CA] * rsA;
+  const double lBA = __shfl_sync(0xffffffffu, la[U], kB & 31);   // L[kB][kA]
+#pragma unroll
+  for (int u = U; u < 4; ++u) lb[u] = m[u][CB] - la[u] * lBA;
+  double pivB = __shfl_sync(0xffffffffu, lb[U], kB & 31);
+  if (!(pivB > 0.0)) { pivB = 1e-300; bad = true; }
+  const double rsB = rsqrt(pivB);
+  double* colA = Lt + tri_base(kA);
+  double* colB = Lt + tri_base(kB);
 #pragma unroll
   for (int u = U; u < 4; ++u) {
     const int i = l + 32 * u;
-    if (i >= k) col[i] = m[u][V] * rs;
+    if (i >= kA) colA[i] = la[u];
+    if (i >= kB) colB[i] = lb[u] * rsB;
   }
-  if (l == (k & 31)) invd[k] = rs;                         // 1 / L[k][k]
-  column_arrive(k);
+  if (l == (kA & 31)) invd[kA] = rsA;                      // 1 / L[k][k]
+  if (l == (kB & 31)) invd[kB] = rsB;
+  pair_arrive(p);
 }
 
-// m[.][V] -= L[.][k] L[j][k] for this warp's column j = w + 8V.  MASK: the column may be finished
-// (j <= k), in which case nothing is subtracted.
-template <int V, bool MASK>
-__device__ __forceinline__ void apply_column(double (&m)[4][16], const double (&li)[4], const double* col, int k,
-                                             int w) {
-  const int j = w + 8 * V;
-  double lj = col[j];                                      // one value for the whole warp
-  if (MASK && j <= k) lj = 0.0;
+// m[.][C] -= L[.][kA] L[j][kA] + L[.][kB] L[j][kB] for this warp's column j = column_of(w, C).
+template <int C>
+__device__ __forceinline__ void apply_pair(double (&m)[4][16], const double (&liA)[4], const double (&liB)[4],
+                                           const double* colA, const double* colB, int w) {
+  const int j = column_of(w, C);
+  const double ljA = colA[j], ljB = colB[j];               // one value each for the whole warp
 #pragma unroll
-  for (int u = V / 4; u < 4; ++u) m[u][V] -= li[u] * lj;
+  for (int u = C / 4; u < 4; ++u) m[u][C] = fma(-liB[u], ljB, fma(-liA[u], ljA, m[u][C]));
 }
-template <int V>
-__device__ __forceinline__ void apply_from(double (&m)[4][16], const double (&li)[4], const double* col, int k,
-                                           int w) {
-  if constexpr (V < 16) {
-    apply_column<V, false>(m, li, col, k, w);
-    apply_from<V + 1>(m, li, col, k, w);
+template <int C>
+__device__ __forceinline__ void apply_pair_from(double (&m)[4][16], const double (&liA)[4],
+                                                const double (&liB)[4], const double* colA, const double* colB,
+                                                int w) {
+  if constexpr (C < 16) {
+    apply_pair<C>(m, liA, liB, colA, colB, w);
+    apply_pair_from<C + 1>(m, liA, liB, colA, colB, w);
   }
 }
 
-// Elimination steps k = 16*KH .. 16*KH + 15: only the columns v >= 2*KH and the row blocks
-// u >= KH / 2 still change, so the steps are compiled for exactly those.
+// Elimination by the column pairs p = 8*KH .. 8*KH + 7 (columns 16*KH .. 16*KH + 15): only the
+// register columns c >= 2*KH and the row blocks u >= KH / 2 still change, so the steps are
+// compiled for exactly those.  Loads of rows or columns before the pair stay inside the packed
+// triangle (they reach at most 31 elements back) and only feed dead elements.
 template <int KH>
-__device__ __forceinline__ void cholesky_steps(double (&m)[4][16], double* Lt, double* invd, int w, int l,
+__device__ __forceinline__ void cholesky_pairs(double (&m)[4][16], double* Lt, double* invd, int w, int l,
                                                bool& bad) {
-  constexpr int D = kFactorD, V0 = 2 * KH, U0 = KH / 2;
+  constexpr int U0 = KH / 2;
 #pragma unroll 1
-  for (int kt = 0; kt < 16; ++kt) {
-    const int k = 16 * KH + kt;
-    if ((k & 7) != w) column_wait(k);                      // its own column needs no waiting for
-    const double* col = Lt + tri_base(k);
-    double li[4];
+  for (int pt = 0; pt < 8; ++pt) {
+    const int p = 8 * KH + pt, kA = 2 * p;
+    if (pt != w) pair_wait(p);                             // its own pair needs no waiting for
+    const double* colA = Lt + tri_base(kA);
+    const double* colB = colA + (kFactorD - 1 - kA);       // tri_base(kA + 1)
+    double liA[4], liB[4];
 #pragma unroll
-    for (int u = U0; u < 4; ++u) li[u] = col[l + 32 * u];  // rows above k read a neighbouring column: masked
-    if (l + 32 * U0 <= k) li[U0] = 0.0;                    // rows up to k are finished
-    // the owner of column k + 1 brings it up to date and publishes it before anything else
-    const int kn = k + 1, vn = kn >> 3;                    // vn is V0, V0 + 1 or (last step) V0 + 2
-    const bool owner_next = kn < D && (kn & 7) == w;
-    if (owner_next) {
-      if (vn == V0) {
-        apply_column<V0, true>(m, li, col, k, w);
-        publish_column<V0>(m, kn, Lt, invd, l, bad);
-      } else if (vn == V0 + 1) {
-        apply_column<V0 + 1, true>(m, li, col, k, w);
-        publish_column<V0 + 1>(m, kn, Lt, invd, l, bad);
-      } else if constexpr (V0 + 2 < 16) {
-        apply_column<V0 + 2, false>(m, li, col, k, w);
-        publish_column<V0 + 2>(m, kn, Lt, invd, l, bad);
+    for (int u = U0; u < 4; ++u) {
+      liA[u] = colA[l + 32 * u];
+      liB[u] = colB[l + 32 * u];
+    }
+    // the owner of the next pair brings it up to date and publishes it before anything else
+    if (pt + 1 == w) {
+      apply_pair<2 * KH>(m, liA, liB, colA, colB, w);
+      apply_pair<2 * KH + 1>(m, liA, liB, colA, colB, w);
+      publish_pair<KH>(m, p + 1, Lt, invd, l, bad);
+    } else if (pt == 7 && w == 0) {
+      if constexpr (KH + 1 < 8) {
+        apply_pair<2 * KH + 2>(m, liA, liB, colA, colB, w);
+        apply_pair<2 * KH + 3>(m, liA, liB, colA, colB, w);
+        publish_pair<KH + 1>(m, p + 1, Lt, invd, l, bad);
       }
     }
-    // (the owner applies column k to the column it has just published once more: those registers are dead)
-    apply_column<V0, true>(m, li, col, k, w);
-    apply_column<V0 + 1, true>(m, li, col, k, w);
-    apply_from<V0 + 2>(m, li, col, k, w);
+    // (the owner applies the pair once more to the columns it has just published: dead registers)
+    apply_pair_from<2 * KH>(m, liA, liB, colA, colB, w);
   }
 }
 
@@ -171,7 +189,7 @@ __device__ __forceinline__ void backsub_steps(double (&x)[4][4], const int (&tb)
 #pragma unroll
     for (int c = 0; c < 4; ++c) wv[c] = __shfl_sync(0xffffffffu, x[IU][c] * dinv, it);   // W[i][4w + c]
 #pragma unroll
-    for (int u = 0; u <= IU; ++u) {
+    for (int u = IU; u >= 0; --u) {                        // block IU first: the next step waits for it
       double lv = Lt[tb[u] + i];                           // L[i][row]; finished rows read a neighbour: masked
       if (u == IU && l >= it) lv = 0.0;
 #pragma unroll
@@ -220,7 +238,7 @@ __global__ void __launch_bounds__(kFactorThreads, 2) whiten_factor_kernel(const 
     for (int v = 0; v < 16; ++v) {
 #pragma unroll
       for (int u = v / 4; u < 4; ++u) {
-        const int i = l + 32 * u, j = w + 8 * v;
+        const int i = l + 32 * u, j = column_of(w, v);
         const int lo = min(i, j), hi = max(i, j);
         m[u][v] += (double)(v < 8 ? top[lo * D + hi] : quad[(lo - 64) * 64 + (hi - 64)]);
       }
@@ -232,7 +250,7 @@ __global__ void __launch_bounds__(kFactorThreads, 2) whiten_factor_kernel(const 
   double tr = 0.0;
 #pragma unroll
   for (int v = 0; v < 16; ++v)
-    if (l + 32 * (v / 4) == w + 8 * v) tr += m[v / 4][v];  // diagonal elements sit in the blocks u = v / 4
+    if (l + 32 * (v / 4) == column_of(w, v)) tr += m[v / 4][v];   // the diagonal sits in the blocks u = v / 4
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
   if (l == 0) red[w] = tr;
@@ -248,20 +266,20 @@ __global__ void __launch_bounds__(kFactorThreads, 2) whiten_factor_kernel(const 
   const double lambda = a.ridge * trace / D;
 #pragma unroll
   for (int v = 0; v < 16; ++v)
-    if (l + 32 * (v / 4) == w + 8 * v) m[v / 4][v] += lambda;
+    if (l + 32 * (v / 4) == column_of(w, v)) m[v / 4][v] += lambda;
 
   // ---- Cholesky by outer products: column k of L is published as soon as columns 0 .. k-1 have
   // been applied to it, and every thread subtracts L_ik L_jk from its elements right of it
   bool bad = false;
-  if (w == 0) publish_column<0>(m, 0, Lt, invd, l, bad);
-  cholesky_steps<0>(m, Lt, invd, w, l, bad);
-  cholesky_steps<1>(m, Lt, invd, w, l, bad);
-  cholesky_steps<2>(m, Lt, invd, w, l, bad);
-  cholesky_steps<3>(m, Lt, invd, w, l, bad);
-  cholesky_steps<4>(m, Lt, invd, w, l, bad);
-  cholesky_steps<5>(m, Lt, invd, w, l, bad);
-  cholesky_steps<6>(m, Lt, invd, w, l, bad);
-  cholesky_steps<7>(m, Lt, invd, w, l, bad);
+  if (w == 0) publish_pair<0>(m, 0, Lt, invd, l, bad);
+  cholesky_pairs<0>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<1>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<2>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<3>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<4>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<5>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<6>(m, Lt, invd, w, l, bad);
+  cholesky_pairs<7>(m, Lt, invd, w, l, bad);
   if (bad && l == 0) flag_status(a.status, CURDKV_DEV_NOT_SPD);
 
   // ---- back substitution L^T W = G, last row first, 32 columns of G per pass
