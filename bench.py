@@ -28,7 +28,7 @@ NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one sketch-kernel launch, from the ncu
 # capture summarised under profiles/ (None: not captured for the kernel as it stands)
-TRAFFIC_BYTES = {"cfg2": 1.0776e9, "cfg3": 16 * 1.0776e9}   # cfg3 = cfg2's capture x 16 head-tokens
+TRAFFIC_BYTES = {"cfg2": 1.0787e9, "cfg3": 16 * 1.0787e9}   # cfg3 = cfg2's capture x 16 head-tokens
 FALLBACK_HBM_GBS = 6650.0
 
 
