@@ -177,14 +177,45 @@ __global__ void __launch_bounds__(256) cache_fill_holes_kernel(const CacheView c
   // copy mover i into hole i: a half-warp per tensor row (K in lanes 0-15, V in lanes 16-31)
   const int half = lane >> 4, l16 = lane & 15, chunks = d >> 3;
   __nv_bfloat16* rows = (half ? c.V : c.K) + (size_t)p * c.capacity * d;
+  float* raw = c.raw + (size_t)p * c.capacity;
+  int32_t* pos = c.pos + (size_t)p * c.capacity;
+  if (chunks == 16) {
+    // d = 128: one 16-byte piece per lane and row; four rows per warp in flight (sources and
+    // destinations are disjoint slot ranges, so the order of the copies is free)
+    for (int i0 = warp; i0 < moves; i0 += 32) {
+      int src[4], dst[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int i = min(i0 + 8 * q, moves - 1);
+        src[q] = ix[first_mover + i];
+        dst[q] = my_holes[i];
+      }
+      uint4 v[4];
+      float rv = 0.f;
+      int pv = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        v[q] = *reinterpret_cast<const uint4*>(rows + (size_t)src[q] * d + l16 * 8);
+        if (lane == q) { rv = raw[src[q]]; pv = pos[src[q]]; }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (i0 + 8 * q < moves) {
+          reinterpret_cast<uint4*>(rows + (size_t)dst[q] * d)[l16] = v[q];
+          if (lane == q) { raw[dst[q]] = rv; pos[dst[q]] = pv; }
+        }
+      }
+    }
+    return;
+  }
   for (int i = warp; i < moves; i += 8) {
     const int src = ix[first_mover + i], dst = my_holes[i];
     for (int ch = l16; ch < chunks; ch += 16)
       reinterpret_cast<uint4*>(rows + (size_t)dst * d)[ch] =
           *reinterpret_cast<const uint4*>(rows + (size_t)src * d + ch * 8);
     if (lane == 0) {
-      c.raw[(size_t)p * c.capacity + dst] = c.raw[(size_t)p * c.capacity + src];
-      c.pos[(size_t)p * c.capacity + dst] = c.pos[(size_t)p * c.capacity + src];
+      raw[dst] = raw[src];
+      pos[dst] = pos[src];
     }
   }
 }

@@ -466,10 +466,11 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
   if (cudaFuncSetAttribute(select_fixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSelStageBytes + kSelListBytes) != cudaSuccess)
     return CURDKV_ERR_CUDA;
-  // rows of up to 16384 tokens run as CTAs of 512 threads with a smaller list, two per SM
-  const bool small_rows = desc->n_max <= 16384;
-  const int sel_threads = small_rows ? 512 : kSelThreads;
-  const int list_cap = small_rows ? kSelListCap / 2 : kSelListCap;
+  // shorter rows run as smaller CTAs with a smaller list, several per SM: the many short phases
+  // of a row then overlap with those of its neighbours
+  int sel_threads = kSelThreads, list_cap = kSelListCap;
+  if (desc->n_max <= 4096) { sel_threads = 256; list_cap = kSelListCap / 4; }
+  else if (desc->n_max <= 16384) { sel_threads = 512; list_cap = kSelListCap / 2; }
   select_fixed_kernel<<<(unsigned)P, sel_threads, stage_bytes + (size_t)list_cap * 8, stream>>>(
       scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,
       (int)(stage_bytes / sizeof(uint4)), list_cap, idx, head_counts, head_offsets);

@@ -137,7 +137,8 @@ __device__ __forceinline__ void pick_digit_impl(const uint32_t* hist, uint32_t r
 }
 __device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
   if (blockDim.x == 1024) pick_digit_impl<4>(hist, remaining, sm);
-  else pick_digit_impl<8>(hist, remaining, sm);
+  else if (blockDim.x == 512) pick_digit_impl<8>(hist, remaining, sm);
+  else pick_digit_impl<16>(hist, remaining, sm);
 }
 
 // Number of keys of `hist` in bins above `digit`.  Whole CTA; every thread gets the sum.
@@ -160,7 +161,9 @@ __device__ __forceinline__ uint32_t count_above_impl(const uint32_t* hist, uint3
   return t;
 }
 __device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
-  return blockDim.x == 1024 ? count_above_impl<4>(hist, digit, sm) : count_above_impl<8>(hist, digit, sm);
+  if (blockDim.x == 1024) return count_above_impl<4>(hist, digit, sm);
+  if (blockDim.x == 512) return count_above_impl<8>(hist, digit, sm);
+  return count_above_impl<16>(hist, digit, sm);
 }
 
 // Rank keys of one row, four tokens at a time ("quad" q holds tokens
@@ -470,7 +473,7 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
 }
 
 // ---------------------------------------------------------------------------
-// Fixed per-head budget.  grid = batch*heads, block = 1024 or 512, dynamic shared
+// Fixed per-head budget.  grid = batch*heads, block = 1024, 512 or 256, dynamic shared
 // memory = 16 * stage_quads bytes (0: rows are read from global memory) followed
 // by one candidate list of list_cap entries.
 // ---------------------------------------------------------------------------
