@@ -147,6 +147,8 @@ def run_cuda(args):
     dev = torch.device("cuda", local)
 
     w = rank_workload(synth.CONFIGS[args.workload], rank)
+    if args.batch > 0:                                     # the same recipe at another batch size
+        w = synth.shrink(w, batch=args.batch)
     K, V, seqlens = synth.make_kv(w, dev)
     G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
     sl = None if seqlens is None else torch.as_tensor(seqlens, device=dev)
@@ -273,7 +275,7 @@ def run_cuda(args):
             "bound": "hbm", "kernel": "sketch_umma_kernel (inside curdkv_score)",
             "achieved": sketch_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
             "unit": "GB/s", "frac": sketch_gbs / peak,
-            "traffic": None if args.whiten else TRAFFIC_BYTES.get(w.name),
+            "traffic": None if (args.whiten or args.batch > 0) else TRAFFIC_BYTES.get(w.name),
             "algorithmic_bytes_per_launch": pass_bytes, "ms_per_launch": sketch_ms,
             "timer": "CUDA events recorded by the library around the kernel, mean over the timed steps",
         },
@@ -571,6 +573,8 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     w = synth.CONFIGS[args.workload]
+    if args.batch > 0:
+        w = synth.shrink(w, batch=args.batch)
     elems = sample_elements(w, core_seconds=20.0)
     Ku, Vu, sl = oracle_sample(w, elems)
     G = synth.make_G(w.d, w.r, seed=0)
@@ -604,6 +608,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode", "evict"])
+    ap.add_argument("--batch", type=int, default=0,
+                    help="sequences per layer instead of the workload's own (cfg1-cfg5 only); 0 keeps it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
                     help="--workload decode: compress inside the cache (unordered) or copy in order")
