@@ -5,9 +5,14 @@
 //
 // One CTA per (problem, block of 128 queries), one pass over the keys with an
 // online softmax on the tensor cores:
-//   S = Q K_t^T per 128-key tile (tcgen05.mma, fp32 in TMEM, double-buffered);
-//   P = exp2(S - m) split into bf16 P_hi + P_lo in shared memory;
-//   O_g += P_hi V_t + P_lo V_t (V tile read MN-major), row sums l_g.
+//   S = Q K_t^T per 128-key tile (tcgen05.mma, fp32 in TMEM, one buffer per group);
+//   P = exp2(S - m) split into bf16 P_hi + P_lo, written back over S in TMEM;
+//   O_g += P_hi V_t + P_lo V_t (A operand read from TMEM, V tile MN-major in
+//   shared memory), row sums l_g.
+// Keeping P in TMEM matters: an M = N = 128, K = 16 MMA with both operands in
+// shared memory reads 8 KB per 64 cycles, all the 128 B/clk an SM has, so a P that
+// went through shared memory (64 KB written and read again per tile, next to
+// the 64 KB the TMA brings in) made shared memory the bound, not the tensor pipe.
 // Warp 0 feeds the TMA ring, warp 1 issues the MMAs, and two groups of four
 // softmax warps take alternate key tiles.  Each group runs its own online
 // softmax (running maximum m_g, sum l_g, accumulator O_g in TMEM); the running
@@ -34,14 +39,14 @@ struct AttnArgs {
 };
 
 constexpr int kAttnThreads = 320;                          // TMA, MMA, 2 x 4 softmax warps
-constexpr int kAttnRing = 2;
+constexpr int kAttnRing = 5;
 constexpr int kAttnQ = 0;
-constexpr int kAttnP = kSlotBytes;                         // P[buf]: hi at +0, lo at +kSlotBytes
-constexpr int kAttnPBytes = 2 * kSlotBytes;
-constexpr int kAttnSlot0 = kAttnP + 2 * kAttnPBytes;
+constexpr int kAttnSlot0 = kSlotBytes;
 constexpr int kAttnBar = kAttnSlot0 + kAttnRing * kSlotBytes;
 constexpr int kAttnDynamic = kAttnBar + 256 + 1024;
-constexpr int kAttnTmemCols = 512;                         // S[2] at 0 / 128, O[2] at 256 / 384
+// TMEM columns: S of group g at 128 g, overwritten in place by its P (bf16 pairs: P_hi in the
+// first 64 columns, P_lo in the last 64); O of group g at 256 + 128 g
+constexpr int kAttnTmemCols = 512;
 constexpr float kAttnMaxSlack = 8.f;                       // log2 units a tile may exceed the running maximum
 
 // P V: A = P K-major, B = V tile MN-major (contraction over the keys)
@@ -58,6 +63,26 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
       "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]), "r"(u[16]),
       "r"(u[17]), "r"(u[18]), "r"(u[19]), "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]), "r"(u[24]),
       "r"(u[25]), "r"(u[26]), "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31])
+      : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's TMEM lane, written.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&u)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), "r"(u[8]),
+      "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15])
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem], bf16 inputs, fp32 accumulate, M = 128: row i of A is TMEM lane
+// i, its K = 16 elements sit in 8 consecutive 32-bit columns.
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() {
@@ -89,13 +114,11 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kAttnRing + s); };
   auto s_full_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + s); };
-  auto s_empty_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 2 + s); };
-  auto p_ready_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 4 + s); };
-  auto p_empty_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 6 + s); };
-  const uint32_t q_full_bar = bar0 + 8u * (2 * kAttnRing + 8);
-  const uint32_t o_full_bar = bar0 + 8u * (2 * kAttnRing + 9);
-  const uint32_t drain_bar = bar0 + 8u * (2 * kAttnRing + 10);
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + kAttnBar + 8 * (2 * kAttnRing + 11));
+  auto p_ready_bar = [&](int s) { return bar0 + 8u * (2 * kAttnRing + 2 + s); };
+  const uint32_t q_full_bar = bar0 + 8u * (2 * kAttnRing + 4);
+  const uint32_t o_full_bar = bar0 + 8u * (2 * kAttnRing + 5);
+  const uint32_t drain_bar = bar0 + 8u * (2 * kAttnRing + 6);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(base_ptr + kAttnBar + 8 * (2 * kAttnRing + 7));
   __shared__ float xchg[2][kTileRows];                     // running maximum and row sum of the second group
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -121,9 +144,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     for (int s = 0; s < kAttnRing; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(s_full_bar(s), 1);
-      mbar_init(s_empty_bar(s), 128);
       mbar_init(p_ready_bar(s), 128);
-      mbar_init(p_empty_bar(s), 1);
     }
     mbar_init(q_full_bar, 1);
     mbar_init(o_full_bar, 1);
@@ -144,7 +165,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
   const uint32_t tmem_base = *tmem_holder;
 
   // Tiles go through the ring in the order the MMA issuer consumes them:
-  //   K_0, then for every t: K_{t+1} (if any), V_t.
+  //   K_0, K_1, then for every t: V_t, K_{t+2} (if any).
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -167,9 +188,10 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         ++it;
       };
       load(&map_k, 0);
+      if (ok && T > 1) load(&map_k, 1);
       for (int t = 0; ok && t < T; ++t) {
-        if (t + 1 < T) load(&map_k, t + 1);
-        if (ok) load(&map_v, t);
+        load(&map_v, t);
+        if (ok && t + 2 < T) load(&map_k, t + 2);
       }
       if (!ok) {
         const uint32_t pending = it < (uint32_t)kAttnRing ? it : (uint32_t)kAttnRing;
@@ -185,12 +207,10 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     if (lane == 0) {
       constexpr uint32_t idesc_s = instr_desc_bf16(128);
       constexpr uint32_t idesc_pv = instr_desc_pv();
-      uint32_t it = 0, job = 0;
+      uint32_t it = 0;
       bool ok = mbar_wait(q_full_bar, 0, abort_flag, a.status);
       tc_fence_after();
-      auto issue_s = [&]() {                               // S[job & 1] = Q K^T for the next K tile
-        const uint32_t buf = job & 1u;
-        if (!(ok = mbar_wait(s_empty_bar(buf), ((job >> 1) & 1u) ^ 1u, abort_flag, a.status))) return;
+      auto issue_s = [&](uint32_t buf) {                   // S[buf] = Q K^T for the next K tile of the ring
         const int slot = it % kAttnRing;
         if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status))) return;
         tc_fence_after();
@@ -204,12 +224,12 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         tc_commit(empty_bar(slot));
         tc_commit(s_full_bar(buf));
         ++it;
-        ++job;
       };
-      if (ok) issue_s();                                   // tile 0
+      // A group's S buffer is taken over by its P; S_{t+2} goes into it right behind P_t V_t (the
+      // tensor pipe runs the MMAs of one thread in order, so the product has read P by then).
+      if (ok) issue_s(0);                                  // tile 0
+      if (ok && T > 1) issue_s(1);                         // tile 1
       for (int t = 0; ok && t < T; ++t) {
-        if (t + 1 < T) issue_s();
-        if (!ok) break;
         const int slot = it % kAttnRing;
         if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status))) break;
         const int rows = min(kTileRows, n - t * kTileRows);
@@ -222,21 +242,20 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                                           j * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        const uint32_t pbuf = (uint32_t)t & 1u;            // the group that owns this tile, its P and O
-        if (!(ok = mbar_wait(p_ready_bar(pbuf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status))) break;
+        const uint32_t buf = (uint32_t)t & 1u;             // the group that owns this tile, its P and O
+        if (!(ok = mbar_wait(p_ready_bar(buf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status))) break;
         tc_fence_after();
         const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
         for (int part = 0; part < 2; ++part) {             // P_hi, then P_lo
-          const uint32_t p_base = base + kAttnP + pbuf * kAttnPBytes + part * kSlotBytes;
-          for (int g = 0; g < groups; ++g) {               // 16 keys per MMA
-            const uint32_t poff = (g >> 2) * kHalfBytes + (g & 3) * 32;
-            tc_mma_bf16(tmem_base + 256u + pbuf * 128u, smem_desc_sw128(p_base + poff),
-                        smem_desc_mn_sw128(v_base + g * 2048), idesc_pv, (t > 1 || part > 0 || g > 0) ? 1u : 0u);
-          }
+          const uint32_t p_tmem = tmem_base + buf * 128u + part * 64u;
+          for (int g = 0; g < groups; ++g)                 // 16 keys per MMA: 8 columns of P
+            tc_mma_bf16_ts(tmem_base + 256u + buf * 128u, p_tmem + 8u * g,
+                           smem_desc_mn_sw128(v_base + g * 2048), idesc_pv,
+                           (t > 1 || part > 0 || g > 0) ? 1u : 0u);
         }
         tc_commit(empty_bar(slot));
-        tc_commit(p_empty_bar(pbuf));
         ++it;
+        if (t + 2 < T) issue_s(buf);
       }
       if (ok) tc_commit(o_full_bar);
       if (!ok) {
@@ -258,80 +277,73 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     float top = (extra > 0 && group == 0) ? 0.f : -INFINITY;
     float sum = (extra > 0 && group == 0) ? (float)extra : 0.f;
     bool has_o = false, ok = true;                         // has_o: O_group holds at least one product
-    unsigned char* Pbuf = base_ptr + kAttnP + group * kAttnPBytes;
     const uint32_t s_addr = lane_addr + group * 128u, o_addr = lane_addr + 256u + group * 128u;
     for (int t = group; ok && t < T; t += 2) {
       ok = mbar_wait(s_full_bar(group), (uint32_t)(t >> 1) & 1u, abort_flag, a.status);
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const int valid = n - t * kTileRows;                 // keys of this tile that exist
-      float tile_top = -INFINITY;
-#pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        float v[32];
-        tmem_ld32(s_addr + c0, v);
-        tmem_ld_wait();
-        if (valid >= kTileRows) {
+      // the whole row of S into registers: its columns are about to take P
+      float v[128];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) tile_top = fmaxf(tile_top, v[c] * sc);
+      for (int c0 = 0; c0 < 128; c0 += 32) tmem_ld32(s_addr + c0, *reinterpret_cast<float(*)[32]>(v + c0));
+      tmem_ld_wait();
+      float tile_top = -INFINITY;
+      if (valid >= kTileRows) {
+        // max_c (v_c * sc) = sc * max_c v_c or sc * min_c v_c
+        float ext = v[0];
+        if (sc >= 0.f) {
+#pragma unroll
+          for (int c = 1; c < 128; ++c) ext = fmaxf(ext, v[c]);
         } else {
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (c0 + c < valid) tile_top = fmaxf(tile_top, v[c] * sc);
+          for (int c = 1; c < 128; ++c) ext = fminf(ext, v[c]);
         }
+        tile_top = ext * sc;
+      } else {
+#pragma unroll
+        for (int c = 0; c < 128; ++c)
+          if (c < valid) tile_top = fmaxf(tile_top, v[c] * sc);
       }
       // move the running maximum only when the tile exceeds it by more than the slack
       const bool move = tile_top > top + kAttnMaxSlack || top == -INFINITY;
       const float new_top = move ? fmaxf(top, tile_top) : top;
       const float alpha = move ? fast_exp2(top - new_top) : 1.f;      // 0 when top was -inf
-      if (t >= 2) {                                        // this group's previous product has retired
-        ok = mbar_wait(p_empty_bar(group), (uint32_t)((t >> 1) - 1) & 1u, abort_flag, a.status);
-        if (!(ok = __all_sync(0xffffffffu, ok))) break;
-        tc_fence_after();
-      }
+      // (this group's previous product has retired: S of this tile was issued behind it)
       if (has_o && __any_sync(0xffffffffu, move)) {        // rescale O_group in TMEM
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
-          float v[32];
-          tmem_ld32(o_addr + c0, v);
+          float o[32];
+          tmem_ld32(o_addr + c0, o);
           tmem_ld_wait();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) v[c] *= alpha;
-          tmem_st32(o_addr + c0, v);
+          for (int c = 0; c < 32; ++c) o[c] *= alpha;
+          tmem_st32(o_addr + c0, o);
         }
         tmem_st_wait();
       }
       sum *= alpha;
       top = new_top;
-#pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        float v[32];
-        tmem_ld32(s_addr + c0, v);
-        tmem_ld_wait();
+      const bool ragged = valid < kTileRows;               // last tile of the cache: mask by index
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {                      // 8 keys -> one 16-byte chunk of P_hi, P_lo
-          uint32_t hi[4], lo[4];
+      for (int c0 = 0; c0 < 128; c0 += 32) {               // 32 keys -> 16 columns of P_hi and of P_lo
+        uint32_t hi[16], lo[16];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int c = g * 8 + e * 2;
-            float w0 = fast_exp2(fmaf(v[c], sc, -top)), w1 = fast_exp2(fmaf(v[c + 1], sc, -top));
-            if (valid < kTileRows) {                       // last tile of the cache: mask by index
-              if (c0 + c >= valid) w0 = 0.f;
-              if (c0 + c + 1 >= valid) w1 = 0.f;
-            }
-            sum += w0 + w1;                                // equals the bf16 pairs to 2^-17
-            split_bf16x2(w0, w1, hi[e], lo[e]);
+        for (int e = 0; e < 16; ++e) {
+          const int c = c0 + 2 * e;
+          float w0 = fast_exp2(fmaf(v[c], sc, -top)), w1 = fast_exp2(fmaf(v[c + 1], sc, -top));
+          if (ragged) {
+            if (c >= valid) w0 = 0.f;
+            if (c + 1 >= valid) w1 = 0.f;
           }
-          const int key = c0 + g * 8;                      // first key of the chunk inside the tile
-          const uint32_t off = (uint32_t)(key >> 6) * kHalfBytes + (uint32_t)r * 128u +
-                               ((((uint32_t)(key & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4);
-          *reinterpret_cast<uint4*>(Pbuf + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(Pbuf + kSlotBytes + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          sum += w0 + w1;                                  // equals the bf16 pairs to 2^-17
+          split_bf16x2(w0, w1, hi[e], lo[e]);
         }
+        tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
+        tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
       }
+      tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(s_empty_bar(group));
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(p_ready_bar(group));
       has_o = true;
     }
