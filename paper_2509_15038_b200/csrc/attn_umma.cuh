@@ -95,6 +95,40 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Packed fp32 pairs (one instruction for two lanes of arithmetic) and three-input max / min.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t r, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float d;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 // Two weights -> packed bf16 (hi) and packed bf16 of the remainders (lo).
 __device__ __forceinline__ void split_bf16x2(float w0, float w1, uint32_t& hi, uint32_t& lo) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
@@ -290,16 +324,21 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       tmem_ld_wait();
       float tile_top = -INFINITY;
       if (valid >= kTileRows) {
-        // max_c (v_c * sc) = sc * max_c v_c or sc * min_c v_c
-        float ext = v[0];
+        // max_c (v_c * sc) = sc * max_c v_c or sc * min_c v_c; four independent chains
+        float ext[4] = {v[0], v[1], v[2], v[3]};
         if (sc >= 0.f) {
 #pragma unroll
-          for (int c = 1; c < 128; ++c) ext = fmaxf(ext, v[c]);
+          for (int c = 4; c < 128; c += 8)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ext[j] = c + 2 * j + 1 < 128 ? max3(ext[j], v[c + 2 * j], v[c + 2 * j + 1]) : ext[j];
+          tile_top = fmaxf(fmaxf(ext[0], ext[1]), fmaxf(ext[2], ext[3])) * sc;
         } else {
 #pragma unroll
-          for (int c = 1; c < 128; ++c) ext = fminf(ext, v[c]);
+          for (int c = 4; c < 128; c += 8)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ext[j] = c + 2 * j + 1 < 128 ? min3(ext[j], v[c + 2 * j], v[c + 2 * j + 1]) : ext[j];
+          tile_top = fminf(fminf(ext[0], ext[1]), fminf(ext[2], ext[3])) * sc;
         }
-        tile_top = ext * sc;
       } else {
 #pragma unroll
         for (int c = 0; c < 128; ++c)
@@ -324,23 +363,51 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       }
       sum *= alpha;
       top = new_top;
-      const bool ragged = valid < kTileRows;               // last tile of the cache: mask by index
+      if (valid >= kTileRows) {
+        // full tile: the arithmetic runs on packed pairs of keys
+        const uint64_t sc2 = pack2(sc, sc), ntop2 = pack2(-top, -top);
+        uint64_t part[4] = {0ull, 0ull, 0ull, 0ull};       // eight partial row sums
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {               // 32 keys -> 16 columns of P_hi and of P_lo
-        uint32_t hi[16], lo[16];
+        for (int c0 = 0; c0 < 128; c0 += 32) {             // 32 keys -> 16 columns of P_hi and of P_lo
+          uint32_t hi[16], lo[16];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const int c = c0 + 2 * e;
-          float w0 = fast_exp2(fmaf(v[c], sc, -top)), w1 = fast_exp2(fmaf(v[c + 1], sc, -top));
-          if (ragged) {
-            if (c >= valid) w0 = 0.f;
-            if (c + 1 >= valid) w1 = 0.f;
+          for (int e = 0; e < 16; ++e) {
+            const int c = c0 + 2 * e;
+            float x0, x1;
+            unpack2(fma2(pack2(v[c], v[c + 1]), sc2, ntop2), x0, x1);
+            const uint64_t w2 = pack2(fast_exp2(x0), fast_exp2(x1));
+            part[e & 3] = add2(part[e & 3], w2);           // equals the bf16 pairs to 2^-17
+            float w0, w1;
+            unpack2(w2, w0, w1);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
+            hi[e] = *reinterpret_cast<const uint32_t*>(&h);
+            float r0, r1;
+            unpack2(sub2(w2, pack2(__uint_as_float(hi[e] << 16), __uint_as_float(hi[e] & 0xffff0000u))), r0, r1);
+            const __nv_bfloat162 q = __floats2bfloat162_rn(r0, r1);
+            lo[e] = *reinterpret_cast<const uint32_t*>(&q);
           }
-          sum += w0 + w1;                                  // equals the bf16 pairs to 2^-17
-          split_bf16x2(w0, w1, hi[e], lo[e]);
+          tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
+          tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
         }
-        tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
-        tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
+        float p0, p1;
+        unpack2(add2(add2(part[0], part[1]), add2(part[2], part[3])), p0, p1);
+        sum += p0 + p1;
+      } else {
+        // last tile of the cache: keys beyond its end are masked by index
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t hi[16], lo[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int c = c0 + 2 * e;
+            const float w0 = c < valid ? fast_exp2(fmaf(v[c], sc, -top)) : 0.f;
+            const float w1 = c + 1 < valid ? fast_exp2(fmaf(v[c + 1], sc, -top)) : 0.f;
+            sum += w0 + w1;
+            split_bf16x2(w0, w1, hi[e], lo[e]);
+          }
+          tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
+          tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
+        }
       }
       tmem_st_wait();
       tc_fence_before();
