@@ -164,6 +164,24 @@ def test_attention_running_maximum_moves_every_tile():
         _check_out(O, Q, K, V, np.full((B, H), n), 1.0, what=f"ramp {direction:+.0f}")
 
 
+@pytest.mark.parametrize("scale", [-0.3, 0.0])
+def test_attention_negative_and_zero_scale(scale):
+    """A negative scale turns the row maximum of the logits into a minimum of the raw products
+    (the kernel takes the extreme of the unscaled row); scale 0 gives the mean of the value rows.
+    Several full tiles and a ragged last one."""
+    B, H, n, d, m = 1, 2, 600, 128, 130
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=B, n_max=n, kv_heads=H, q_heads=H, data_seed=13)
+    K, V, _ = synth.make_kv(w, DEV)
+    Q = _queries(B, H, m, d, seed=21)
+    desc = cur.make_desc(K, V, 32)
+    O, ws = cur.curdkv_attention_out(Q, K, V, desc, scale=scale)
+    assert cur.curdkv_device_status(ws) == 0
+    _check_out(O, Q, K, V, np.full((B, H), n, dtype=np.int32), scale, what=f"scale={scale}")
+    if scale == 0.0:
+        mean = _f64(V)[0, 0].mean(axis=0)
+        assert np.abs(O.cpu().numpy()[0, 0, 0] - mean).max() <= OUT_TOL * np.abs(mean).max()
+
+
 def test_attention_rejects_bad_arguments():
     K = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device=DEV)
     Q = torch.zeros((1, 1, 16, 64), dtype=torch.bfloat16, device=DEV)
