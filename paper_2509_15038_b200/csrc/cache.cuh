@@ -119,12 +119,25 @@ __global__ void __launch_bounds__(256) cache_keyed_scores_kernel(const CacheView
   const int p = blockIdx.x, b = p / heads;
   const int held = min(max(c.count[b], 0), c.capacity);
   const int recent = c.total[b] - window;
-  for (int s = threadIdx.x; s < held; s += blockDim.x) {
-    const int pos = c.pos[(size_t)p * c.capacity + s];
-    const float raw = c.raw[(size_t)p * c.capacity + s];
-    keyed[(size_t)p * c.capacity + s] =
-        (pos < num_sink || pos >= recent) ? __int_as_float(0x7f800000) : fmaxf(raw, 1.17549435e-38f);
+  const int32_t* pos_row = c.pos + (size_t)p * c.capacity;
+  const float* raw_row = c.raw + (size_t)p * c.capacity;
+  float* key_row = keyed + (size_t)p * c.capacity;
+  auto key_of = [&](int pos, float raw) {
+    return (pos < num_sink || pos >= recent) ? __int_as_float(0x7f800000) : fmaxf(raw, 1.17549435e-38f);
+  };
+  int done = 0;
+  if ((c.capacity & 3) == 0 && ((reinterpret_cast<uintptr_t>(c.pos) | reinterpret_cast<uintptr_t>(c.raw) |
+                                 reinterpret_cast<uintptr_t>(keyed)) & 15u) == 0) {
+    const int quads = held >> 2;                           // four slots per thread and step
+    for (int q = threadIdx.x; q < quads; q += blockDim.x) {
+      const int4 ps = reinterpret_cast<const int4*>(pos_row)[q];
+      const float4 rw = reinterpret_cast<const float4*>(raw_row)[q];
+      reinterpret_cast<float4*>(key_row)[q] =
+          make_float4(key_of(ps.x, rw.x), key_of(ps.y, rw.y), key_of(ps.z, rw.z), key_of(ps.w, rw.w));
+    }
+    done = quads << 2;
   }
+  for (int s = done + threadIdx.x; s < held; s += blockDim.x) key_row[s] = key_of(pos_row[s], raw_row[s]);
 }
 
 // After the selection: rows kept at slots >= kept ("movers", the tail of the ascending idx list)
