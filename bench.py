@@ -272,7 +272,8 @@ def run_cuda(args):
         "clocks": clocks,
         "gpu_launches": int(launches),
         "roofline": {
-            "bound": "hbm", "kernel": "sketch_umma_kernel (inside curdkv_score)",
+            "bound": "hbm",
+            "kernel": ("sketch_items_kernel" if args.whiten else "sketch_umma_kernel") + " (inside curdkv_score)",
             "achieved": sketch_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
             "unit": "GB/s", "frac": sketch_gbs / peak,
             "traffic": None if (args.whiten or args.batch > 0) else TRAFFIC_BYTES.get(w.name),
