@@ -149,6 +149,8 @@ def run_cuda(args):
     w = rank_workload(synth.CONFIGS[args.workload], rank)
     if args.batch > 0:                                     # the same recipe at another batch size
         w = synth.shrink(w, batch=args.batch)
+    if args.layers > 0:                                    # ... or with fewer layers (small profiling cases)
+        w = synth.shrink(w, layers=args.layers)
     K, V, seqlens = synth.make_kv(w, dev)
     G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
     sl = None if seqlens is None else torch.as_tensor(seqlens, device=dev)
@@ -276,7 +278,7 @@ def run_cuda(args):
             "kernel": ("sketch_items_kernel" if args.whiten else "sketch_umma_kernel") + " (inside curdkv_score)",
             "achieved": sketch_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
             "unit": "GB/s", "frac": sketch_gbs / peak,
-            "traffic": None if (args.whiten or args.batch > 0) else TRAFFIC_BYTES.get(w.name),
+            "traffic": None if (args.whiten or args.batch > 0 or args.layers > 0) else TRAFFIC_BYTES.get(w.name),
             "algorithmic_bytes_per_launch": pass_bytes, "ms_per_launch": sketch_ms,
             "timer": "CUDA events recorded by the library around the kernel, mean over the timed steps",
         },
@@ -576,6 +578,8 @@ def run_reference(args):
     w = synth.CONFIGS[args.workload]
     if args.batch > 0:
         w = synth.shrink(w, batch=args.batch)
+    if args.layers > 0:
+        w = synth.shrink(w, layers=args.layers)
     elems = sample_elements(w, core_seconds=20.0)
     Ku, Vu, sl = oracle_sample(w, elems)
     G = synth.make_G(w.d, w.r, seed=0)
@@ -611,6 +615,8 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(synth.CONFIGS) + ["decode", "evict"])
     ap.add_argument("--batch", type=int, default=0,
                     help="sequences per layer instead of the workload's own (cfg1-cfg5 only); 0 keeps it")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="layers instead of the workload's own (cfg1-cfg5 only); 0 keeps them")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
                     help="--workload decode: compress inside the cache (unordered) or copy in order")
