@@ -283,6 +283,27 @@ def run_cuda(args):
             "timer": "CUDA events recorded by the library around the kernel, mean over the timed steps",
         },
     }
+    if args.graph and world == 1:
+        # the same step captured once into a CUDA graph and replayed: what a caller that runs the
+        # three calls back to back saves in launch overhead (only visible on small workloads)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        gev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        for i in range(args.steps):
+            if flush is not None:
+                flush.zero_()
+            gev[i][0].record()
+            graph.replay()
+            gev[i][1].record()
+        torch.cuda.synchronize()
+        out["cuda_graph"] = {"ms_per_step": float(np.mean([a_.elapsed_time(b_) for a_, b_ in gev])),
+                             "eager_ms_per_step": ms_step}
     out["e2e"] = run_e2e(cur, w, K, V, seqlens, value_tokens=tokens, world=world, dev=dev,
                          steps=min(args.steps, args.e2e_steps))
     if rank == 0:
@@ -617,6 +638,8 @@ def main():
                     help="sequences per layer instead of the workload's own (cfg1-cfg5 only); 0 keeps it")
     ap.add_argument("--layers", type=int, default=0,
                     help="layers instead of the workload's own (cfg1-cfg5 only); 0 keeps them")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the step replayed from a CUDA graph (extra 'cuda_graph' object)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
                     help="--workload decode: compress inside the cache (unordered) or copy in order")

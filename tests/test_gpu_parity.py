@@ -413,3 +413,46 @@ def test_compress_host_matches_device_calls(adaptive):
                 for h in range(w.kv_heads):
                     assert torch.equal(bufs.K_out[b, h, : c[b, h]], Ko.cpu()[b, h, : c[b, h]])
                     assert torch.equal(bufs.V_out[b, h, : c[b, h]], Vo.cpu()[b, h, : c[b, h]])
+
+
+def test_calls_can_be_captured_into_a_cuda_graph():
+    """score -> select -> compact enqueue only kernels and memsets on the caller's stream, so the
+    three calls can be captured once and replayed; the replay must reproduce the eager results."""
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=2, n_max=3000)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=DEV)
+    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads)
+    ws = cur.alloc_workspace(desc, 400, False)
+    B, H = w.folded_batch, w.kv_heads
+    scores = torch.empty((B, H, w.n_max), dtype=torch.float32, device=DEV)
+    sums = torch.empty((B, H), dtype=torch.float32, device=DEV)
+    idx = torch.empty((B, H, 400), dtype=torch.int32, device=DEV)
+    Ko = torch.empty((B, H, 400, w.d), dtype=torch.bfloat16, device=DEV)
+    Vo = torch.empty_like(Ko)
+    cnt = torch.empty((B, H), dtype=torch.int32, device=DEV)
+    off = torch.empty((B * H + 1,), dtype=torch.int32, device=DEV)
+
+    def step():
+        cur.curdkv_score(K, V, G, desc, ws, scores=scores, head_sums=sums)
+        cur.curdkv_select(scores, desc, 400, num_sink=4, window=32, workspace=ws, idx=idx, head_counts=cnt,
+                          head_offsets=off)
+        cur.curdkv_compact(K, V, desc, idx, cnt, off, K_out=Ko, V_out=Vo, workspace=ws)
+
+    step()
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (scores, sums, idx, cnt, Ko, Vo)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (scores, sums, idx, cnt, Ko, Vo):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert cur.curdkv_device_status(ws) == 0
+    for a, b in zip(want, (scores, sums, idx, cnt, Ko, Vo)):
+        assert torch.equal(a, b)
