@@ -433,29 +433,39 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
     if (P * (int64_t)(budget < desc->n_max ? budget : desc->n_max) > 0x7fffffffLL)
       return CURDKV_ERR_UNSUPPORTED;
     const int min_protected = (int)floor(alpha * (double)budget);
-    if (cudaFuncSetAttribute(select_adaptive_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kAdaptiveDynamic) != cudaSuccess)
-      return CURDKV_ERR_CUDA;
-    if (desc->kv_heads > 8 &&
-        cudaFuncSetAttribute(select_adaptive_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
-                             1) != cudaSuccess)
-      return CURDKV_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)P);
-    cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = kAdaptiveDynamic;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)desc->kv_heads;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, select_adaptive_kernel, scores, desc->seqlens,
-                                             (int)desc->kv_heads, (int)desc->n_max, (int)budget,
-                                             (int)num_sink, (int)window, min_protected, idx,
-                                             head_counts, head_offsets);
+    // With one CTA of 1024 threads per SM, floor(148 / heads) clusters run at a time.  When the
+    // batch needs more than one such round, CTAs of 512 threads (two per SM) keep all clusters
+    // resident instead; ADAPTIVE_VARIANT (a build-time switch for measurements) forces a choice.
+    const int64_t one_round = 148 / (desc->kv_heads > 0 ? desc->kv_heads : 1);
+    bool small_ctas = desc->batch > one_round;
+#if defined(ADAPTIVE_VARIANT)
+    small_ctas = ADAPTIVE_VARIANT == 512;
+#endif
+    auto launch = [&](auto kernel, int threads) -> cudaError_t {
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               adaptive_dynamic_bytes(threads)) != cudaSuccess)
+        return cudaErrorUnknown;
+      if (desc->kv_heads > 8 &&
+          cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+        return cudaErrorUnknown;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)P);
+      cfg.blockDim = dim3((unsigned)threads);
+      cfg.dynamicSmemBytes = (size_t)adaptive_dynamic_bytes(threads);
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = (unsigned)desc->kv_heads;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      return cudaLaunchKernelEx(&cfg, kernel, scores, desc->seqlens, (int)desc->kv_heads, (int)desc->n_max,
+                                (int)budget, (int)num_sink, (int)window, min_protected, idx, head_counts,
+                                head_offsets);
+    };
+    const cudaError_t e = small_ctas ? launch(select_adaptive_kernel<512>, 512)
+                                     : launch(select_adaptive_kernel<1024>, 1024);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
     return CURDKV_OK;

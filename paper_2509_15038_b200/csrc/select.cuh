@@ -545,7 +545,9 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
 // slots go to the best unprotected keys of all heads (ties: lower head, then
 // lower token), found by a radix select whose digit histograms are summed
 // across the cluster through distributed shared memory.
-// grid = batch*heads, cluster = heads, block = 1024.
+// grid = batch*heads, cluster = heads, block = THREADS (1024, or 512 with lists
+// of half the size so that two CTAs share an SM: more clusters are resident at
+// once, which pays when there are more clusters than fit in one round).
 // ---------------------------------------------------------------------------
 struct AdaptiveSmem {
   SelectSmem s;
@@ -553,18 +555,22 @@ struct AdaptiveSmem {
   uint32_t pub_eq;                                         // unprotected keys equal to the global cut
   uint32_t pub_count;                                      // rows this head keeps
 };
-constexpr int kAdaptiveDynamic = kSelBins * 4 + 2 * kSelListBytes;   // leading-digit histogram + two lists
+// dynamic shared memory: leading-digit histogram + two lists
+__host__ __device__ constexpr int adaptive_list_cap(int threads) { return threads == 1024 ? kSelListCap : kSelListCap / 2; }
+__host__ __device__ constexpr int adaptive_dynamic_bytes(int threads) { return kSelBins * 4 + 2 * adaptive_list_cap(threads) * 8; }
 
-__global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kernel(
     const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
     int budget, int num_sink, int window, int min_protected, int32_t* __restrict__ idx,
     int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   __shared__ AdaptiveSmem sm;
   extern __shared__ uint4 adaptive_dyn[];
   uint32_t* hist_all = reinterpret_cast<uint32_t*>(adaptive_dyn);          // leading digits of all keys
-  const KeyList list_a{reinterpret_cast<uint2*>(hist_all + kSelBins), &sm.s.list_count[0],
-                       (uint32_t)kSelListCap};
-  const KeyList list_b{list_a.items + kSelListCap, &sm.s.list_count[1], (uint32_t)kSelListCap};
+  constexpr int B = kSelBins / THREADS, Q = B / 4;         // histogram bins (quads of bins) per thread
+  constexpr int kCap = adaptive_list_cap(THREADS);
+  const KeyList list_a{reinterpret_cast<uint2*>(hist_all + kSelBins), &sm.s.list_count[0], (uint32_t)kCap};
+  const KeyList list_b{list_a.items + kCap, &sm.s.list_count[1], (uint32_t)kCap};
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x;
   const int h = (int)cluster.block_rank();
@@ -587,7 +593,7 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   __syncthreads();
   uint32_t d0 = 0xffffffffu, rank_own = 0;
   if (!none && !all) {
-    pick_digit_impl<4>(hist_all, (uint32_t)prot, sm.s);
+    pick_digit_impl<B>(hist_all, (uint32_t)prot, sm.s);
     d0 = sm.s.digit;
     rank_own = sm.s.remaining;
     __syncthreads();
@@ -598,32 +604,34 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
   // protected keys in it, nothing above.
   uint32_t dg = 0, remaining = pool, local_gt = 0, local_eq = 0;
   if (pool > 0) {
-    {
-      const uint4 v = reinterpret_cast<const uint4*>(hist_all)[tid];
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+      const uint4 v = reinterpret_cast<const uint4*>(hist_all)[tid * Q + q];
       uint32_t c[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const uint32_t bin = (uint32_t)(4 * tid + u);
+        const uint32_t bin = (uint32_t)(B * tid + 4 * q + u);
         if (all) c[u] = 0;
         else if (!none && bin > d0) c[u] = 0;
         else if (!none && bin == d0) c[u] -= rank_own;
       }
-      reinterpret_cast<uint4*>(sm.hist_local)[tid] = make_uint4(c[0], c[1], c[2], c[3]);
+      reinterpret_cast<uint4*>(sm.hist_local)[tid * Q + q] = make_uint4(c[0], c[1], c[2], c[3]);
     }
     cluster.sync();
-    {
-      uint4 acc = make_uint4(0u, 0u, 0u, 0u);              // this thread's four bins over all heads
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+      uint4 acc = make_uint4(0u, 0u, 0u, 0u);              // four of this thread's bins over all heads
       for (int r = 0; r < heads; ++r) {
-        const uint4 v = reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid];
+        const uint4 v = reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid * Q + q];
         acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
       }
-      reinterpret_cast<uint4*>(sm.s.hist)[tid] = acc;
+      reinterpret_cast<uint4*>(sm.s.hist)[tid * Q + q] = acc;
     }
     __syncthreads();
-    pick_digit_impl<4>(sm.s.hist, remaining, sm.s);
+    pick_digit_impl<B>(sm.s.hist, remaining, sm.s);
     dg = sm.s.digit;
     remaining = sm.s.remaining;
-    local_gt = count_above_impl<4>(sm.hist_local, dg, sm.s);
+    local_gt = count_above_impl<B>(sm.hist_local, dg, sm.s);
     cluster.sync();                                        // peers are done reading hist_local
   }
 
@@ -662,21 +670,23 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
       if (tid == 0 && own.eq_take > 0 && (own.T & mask) == prefix)
         sm.hist_local[(own.T >> shift) & pass_digit_mask(pass)] -= own.eq_take;   // those are protected
       cluster.sync();
-      {
+#pragma unroll
+      for (int q = 0; q < Q; ++q) {
         uint4 acc = make_uint4(0u, 0u, 0u, 0u);
         for (int r = 0; r < heads; ++r) {
-          const uint4 v = reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid];
+          const uint4 v =
+              reinterpret_cast<const uint4*>(cluster.map_shared_rank(sm.hist_local, r))[tid * Q + q];
           acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
-        reinterpret_cast<uint4*>(sm.s.hist)[tid] = acc;
+        reinterpret_cast<uint4*>(sm.s.hist)[tid * Q + q] = acc;
       }
       __syncthreads();
-      pick_digit_impl<4>(sm.s.hist, remaining, sm.s);
+      pick_digit_impl<B>(sm.s.hist, remaining, sm.s);
       const uint32_t dgt = sm.s.digit;
       remaining = sm.s.remaining;
       prefix |= dgt << shift;
       mask |= pass_digit_mask(pass) << shift;
-      local_gt += count_above_impl<4>(sm.hist_local, dgt, sm.s);
+      local_gt += count_above_impl<B>(sm.hist_local, dgt, sm.s);
       if (pass == kSelPasses - 1) local_eq = sm.hist_local[dgt];
       cluster.sync();                                      // peers are done reading hist_local
     }
@@ -702,14 +712,14 @@ __global__ void __launch_bounds__(kSelThreads) select_adaptive_kernel(
 
   // ---- packed output position: rows of earlier sequences, then earlier heads
   uint32_t part = 0;
-  for (int bb = tid; bb < b; bb += kSelThreads)
+  for (int bb = tid; bb < b; bb += THREADS)
     part += (uint32_t)heads * (uint32_t)min(budget, seq_len_of(seqlens, bb, n_max));
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
   if ((tid & 31) == 0) sm.s.warp_def[tid >> 5] = part;
   __syncthreads();
   uint32_t off = 0;
-  for (int w = 0; w < kSelThreads / 32; ++w) off += sm.s.warp_def[w];
+  for (int w = 0; w < THREADS / 32; ++w) off += sm.s.warp_def[w];
   for (int r = 0; r < h; ++r) off += *cluster.map_shared_rank(&sm.pub_count, r);
   __syncthreads();
 
