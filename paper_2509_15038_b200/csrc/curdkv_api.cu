@@ -435,12 +435,9 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
     const int min_protected = (int)floor(alpha * (double)budget);
     // With one CTA of 1024 threads per SM, floor(148 / heads) clusters run at a time.  When the
     // batch needs more than one such round, CTAs of 512 threads (two per SM) keep all clusters
-    // resident instead; ADAPTIVE_VARIANT (a build-time switch for measurements) forces a choice.
+    // resident instead.
     const int64_t one_round = 148 / (desc->kv_heads > 0 ? desc->kv_heads : 1);
-    bool small_ctas = desc->batch > one_round;
-#if defined(ADAPTIVE_VARIANT)
-    small_ctas = ADAPTIVE_VARIANT == 512;
-#endif
+    const bool small_ctas = desc->batch > one_round;
     auto launch = [&](auto kernel, int threads) -> cudaError_t {
       if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                adaptive_dynamic_bytes(threads)) != cudaSuccess)
