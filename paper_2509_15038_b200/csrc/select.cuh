@@ -219,6 +219,7 @@ struct DigitRun {
   }
 };
 
+constexpr int kSelRankDirect = 192;                        // lists up to this size are ranked without histograms
 constexpr int kSelUnroll = 4;                              // quads in flight per thread
 
 // Adds the keys <= ceiling whose bits under `mask` equal `prefix` to the
@@ -395,6 +396,28 @@ __device__ __forceinline__ Cut finish_cut(const RowKeys& keys, const KeyList& li
                                           uint32_t rank, SelectSmem& sm) {
   uint32_t prefix = d0 << 20, mask = 0xfffu << 20, remaining = rank;
   const bool from_list = list.complete();
+  if (from_list && list.size() <= kSelRankDirect) {
+    // a short list is ranked directly: thread t counts the keys above and equal to key t (equal
+    // keys find the same cut, so it does not matter which of their threads writes it)
+    const int L = list.size();
+    if ((int)threadIdx.x < L) {
+      const uint32_t key = list.items[threadIdx.x].x;
+      uint32_t gt = 0, eq = 0;
+      for (int e = 0; e < L; ++e) {
+        const uint32_t other = list.items[e].x;
+        gt += other > key ? 1u : 0u;
+        eq += other == key ? 1u : 0u;
+      }
+      if (gt < rank && rank <= gt + eq) {
+        sm.digit = key;
+        sm.remaining = rank - gt;
+      }
+    }
+    __syncthreads();
+    const Cut cut{sm.digit, sm.remaining};
+    __syncthreads();                                       // sm.digit may be rewritten
+    return cut;
+  }
   for (int pass = 1; pass < kSelPasses; ++pass) {
     clear_hist(sm.hist);
     __syncthreads();
