@@ -148,14 +148,26 @@ void* static_scratch_ptr() {
 }
 
 // Whitened scoring cuts every head into this many runs of tiles (the work items of the two
-// streaming kernels): enough items to balance the SMs, never more than the head has tiles.
+// streaming kernels).  An item costs its tiles plus a fixed part (staging W, draining and storing
+// a partial Gram matrix: about ten tiles' worth, measured), and every CTA walks ceil(P s / 148)
+// items, so the count that minimises rounds x (tiles per item + fixed part) is taken: many
+// segments balance the SMs, few keep the fixed part small.
 int whiten_segments(const curdkv_desc* d) {
   const int64_t P = (int64_t)d->batch * d->kv_heads;
   if (P <= 0) return 1;
-  int64_t s = (8 * 148 + P - 1) / P;
   const int tiles = tiles_per_head(d);
-  if (s > tiles) s = tiles;
-  return s < 1 ? 1 : (int)s;
+  constexpr int64_t kItemOverheadTiles = 10;
+  int best = 1;
+  int64_t best_cost = -1;
+  for (int s = 1; s <= tiles && s <= 32; ++s) {
+    const int64_t rounds = (P * s + 147) / 148;
+    const int64_t cost = rounds * ((tiles + s - 1) / s + kItemOverheadTiles);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = s;
+    }
+  }
+  return best;
 }
 
 struct WhitenLayout {      // byte offsets from the workspace base, after the tile sums
