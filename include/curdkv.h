@@ -18,7 +18,9 @@
  *     never retains a pointer after a call returns.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     All work is enqueued on it; calls return without synchronising unless
- *     stated otherwise.
+ *     stated otherwise.  Such calls only launch kernels and memsets on the
+ *     stream, so a sequence of them can be captured into a CUDA graph and
+ *     replayed (curdkv_compress_host, which synchronises, cannot).
  *   - Return codes report errors the host can see (bad arguments, unsupported
  *     shapes, small workspace, launch failure).  Anomalies seen on the device
  *     (an out-of-range index, a bounded wait that ran out) are OR-ed into a
