@@ -63,3 +63,26 @@ def test_workspace_sizes_of_the_added_modes_without_a_device():
     assert lib.curdkv_eviction_loss(None, None, 1, 1, None, None, None) == 1
     assert lib.curdkv_gqa_expand(None, None, None, 1, None, None, None) == 1
     assert binding.launch_count() == before
+
+
+def _whiten_segments(batch, heads, n, r=32):
+    """Segments per head the library plans for a whitened call, read off its workspace size."""
+    plain = binding.Desc(batch, heads, heads, n, 128, r, 0, 0, 128, 0, 0, 128, None, 0, 1)
+    white = binding.Desc(batch, heads, heads, n, 128, r, 0, 0, 128, 0, 0, 128, None, 0, 1, 0, 1, 1e-4)
+    extra = binding.workspace_bytes(white) - binding.workspace_bytes(plain)
+    P = batch * heads
+    w_bytes = -(-(P * 2 * 128 * r * 4) // 256) * 256
+    return (extra - w_bytes) // (P * 2 * 128 * 128 * 4)
+
+
+def test_whitened_segment_count_follows_the_cost_model():
+    """Segments per head minimise ceil(P s / 148) x (tiles per item + 10) over s (host logic only):
+    the three bench shapes, and a single long head, which must be cut up to feed all SMs."""
+    def model(P, tiles):
+        cost = lambda s: -(-(P * s) // 148) * (-(-tiles // s) + 10)
+        return min(range(1, min(tiles, 32) + 1), key=lambda s: (cost(s), s))
+    for batch, heads, n in [(32, 8, 8192), (128, 8, 32768), (32, 8, 131072), (1, 1, 131072), (1, 2, 1000)]:
+        tiles = -(-n // 128)
+        assert _whiten_segments(batch, heads, n) == model(batch * heads, tiles), (batch, heads, n)
+    assert _whiten_segments(32, 8, 8192) == 1 and _whiten_segments(32, 8, 131072) == 4
+    assert _whiten_segments(1, 1, 131072) == 32
