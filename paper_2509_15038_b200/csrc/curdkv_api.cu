@@ -159,7 +159,7 @@ int whiten_segments(const curdkv_desc* d) {
   constexpr int64_t kItemOverheadTiles = 10;
   int best = 1;
   int64_t best_cost = -1;
-  for (int s = 1; s <= tiles && s <= 32; ++s) {
+  for (int s = 1; s <= tiles && s <= 1024; ++s) {
     const int64_t rounds = (P * s + 147) / 148;
     const int64_t cost = rounds * ((tiles + s - 1) / s + kItemOverheadTiles);
     if (best_cost < 0 || cost < best_cost) {

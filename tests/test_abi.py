@@ -80,9 +80,9 @@ def test_whitened_segment_count_follows_the_cost_model():
     the three bench shapes, and a single long head, which must be cut up to feed all SMs."""
     def model(P, tiles):
         cost = lambda s: -(-(P * s) // 148) * (-(-tiles // s) + 10)
-        return min(range(1, min(tiles, 32) + 1), key=lambda s: (cost(s), s))
+        return min(range(1, min(tiles, 1024) + 1), key=lambda s: (cost(s), s))
     for batch, heads, n in [(32, 8, 8192), (128, 8, 32768), (32, 8, 131072), (1, 1, 131072), (1, 2, 1000)]:
         tiles = -(-n // 128)
         assert _whiten_segments(batch, heads, n) == model(batch * heads, tiles), (batch, heads, n)
     assert _whiten_segments(32, 8, 8192) == 1 and _whiten_segments(32, 8, 131072) == 4
-    assert _whiten_segments(1, 1, 131072) == 32
+    assert _whiten_segments(1, 1, 131072) == 147          # 147 items of 7 tiles: one round on 148 SMs
