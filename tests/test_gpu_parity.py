@@ -302,6 +302,24 @@ def _adaptive_case(scores_np, budget, s, w, alpha, seqlens=None):
     return idx, cnt, off
 
 
+def test_adaptive_select_many_sequences_small_ctas():
+    """More (layer, sequence) clusters than one round of 1024-thread CTAs holds: the kernel then runs
+    with CTAs of 512 threads, two per SM, and lists of half the size.  Same rule, ties and ragged
+    lengths included, and a row whose candidates overflow the shorter list."""
+    rng = np.random.default_rng(77)
+    B, H, n = 40, 8, 2500
+    mass = rng.random((B, H, 1)) ** 3 + 0.01
+    sc = (rng.random((B, H, n)) ** 4 * mass).astype(np.float32)
+    _adaptive_case(sc, 300, 4, 16, 0.2)
+    tied = (np.round(sc / sc.max() * 32) / 32).astype(np.float32)
+    _adaptive_case(tied, 700, 2, 3, 0.5)
+    lens = rng.integers(0, n + 1, size=B).astype(np.int32)
+    lens[:3] = (n, 1, 0)
+    _adaptive_case(sc, 500, 1, 7, 0.2, seqlens=lens)
+    near = (1.0 + rng.random((B, H, 6000)) * 2.0 ** -13).astype(np.float32)   # one leading digit: list overflow
+    _adaptive_case(near, 1000, 2, 10, 0.3)
+
+
 @pytest.mark.parametrize("H", [1, 2, 3, 8, 16])
 def test_adaptive_select_matches_oracle_rule(H):
     rng = np.random.default_rng(H)
