@@ -175,6 +175,25 @@ def _select_case(scores_np, budget, s, w, seqlens=None, head_budgets=None):
     np.testing.assert_array_equal(idx.cpu().numpy(), ridx)
 
 
+@pytest.mark.parametrize("n", [3000, 12000, 30000])      # CTAs of 256, 512 and 1024 threads
+def test_select_short_candidate_lists(n):
+    """The keys that share the cut's leading digit are ranked directly when there are at most 192
+    of them and by two more histogram passes otherwise: list lengths around that limit, cuts at
+    the first, an inner and the last key of the list, duplicates among them."""
+    rng = np.random.default_rng(n)
+    for L in (1, 2, 64, 191, 192, 193, 400):
+        sc = np.empty((1, 2, n), dtype=np.float32)
+        for h in range(2):
+            high = n // 3
+            row = np.concatenate([2.0 + rng.random(high),                    # above the list's digit
+                                  1.0 + rng.integers(0, 20, size=L) / 256.0,  # the list: few distinct values
+                                  0.1 + 0.4 * rng.random(n - high - L)]).astype(np.float32)
+            sc[0, h] = row[rng.permutation(n)]
+        for j in sorted({1, (L + 1) // 2, L}):
+            _select_case(sc, n // 3 + j, 0, 0)
+            _select_case(sc, n // 3 + j + 6, 2, 4)
+
+
 def test_select_edges_and_ties():
     rng = np.random.default_rng(0)
     sc = rng.random((2, 3, 5000)).astype(np.float32)
