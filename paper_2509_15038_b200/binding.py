@@ -19,6 +19,8 @@ _lib = None
 STATUS_OK = 0
 DEV_TIMEOUT = 0x1
 DEV_BAD_INDEX = 0x2
+DEV_CACHE_FULL = 0x4
+DEV_NOT_SPD = 0x8
 
 EXPORTS = (
     "curdkv_workspace_bytes", "curdkv_score", "curdkv_select", "curdkv_compact",

@@ -136,3 +136,27 @@ def test_whitened_rejects_unsupported_shapes():
     desc = cur.make_desc(K, K, 32, whiten=1, ridge=-1.0)
     with pytest.raises((cur.CurdkvError, ValueError)):
         cur.curdkv_score(K, K, G, desc, torch.zeros(1 << 20, dtype=torch.uint8, device=DEV))
+
+
+def test_singular_gram_matrix_is_flagged_not_faulted():
+    """Channels that are zero in every row make the Gram matrix singular: without a ridge the
+    factorisation meets a zero pivot and raises the NOT_SPD bit of the status word (the results of
+    that call are void); with the ridge the same input is scored normally."""
+    g = torch.Generator(device=DEV).manual_seed(9)
+    K = torch.randn((1, 2, 1024, 128), generator=g, device=DEV)
+    K[..., 5] = 0.0
+    K[..., 77] = 0.0
+    K = K.to(torch.bfloat16)
+    V = torch.randn((1, 2, 1024, 128), generator=g, device=DEV).to(torch.bfloat16)
+    G = torch.as_tensor(synth.make_G(128, 32, seed=1), device=DEV)
+    desc = cur.make_desc(K, V, 32, whiten=1, ridge=0.0)
+    ws = cur.alloc_workspace(desc)
+    cur.curdkv_score(K, V, G, desc, ws)
+    torch.cuda.synchronize()
+    assert cur.curdkv_device_status(ws) & cur.DEV_NOT_SPD
+    desc = cur.make_desc(K, V, 32, whiten=1, ridge=1e-4)
+    ws = cur.alloc_workspace(desc)
+    scores, sums = cur.curdkv_score(K, V, G, desc, ws)
+    assert cur.curdkv_device_status(ws) == 0
+    assert bool(torch.isfinite(scores).all())
+    assert torch.allclose(scores.sum(-1), torch.ones_like(scores.sum(-1)), atol=1e-4)
