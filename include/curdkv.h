@@ -118,9 +118,12 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
  * the per-tile partial sums of the head normaliser) lives here in an array built
  * into the library: 4 MiB + 256 bytes of device memory held by every GPU that
  * loads the library, until the process exits.
- *   - Same arguments and results as curdkv_score, minus the workspace.
+ *   - Same arguments and results (bit for bit) as curdkv_score, minus the
+ *     workspace.
  *   - Limit: batch * kv_heads * ceil(n_max / 128) <= 262144 tiles (2^20 partial
  *     sums); larger shapes return CURDKV_ERR_STATIC_LIMIT and enqueue nothing.
+ *   - desc->whiten = 1 is not available here (its Gram matrices and factors
+ *     need 256 KiB and more of scratch per head): CURDKV_ERR_UNSUPPORTED.
  *   - status_flags: NULL, or a device uint32 that receives the device status
  *     word of this call (copied on the stream after the kernels).
  *   - The first call on each device looks up the array's device address (with
@@ -307,6 +310,17 @@ curdkv_status curdkv_gqa_expand(const curdkv_desc* desc, const int32_t* idx, con
  * synchronising the stream.  Returns CURDKV_ERR_TIMEOUT if the timeout bit is
  * set, CURDKV_OK otherwise (other bits are reported through *host_flags). */
 curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, void* cuda_stream);
+
+/* Self-test of the failure path (no counterpart in the paper).  Every wait inside the
+ * pipelined kernels (TMA producer, MMA issuer, epilogue warps of the score, Gram and
+ * attention kernels) is bounded: when its limit runs out the kernel sets
+ * CURDKV_DEV_TIMEOUT, drains what it issued and returns.  This call runs that same
+ * wait routine, with `limit_ns` (1 .. 10^9 nanoseconds) in place of the kernels'
+ * 2 s, on a barrier that is never completed: one small kernel that comes back after
+ * about limit_ns with CURDKV_DEV_TIMEOUT in the status word of `workspace` (at least
+ * 256 bytes, 256-byte aligned; cleared first).  Nothing faults or traps, and the
+ * stream stays usable: read the word with curdkv_device_status(). */
+curdkv_status curdkv_selftest_bounded_wait(uint64_t limit_ns, void* workspace, void* cuda_stream);
 
 /* Profiling aid (no counterpart in the paper): asks the next curdkv_score or
  * curdkv_score_static call of THIS host thread to record the two cudaEvent_t

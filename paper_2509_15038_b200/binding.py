@@ -29,6 +29,7 @@ EXPORTS = (
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
     "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
     "curdkv_eviction_loss", "curdkv_gqa_expand", "curdkv_cache_compress_inplace",
+    "curdkv_selftest_bounded_wait",
 )
 
 
@@ -117,6 +118,8 @@ def load():
                                          ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
     lib.curdkv_eviction_loss.restype = ctypes.c_int
     lib.curdkv_eviction_loss.argtypes = [vp, vp, i32, i64, vp, vp, vp]
+    lib.curdkv_selftest_bounded_wait.restype = ctypes.c_int
+    lib.curdkv_selftest_bounded_wait.argtypes = [ctypes.c_uint64, vp, vp]
     lib.curdkv_profile_next_score.restype = ctypes.c_int
     lib.curdkv_profile_next_score.argtypes = [vp, vp]
     lib.curdkv_launch_count.restype = ctypes.c_uint64
@@ -399,6 +402,12 @@ def curdkv_profile_next_score(start: torch.cuda.Event, stop: torch.cuda.Event) -
            "curdkv_profile_next_score")
 
 
+def curdkv_selftest_bounded_wait(limit_ns: int, workspace: torch.Tensor) -> None:
+    """Runs the kernels' bounded wait on a barrier nobody completes; leaves DEV_TIMEOUT in the status word."""
+    _check(load().curdkv_selftest_bounded_wait(int(limit_ns), _ptr(workspace), _stream()),
+           "curdkv_selftest_bounded_wait")
+
+
 def curdkv_gqa_map(desc: Desc, device="cuda") -> torch.Tensor:
     out = torch.empty((desc.q_heads,), dtype=torch.int32, device=device)
     _check(load().curdkv_gqa_map(ctypes.byref(desc), _ptr(out), _stream()), "curdkv_gqa_map")
@@ -415,10 +424,11 @@ def curdkv_gqa_expand(desc: Desc, idx: torch.Tensor, head_counts: torch.Tensor):
     return idx_q, counts_q
 
 
-def curdkv_device_status(workspace: torch.Tensor) -> int:
-    """Synchronises the current stream and returns the device status flags."""
+def curdkv_device_status(workspace: torch.Tensor, with_code: bool = False):
+    """Synchronises the current stream and returns the device status flags (with_code: the pair
+    (return code, flags); the code is 5, CURDKV_ERR_TIMEOUT, when the timeout bit is set)."""
     flags = ctypes.c_uint32(0)
     code = load().curdkv_device_status(_ptr(workspace), ctypes.byref(flags), _stream())
     if code not in (STATUS_OK, 5):
         raise CurdkvError(code, "curdkv_device_status")
-    return int(flags.value)
+    return (int(code), int(flags.value)) if with_code else int(flags.value)

@@ -36,6 +36,7 @@ struct AttnArgs {
   float scale;
   float* O;                  // [problems][m][128]
   uint32_t* status;
+  unsigned long long wait_ns = kWaitLimitNs;   // limit of each pipeline wait
 };
 
 constexpr int kAttnThreads = 320;                          // TMA, MMA, 2 x 4 softmax warps
@@ -213,7 +214,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       auto load = [&](const CUtensorMap* map, int t) {
         const int slot = it % kAttnRing;
         const uint32_t phase = (it / kAttnRing) & 1u;
-        if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status))) return;
+        if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status, a.wait_ns))) return;
         mbar_arrive_expect_tx(full_bar(slot), kSlotBytes);
         const uint32_t dst = base + kAttnSlot0 + slot * kSlotBytes;
         // the key tiles of a problem are read by all of its query blocks: no evict-first
@@ -232,7 +233,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         for (uint32_t q = it - pending; q < it; ++q) {
           unsigned long long t0 = global_ns();
           while (!mbar_try_wait(full_bar(q % kAttnRing), (q / kAttnRing) & 1u) &&
-                 global_ns() - t0 < kWaitLimitNs) {}
+                 global_ns() - t0 < a.wait_ns) {}
         }
       }
     }
@@ -242,11 +243,11 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       constexpr uint32_t idesc_s = instr_desc_bf16(128);
       constexpr uint32_t idesc_pv = instr_desc_pv();
       uint32_t it = 0;
-      bool ok = mbar_wait(q_full_bar, 0, abort_flag, a.status);
+      bool ok = mbar_wait(q_full_bar, 0, abort_flag, a.status, a.wait_ns);
       tc_fence_after();
       auto issue_s = [&](uint32_t buf) {                   // S[buf] = Q K^T for the next K tile of the ring
         const int slot = it % kAttnRing;
-        if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status))) return;
+        if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status, a.wait_ns))) return;
         tc_fence_after();
         const uint32_t k_base = base + kAttnSlot0 + slot * kSlotBytes;
 #pragma unroll
@@ -265,7 +266,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       if (ok && T > 1) issue_s(1);                         // tile 1
       for (int t = 0; ok && t < T; ++t) {
         const int slot = it % kAttnRing;
-        if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status))) break;
+        if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status, a.wait_ns))) break;
         const int rows = min(kTileRows, n - t * kTileRows);
         const int groups = (rows + 15) >> 4;
         if (rows < groups * 16) {                          // clear the padding rows the last MMA reads
@@ -277,7 +278,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         const uint32_t buf = (uint32_t)t & 1u;             // the group that owns this tile, its P and O
-        if (!(ok = mbar_wait(p_ready_bar(buf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status))) break;
+        if (!(ok = mbar_wait(p_ready_bar(buf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status, a.wait_ns))) break;
         tc_fence_after();
         const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
         for (int part = 0; part < 2; ++part) {             // P_hi, then P_lo
@@ -295,7 +296,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       if (!ok) {
         tc_commit(drain_bar);
         unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < a.wait_ns) {}
       }
     }
   } else {
@@ -313,7 +314,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     bool has_o = false, ok = true;                         // has_o: O_group holds at least one product
     const uint32_t s_addr = lane_addr + group * 128u, o_addr = lane_addr + 256u + group * 128u;
     for (int t = group; ok && t < T; t += 2) {
-      ok = mbar_wait(s_full_bar(group), (uint32_t)(t >> 1) & 1u, abort_flag, a.status);
+      ok = mbar_wait(s_full_bar(group), (uint32_t)(t >> 1) & 1u, abort_flag, a.status, a.wait_ns);
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const int valid = n - t * kTileRows;                 // keys of this tile that exist
@@ -426,7 +427,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       const float w0 = fast_exp2(top - m), w1 = top1 == -INFINITY ? 0.f : fast_exp2(top1 - m);
       const float denom = w0 * sum + w1 * sum1;
       if (ok) {
-        ok = mbar_wait(o_full_bar, 0, abort_flag, a.status);
+        ok = mbar_wait(o_full_bar, 0, abort_flag, a.status, a.wait_ns);
         ok = __all_sync(0xffffffffu, ok);
       }
       if (ok) {

@@ -39,7 +39,11 @@ __global__ void __launch_bounds__(kAppendWarps * 32) cache_append_kernel(const A
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
   int tb = a.t_new != nullptr ? a.t_new[b] : a.t;
   tb = tb < 0 ? 0 : (tb > a.t ? a.t : tb);
-  const int held = a.cache.count[b];
+  int held = a.cache.count[b];
+  if (held < 0 || held > a.cache.capacity) {               // counters the caller never set up
+    if (threadIdx.x == 0 && chunk == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+    held = held < 0 ? 0 : a.cache.capacity;
+  }
   const int room = a.cache.capacity - held;
   if (tb > room) {
     if (threadIdx.x == 0 && chunk == 0) flag_status(a.status, CURDKV_DEV_CACHE_FULL);
@@ -83,8 +87,9 @@ __global__ void cache_advance_kernel(CacheView cache, const int32_t* t_new, int 
   if (b >= batch) return;
   int tb = t_new != nullptr ? t_new[b] : t;
   tb = tb < 0 ? 0 : (tb > t ? t : tb);
-  const int room = cache.capacity - cache.count[b];
-  cache.count[b] += tb < room ? tb : (room > 0 ? room : 0);
+  const int held = min(max(cache.count[b], 0), cache.capacity);   // as cache_append_kernel read it
+  const int room = cache.capacity - held;
+  cache.count[b] = held + (tb < room ? tb : room);
   cache.total[b] += tb;
 }
 

@@ -30,9 +30,17 @@ __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const Compa
   const int p = blockIdx.x / ctas_per_head, part = blockIdx.x % ctas_per_head;
   const int b = p / a.heads, h = p % a.heads;
   const int n = seq_len_of(a.seqlens, b, a.n_max);
-  const int count = a.counts[p];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
   const bool fixed = a.out_stride_h > 0;
+  // a count the layout cannot hold (a stale or unwritten counts buffer) is cut to what it can
+  // hold and flagged, so that neither the index row nor the output rows of a neighbour are touched
+  int count = a.counts[p];
+  const int64_t room = fixed ? (a.idx_stride < a.out_stride_h ? a.idx_stride : a.out_stride_h)
+                             : (int64_t)a.offsets[p + 1] - a.offsets[p];
+  if (count < 0 || count > room) {
+    if (threadIdx.x == 0 && part == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+    count = count < 0 ? 0 : (int)(room > 0 ? room : 0);
+  }
   const int32_t* ix = fixed ? a.idx + (size_t)p * a.idx_stride : a.idx + a.offsets[p];
   const size_t out_row0 = fixed ? (size_t)p * a.out_stride_h : (size_t)a.offsets[p];
   const KvView& T = half ? a.V : a.K;

@@ -581,6 +581,9 @@ curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, 
                                   uint32_t* status_flags, void* cuda_stream) {
   const size_t need = curdkv_workspace_bytes(desc, 0, 0);
   if (need == 0) return CURDKV_ERR_INVALID_ARG;
+  // the whitened mode parks Gram matrices and their factors in the workspace: far beyond what
+  // the built-in array is sized for
+  if (desc->whiten) return CURDKV_ERR_UNSUPPORTED;
   if (need > kStaticBytes) return CURDKV_ERR_STATIC_LIMIT;
   void* scratch = static_scratch_ptr();
   if (scratch == nullptr) return CURDKV_ERR_CUDA;
@@ -678,6 +681,16 @@ curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compresse
   if (problems == 0) return CURDKV_OK;
   umma::frob_diff_kernel<<<(unsigned)problems, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       O_full, O_compressed, (int)elems_per_problem, loss, ref_norm);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_selftest_bounded_wait(uint64_t limit_ns, void* workspace, void* cuda_stream) {
+  if (workspace == nullptr || limit_ns == 0 || limit_ns > 1000000000ull) return CURDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+  umma::wait_selftest_kernel<<<1, 128, 0, stream>>>(static_cast<uint32_t*>(workspace), limit_ns);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }

@@ -32,6 +32,7 @@ constexpr int kSlots = 4;
 constexpr int kHalfBytes = kTileRows * 128;       // 128 rows x 64 bf16 (one 128-byte swizzle span)
 constexpr int kSlotBytes = 2 * kHalfBytes;        // d = 128 -> two spans
 constexpr int kPartsPerTile = 4;                  // partial sums per tile (one per epilogue warp)
+// Default limit of every device-side wait (the launchers pass it to the kernels as an argument).
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct Args {
@@ -43,6 +44,7 @@ struct Args {
   float* scores;
   float* tile_sums;        // [batch*heads][tiles_per_head][kPartsPerTile]
   uint32_t* status;
+  unsigned long long wait_ns = kWaitLimitNs;   // limit of each pipeline wait
 };
 
 // Ragged batches: the kernel walks only the tiles that hold valid rows.  Every
@@ -96,10 +98,10 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait.  Gives up when another role has aborted or after kWaitLimitNs;
+// Bounded wait.  Gives up when another role has aborted or after limit_ns;
 // then raises the CTA's abort flag and the device status bit.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t* status) {
+                                          uint32_t* status, unsigned long long limit_ns) {
   unsigned long long t0 = 0;
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -107,7 +109,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitNs) {
+      if (now - t0 > limit_ns) {
         *abort_flag = 1;
         flag_status(status, CURDKV_DEV_TIMEOUT);
         return false;
@@ -115,6 +117,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// The bounded wait on its own, for tests of the failure path: every warp's first lane waits on a
+// barrier that nothing ever completes.  The first wait to run out raises the abort flag and
+// CURDKV_DEV_TIMEOUT; the others then leave through the abort path.  Returns after ~limit_ns.
+__global__ void wait_selftest_kernel(uint32_t* status, unsigned long long limit_ns) {
+  __shared__ alignas(8) unsigned long long never_completed;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&never_completed), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) mbar_wait(smem_u32(&never_completed), 0, &abort_flag, status, limit_ns);
+}
+
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3, uint64_t policy) {
   asm volatile(
@@ -314,7 +331,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
         for (int tensor = 0; tensor < 2; ++tensor, ++it) {
           const int slot = it % kSlots;
           const uint32_t phase = (it / kSlots) & 1u;
-          if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status))) break;
+          if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
           mbar_arrive_expect_tx(full_bar(slot), kSlotBytes);
           const uint32_t dst = base + L::kSlot0 + slot * kSlotBytes;
           const CUtensorMap* map = tensor ? &map_v : &map_k;
@@ -328,7 +345,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
         for (uint32_t q = it - pending; q < it; ++q) {
           unsigned long long t0 = global_ns();
           while (!mbar_try_wait(full_bar(q % kSlots), (q / kSlots) & 1u) &&
-                 global_ns() - t0 < kWaitLimitNs) {}
+                 global_ns() - t0 < a.wait_ns) {}
         }
       }
     }
@@ -340,11 +357,11 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       bool ok = true;
       for (uint32_t t = first; ok && t < total_tiles; t += stride) {
         const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
-        if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status))) break;
+        if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
         tc_fence_after();
         for (int tensor = 0; tensor < 2; ++tensor, ++it) {
           const int slot = it % kSlots;
-          if (!(ok = mbar_wait(full_bar(slot), (it / kSlots) & 1u, abort_flag, a.status))) break;
+          if (!(ok = mbar_wait(full_bar(slot), (it / kSlots) & 1u, abort_flag, a.status, a.wait_ns))) break;
           tc_fence_after();
           const uint32_t a_base = base + L::kSlot0 + slot * kSlotBytes;
           const uint32_t d_tmem = tmem_base + acc * (2 * L::kN) + tensor * L::kN;
@@ -364,7 +381,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       if (!ok) {                                           // drain MMAs in flight before TMEM is freed
         tc_commit(drain_bar);
         unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < a.wait_ns) {}
       }
     }
   } else {
@@ -383,7 +400,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       float s = 0.f;
       {
         const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
-        ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status);
+        ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status, a.wait_ns);
         if (!(ok = __all_sync(0xffffffffu, ok))) break;    // the TMEM loads need the whole warp
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * (2 * L::kN);

@@ -21,6 +21,7 @@ struct ItemArgs {
   const int32_t* seqlens;  // nullptr: every sequence has n_max rows
   int batch, heads, n_max, segments;
   uint32_t* status;
+  unsigned long long wait_ns = kWaitLimitNs;   // limit of each pipeline wait
   // gram kernel
   float* partials;         // [batch*heads*segments][2][128][128]
   // sketch kernel
@@ -120,7 +121,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
           for (int tensor = 0; tensor < 2; ++tensor, ++it) {
             const int slot = it % kSlots;
             const uint32_t phase = (it / kSlots) & 1u;
-            if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status))) break;
+            if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
             mbar_arrive_expect_tx(full_bar(slot), kSlotBytes);
             const uint32_t dst = base + slot * kSlotBytes;
             const CUtensorMap* map = tensor ? &map_v : &map_k;
@@ -134,7 +135,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         for (uint32_t q = it - pending; q < it; ++q) {
           unsigned long long t0 = global_ns();
           while (!mbar_try_wait(full_bar(q % kSlots), (q / kSlots) & 1u) &&
-                 global_ns() - t0 < kWaitLimitNs) {}
+                 global_ns() - t0 < a.wait_ns) {}
         }
       }
     }
@@ -148,14 +149,14 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         const Item w = item_of(a, item);
         if (w.t_lo >= w.t_hi) continue;
         const uint32_t acc = item_it & 1u, acc_phase = (item_it >> 1) & 1u;
-        if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status))) break;
+        if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
         tc_fence_after();
         for (int t = w.t_lo; ok && t < w.t_hi; ++t) {
           const int rows = min(kTileRows, w.n - t * kTileRows);
           const int groups = (rows + 15) >> 4;             // MMAs of 16 rows each
           for (int tensor = 0; tensor < 2; ++tensor, ++it) {
             const int slot = it % kSlots;
-            if (!(ok = mbar_wait(full_bar(slot), (it / kSlots) & 1u, abort_flag, a.status))) break;
+            if (!(ok = mbar_wait(full_bar(slot), (it / kSlots) & 1u, abort_flag, a.status, a.wait_ns))) break;
             tc_fence_after();
             const uint32_t tile = base + slot * kSlotBytes;
             if (rows < groups * 16) {
@@ -183,7 +184,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
       if (!ok) {
         tc_commit(drain_bar);
         unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < a.wait_ns) {}
       }
     }
   } else {
@@ -202,7 +203,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         continue;
       }
       const uint32_t acc = item_it & 1u, acc_phase = (item_it >> 1) & 1u;
-      ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status);
+      ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status, a.wait_ns);
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256u;
@@ -308,7 +309,7 @@ sketch_items_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
           for (int tensor = 0; tensor < 2; ++tensor, ++it) {
             const int slot = it % kRing;
             const uint32_t phase = (it / kRing) & 1u;
-            if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status))) break;
+            if (!(ok = mbar_wait(empty_bar(slot), phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
             mbar_arrive_expect_tx(full_bar(slot), kSlotBytes);
             const uint32_t dst = base + L::kSlot0 + slot * kSlotBytes;
             const CUtensorMap* map = tensor ? &map_v : &map_k;
@@ -322,7 +323,7 @@ sketch_items_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         for (uint32_t q = it - pending; q < it; ++q) {
           unsigned long long t0 = global_ns();
           while (!mbar_try_wait(full_bar(q % kRing), (q / kRing) & 1u) &&
-                 global_ns() - t0 < kWaitLimitNs) {}
+                 global_ns() - t0 < a.wait_ns) {}
         }
       }
     }
@@ -335,15 +336,15 @@ sketch_items_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       for (uint32_t item = first; ok && item < items; item += stride) {
         const Item w = item_of(a, item);
         if (w.t_lo >= w.t_hi) continue;
-        if (!(ok = mbar_wait(g_ready_bar, item_it & 1u, abort_flag, a.status))) break;   // W staged
+        if (!(ok = mbar_wait(g_ready_bar, item_it & 1u, abort_flag, a.status, a.wait_ns))) break;   // W staged
         ++item_it;
         for (int t = w.t_lo; ok && t < w.t_hi; ++t) {
           const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
-          if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status))) break;
+          if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
           tc_fence_after();
           for (int tensor = 0; tensor < 2; ++tensor, ++it) {
             const int slot = it % kRing;
-            if (!(ok = mbar_wait(full_bar(slot), (it / kRing) & 1u, abort_flag, a.status))) break;
+            if (!(ok = mbar_wait(full_bar(slot), (it / kRing) & 1u, abort_flag, a.status, a.wait_ns))) break;
             tc_fence_after();
             const uint32_t a_base = base + L::kSlot0 + slot * kSlotBytes;
             const uint32_t g_base = base + (tensor ? L::kGV : L::kGK);
@@ -365,7 +366,7 @@ sketch_items_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       if (!ok) {
         tc_commit(drain_bar);
         unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < a.wait_ns) {}
       }
     }
   } else {
@@ -408,7 +409,7 @@ sketch_items_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         const int j = row0 + quarter * 32 + lane;
         float s = 0.f;
         const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
-        ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status);
+        ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, a.status, a.wait_ns);
         if (!(ok = __all_sync(0xffffffffu, ok))) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * (2 * L::kN);

@@ -61,3 +61,34 @@ def assert_selection_within_band(gpu_idx, ref_idx, ref_scores, n, forced, what="
     for j in rs - gs:       # oracle kept, GPU dropped
         assert ref_scores[j] <= T * (1 + TIE_BAND), f"{what}: token {j} dropped but scores above the cut"
     return len(gs ^ rs)
+
+
+def assert_adaptive_within_band(gpu_idx, gpu_off, ref_idx, ref_off, ref_scores, b, H, n, s, w, what=""):
+    """AdaCurDKV, the heads of one (layer, sequence) b.  gpu_idx / ref_idx are the packed index
+    arrays with their offsets; ref_scores [H, n] the oracle's scores of this b.  Every head keeps
+    sorted, distinct, in-range indices containing its forced tokens, the layer total equals the
+    oracle's, and a token on which the two disagree scores within the tie band of one of the two
+    cuts that can decide it: its own head's weakest kept candidate (the safeguard cut, or the
+    layer-wide cut where that lies lower) or the weakest kept candidate of the whole layer."""
+    ref_scores = np.asarray(ref_scores)
+    cuts, sets = [], []
+    for h in range(H):
+        g = np.asarray(gpu_idx[gpu_off[b * H + h]: gpu_off[b * H + h + 1]], dtype=np.int64)
+        r = np.asarray(ref_idx[ref_off[b * H + h]: ref_off[b * H + h + 1]], dtype=np.int64)
+        if len(g):
+            assert g.min() >= 0 and g.max() < n, f"{what} h={h}: index out of range"
+            assert np.all(np.diff(g) > 0), f"{what} h={h}: indices not strictly ascending"
+        forced = forced_tokens(n, min(len(r), len(g)), s, w)
+        assert forced <= set(g.tolist()), f"{what} h={h}: forced tokens missing"
+        cand = [j for j in r.tolist() if j not in forced]
+        cuts.append(min(ref_scores[h][j] for j in cand) if cand else np.inf)
+        sets.append((set(g.tolist()), set(r.tolist())))
+    assert sum(len(g) for g, _ in sets) == sum(len(r) for _, r in sets), f"{what}: layer totals differ"
+    lo_cut = min(cuts)
+    diffs = 0
+    for h, (g, r) in enumerate(sets):
+        for j in g ^ r:
+            rel = min(abs(ref_scores[h][j] / c - 1.0) for c in (lo_cut, cuts[h]) if np.isfinite(c) and c > 0)
+            assert rel < TIE_BAND, f"{what} h={h}: token {j} differs {rel:.3g} away from a cut"
+            diffs += 1
+    return diffs

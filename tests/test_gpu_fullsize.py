@@ -120,9 +120,11 @@ def test_cfg4_adaptive_full_size():
         np.testing.assert_array_equal(cnt[lb].cpu().numpy(), ecnt[0])
         base = offs[lb * H]
         np.testing.assert_array_equal(gi[base: base + eoff[-1]], eidx)
-        # against the oracle's own fp64 scores: per-head counts agree up to band-sized swaps
+        # against the oracle's own fp64 scores: every token on which the two selections differ
+        # lies inside the tie band of a cut
         ridx, rcnt, roff = orc.select_adaptive(rs, w.budget, w.num_sink, w.window, w.alpha)
-        assert np.abs(rcnt[0] - ecnt[0]).max() <= 2
+        pu.assert_adaptive_within_band(gi[base: base + eoff[-1]], eoff, ridx, roff, rs[0], 0, H, w.n_max,
+                                       w.num_sink, w.window, f"cfg4 lb={lb}")
         # gathered rows of this group
         rows = torch.as_tensor(gi[base: base + eoff[-1]].astype(np.int64), device=DEV)
         heads = torch.repeat_interleave(torch.arange(H, device=DEV), torch.as_tensor(ecnt[0], device=DEV))

@@ -621,3 +621,72 @@ def test_eviction_loss_properties_and_lemma1():
     Qpos = np.abs(Q) * np.sign(Q.sum(0, keepdims=True))
     V3[40:] = 0.0
     assert ev.eviction_loss(Qpos, K3, V3, np.arange(40))[0] < 1e-9
+
+
+def test_lemma1_bound_hand_worked_values():
+    """The bound of Lemma 1, sqrt(n)||V - V'||_F + 2 sqrt(n)||V'||_F, on value matrices whose norms
+    are whole numbers (tests/golden/lemma1_example.txt): catches a dropped factor 2, a dropped term,
+    n in place of sqrt(n), and V' built from the evicted instead of the kept rows."""
+    from oracle import curdkv_eviction_oracle as ev
+
+    rows = np.array([[3.0, 0.0], [0.0, 4.0], [12.0, 0.0]])
+    cases = 0
+    for line in open(os.path.join(GOLDEN, "lemma1_example.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        n, kept, bound = line.split()
+        n = int(n)
+        kept = [] if kept == "-" else [int(t) for t in kept.split(",")]
+        V = np.zeros((n, 2))
+        V[:3] = rows
+        assert ev.lemma1_bound(V, kept) == pytest.approx(float(bound), rel=1e-15, abs=0)
+        cases += 1
+    assert cases == 7
+
+
+def test_generation_phase_ragged_appends_equal_dense_appends():
+    """CacheOracle.append with t_new: blocks in which sequence b brings only t_new[b] real rows (the
+    rest of the block is padding) must leave exactly the state that appending the real rows alone
+    leaves -- positions count real rows only, padding rows never enter -- and the final kept set
+    must be that of one application of Alg. 1 to each sequence's real history."""
+    from oracle import curdkv_decode_oracle as dec
+
+    rng = np.random.default_rng(5)
+    B, H, d, r, t = 3, 2, 16, 8, 12
+    G = (rng.standard_normal((d, r)) / np.sqrt(r)).astype(np.float32)
+    k, s, w = 14, 2, 3
+    t_news = [np.array(v) for v in ([12, 5, 0], [0, 12, 7], [3, 1, 12], [12, 12, 12], [1, 0, 2], [9, 4, 0])]
+    ragged = dec.CacheOracle(B, H, d)
+    dense = [dec.CacheOracle(1, H, d) for _ in range(B)]
+    hist_K = [[] for _ in range(B)]
+    hist_V = [[] for _ in range(B)]
+    for step, tn in enumerate(t_news):
+        Kb, Vb = rand_kv(rng, B, H, t, d)
+        ragged.append(Kb, Vb, G, tn)
+        for b in range(B):
+            tb = int(tn[b])
+            hist_K[b].append(Kb[b:b + 1, :, :tb])
+            hist_V[b].append(Vb[b:b + 1, :, :tb])
+            if tb:                                        # the same real rows, as a full block
+                dense[b].append(Kb[b:b + 1, :, :tb], Vb[b:b + 1, :, :tb], G)
+        if step in (2, 4):
+            ragged.compress(k, s, w)
+            for b in range(B):
+                dense[b].compress(k, s, w)
+    ragged.compress(k, s, w)
+    totals = np.sum(t_news, axis=0)
+    np.testing.assert_array_equal(ragged.total, totals)
+    for b in range(B):
+        dense[b].compress(k, s, w)
+        assert dense[b].total[0] == totals[b]
+        Kh, Vh = np.concatenate(hist_K[b], axis=2), np.concatenate(hist_V[b], axis=2)
+        sc, _ = orc.score(Kh, Vh, G)
+        idx, cnt = orc.select_fixed(sc, k, s, w)
+        for h in range(H):
+            np.testing.assert_array_equal(ragged.pos[b][h], dense[b].pos[0][h])
+            np.testing.assert_array_equal(ragged.raw[b][h], dense[b].raw[0][h])
+            np.testing.assert_array_equal(ragged.K[b][h], dense[b].K[0][h])
+            np.testing.assert_array_equal(ragged.V[b][h], dense[b].V[0][h])
+            one_shot = idx[0, h, : cnt[0, h]]
+            np.testing.assert_array_equal(ragged.pos[b][h], one_shot)
+            np.testing.assert_array_equal(ragged.K[b][h], Kh[0, h][one_shot])
