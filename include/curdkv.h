@@ -91,8 +91,11 @@ typedef struct curdkv_desc {
 } curdkv_desc;
 
 /* Bytes of device workspace the calls below need for this shape (256-byte
- * aligned base required).  `max_budget` and `adaptive` describe the largest
- * selection that will be requested.  Returns 0 for an invalid descriptor. */
+ * aligned base required).  max_budget > 0 includes what curdkv_compress needs on
+ * top of curdkv_score (one counter per head); max_budget = 0 sizes a workspace
+ * for curdkv_score / curdkv_select / curdkv_compact alone.  `adaptive` is
+ * reserved (it does not change the size today).  Returns 0 for an invalid
+ * descriptor. */
 size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32_t adaptive);
 
 /* Alg. 1 lines 2-6: scores[b][h][j] = lK_j * lV_j / sum_j(lK_j * lV_j) with
@@ -151,6 +154,7 @@ curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, 
  *   alpha         adaptive = 1 only: safeguard in [0,1]; every head keeps at least
  *                 min(max(floor(alpha*k), forced), min(k, n_b)) rows, the rest of the
  *                 layer total kv_heads*min(k, n_b) goes to the globally best rows
+ *   workspace, workspace_bytes   reserved (not used today; NULL / 0 are accepted)
  *   idx           adaptive = 0: int32 [batch][kv_heads][budget], ascending token
  *                 index, unused tail = -1.  adaptive = 1: packed, head (b,h)
  *                 occupies idx[head_offsets[b*kv_heads+h] ...], ascending; capacity
@@ -178,6 +182,26 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
                              const int32_t* idx, int64_t idx_stride, const int32_t* head_counts,
                              const int32_t* head_offsets, void* K_out, void* V_out,
                              int64_t out_stride_h, void* workspace, void* cuda_stream);
+
+/* Alg. 1 lines 2-10 (or AdaCurDKV) in one call on device buffers: what curdkv_score,
+ * curdkv_select and curdkv_compact do one after the other, with the same arguments,
+ * the same outputs bit for bit (scores, head_sums, idx, head_counts, head_offsets,
+ * gathered rows) and the default output layouts (adaptive = 0: idx
+ * [batch][kv_heads][budget], K_out / V_out [batch][kv_heads][budget][d]; adaptive = 1:
+ * packed).  With a fixed budget, one shared G, projection on, whiten off, d = 128,
+ * r <= 32 and n_max >= 128 the scoring kernel also normalises and selects: the CTA
+ * that writes the last tile of a head runs Alg. 1 lines 6-9 for that head on extra
+ * warps while the stream of K and V goes on, so the selection costs no time of its
+ * own.  Other shapes run the three steps in sequence.
+ *   workspace   curdkv_workspace_bytes(desc, budget > 0 ? budget : 1, adaptive) bytes
+ *   head_offsets  may be NULL when adaptive = 0
+ * Enqueues kernels and memsets on the stream only. */
+curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int32_t g_per_head,
+                              const curdkv_desc* desc, int32_t budget, const int32_t* head_budgets,
+                              int32_t num_sink, int32_t window, int32_t adaptive, double alpha,
+                              float* scores, float* head_sums, int32_t* idx, int32_t* head_counts,
+                              int32_t* head_offsets, void* K_out, void* V_out, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream);
 
 /* The whole path (Alg. 1 lines 2-10, or AdaCurDKV) for a cache that lives in HOST
  * memory: chunks of `chunk_batch` batch elements are copied to the device,

@@ -29,7 +29,7 @@ EXPORTS = (
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
     "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
     "curdkv_eviction_loss", "curdkv_gqa_expand", "curdkv_cache_compress_inplace",
-    "curdkv_selftest_bounded_wait",
+    "curdkv_selftest_bounded_wait", "curdkv_compress",
 )
 
 
@@ -90,6 +90,9 @@ def load():
                                   ctypes.c_size_t, vp]
     lib.curdkv_compact.restype = ctypes.c_int
     lib.curdkv_compact.argtypes = [vp, vp, dp, vp, i64, vp, vp, vp, vp, i64, vp, vp]
+    lib.curdkv_compress.restype = ctypes.c_int
+    lib.curdkv_compress.argtypes = [vp, vp, vp, i32, dp, i32, vp, i32, i32, i32, ctypes.c_double,
+                                    vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.curdkv_host_arena_bytes.restype = ctypes.c_size_t
     lib.curdkv_host_arena_bytes.argtypes = [dp, i32, i32, i32]
     lib.curdkv_compress_host.restype = ctypes.c_int
@@ -177,7 +180,7 @@ def workspace_bytes(desc: Desc, max_budget: int = 0, adaptive: bool = False) -> 
     return int(load().curdkv_workspace_bytes(ctypes.byref(desc), int(max_budget), int(adaptive)))
 
 
-def alloc_workspace(desc: Desc, max_budget: int = 0, adaptive: bool = False, device=None) -> torch.Tensor:
+def alloc_workspace(desc: Desc, max_budget: int = 1, adaptive: bool = False, device=None) -> torch.Tensor:
     nbytes = workspace_bytes(desc, max_budget, adaptive)
     return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device or "cuda")
 
@@ -261,6 +264,43 @@ def curdkv_compact(K, V, desc: Desc, idx, head_counts, head_offsets=None, *, pac
                                  out_stride_h, _ptr(workspace), _stream())
     _check(code, "curdkv_compact")
     return K_out, V_out
+
+
+def curdkv_compress(K, V, G, desc: Desc, budget: int, workspace: torch.Tensor, *, num_sink: int = 0,
+                    window: int = 0, head_budgets=None, adaptive: bool = False, alpha: float = 0.2,
+                    scores=None, head_sums=None, idx=None, head_counts=None, head_offsets=None,
+                    K_out=None, V_out=None):
+    """Alg. 1 lines 2-10 (or AdaCurDKV) in one call; the workspace must come from
+    ``alloc_workspace(desc, budget, adaptive)``.  Returns (scores, head_sums, idx, head_counts,
+    head_offsets, K_out, V_out) with the layouts of the three separate calls."""
+    dev = K.device
+    P, b = desc.batch * desc.kv_heads, max(budget, 0)
+    if scores is None:
+        scores = torch.empty((desc.batch, desc.kv_heads, desc.n_max), dtype=torch.float32, device=dev)
+    if head_sums is None:
+        head_sums = torch.empty((desc.batch, desc.kv_heads), dtype=torch.float32, device=dev)
+    rows = P * (min(b, desc.n_max) if adaptive else b)
+    if idx is None:
+        idx = torch.empty((rows + 1,), dtype=torch.int32, device=dev)[:rows]
+        if not adaptive:
+            idx = idx.view(desc.batch, desc.kv_heads, b)
+    if head_counts is None:
+        head_counts = torch.empty((desc.batch, desc.kv_heads), dtype=torch.int32, device=dev)
+    if head_offsets is None:
+        head_offsets = torch.empty((P + 1,), dtype=torch.int32, device=dev)
+    shape = (rows, desc.d) if adaptive else (desc.batch, desc.kv_heads, b, desc.d)
+    if K_out is None:
+        K_out = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+    if V_out is None:
+        V_out = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+    g_per_head = int(G is not None and G.dim() == 3)
+    code = load().curdkv_compress(_ptr(K), _ptr(V), _ptr(G), g_per_head, ctypes.byref(desc), int(budget),
+                                  _ptr(head_budgets), int(num_sink), int(window), int(adaptive), float(alpha),
+                                  _ptr(scores), _ptr(head_sums), _ptr(idx), _ptr(head_counts),
+                                  _ptr(head_offsets), _ptr(K_out), _ptr(V_out), _ptr(workspace),
+                                  workspace.numel(), _stream())
+    _check(code, "curdkv_compress")
+    return scores, head_sums, idx, head_counts, head_offsets, K_out, V_out
 
 
 class HostBuffers:

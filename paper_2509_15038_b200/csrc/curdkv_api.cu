@@ -55,6 +55,10 @@ inline int tiles_per_head(const curdkv_desc* d) { return (d->n_max + kTileRows -
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
+inline size_t head_counter_bytes(const curdkv_desc* d) {
+  return round256((size_t)d->batch * d->kv_heads * sizeof(int32_t));
+}
+
 // ---- TMA descriptors for the tensor-core sketch kernel ---------------------
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -103,21 +107,21 @@ int sm_count() {
 // host thread (curdkv_profile_next_score).
 thread_local cudaEvent_t g_profile_start = nullptr, g_profile_stop = nullptr;
 
-template <int R>
+template <int R, bool FUSED = false>
 cudaError_t launch_umma(const CUtensorMap& mk, const CUtensorMap& mv, const umma::Args& a,
                         cudaStream_t stream) {
-  using L = umma::Smem<R>;
+  using L = umma::Smem<R, FUSED>;
   const int smem = L::dynamic_bytes(a.seqlens != nullptr ? a.batch : 0);
-  cudaError_t e = cudaFuncSetAttribute(umma::sketch_umma_kernel<R>,
+  cudaError_t e = cudaFuncSetAttribute(umma::sketch_umma_kernel<R, FUSED>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       L::dynamic_bytes(umma::kMaxRaggedBatch));
+                                       L::dynamic_bytes(FUSED ? umma::kMaxRaggedBatchFused : umma::kMaxRaggedBatch));
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   const int64_t tiles = (int64_t)a.batch * a.heads * a.tiles_per_head;   // upper bound if ragged
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
   if (g_profile_start != nullptr) cudaEventRecord(g_profile_start, stream);
-  umma::sketch_umma_kernel<R><<<grid, umma::kThreads, smem, stream>>>(mk, mv, a);
+  umma::sketch_umma_kernel<R, FUSED><<<grid, FUSED ? umma::kFusedThreads : umma::kThreads, smem, stream>>>(mk, mv, a);
   if (g_profile_stop != nullptr) cudaEventRecord(g_profile_stop, stream);
   return cudaSuccess;
 }
@@ -203,12 +207,13 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 extern "C" {
 
 size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32_t adaptive) {
-  (void)max_budget;
   (void)adaptive;
   if (check_desc(desc) != CURDKV_OK) return 0;
   const size_t tiles = (size_t)desc->batch * desc->kv_heads * tiles_per_head(desc);
   const size_t plain = kStatusBytes + round256(tiles * umma::kPartsPerTile * sizeof(float));
-  return desc->whiten ? whiten_layout(desc, plain).total : plain;
+  const size_t score = desc->whiten ? whiten_layout(desc, plain).total : plain;
+  // curdkv_compress also keeps one tile counter per head
+  return score + (max_budget > 0 ? head_counter_bytes(desc) : 0);
 }
 
 curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
@@ -539,6 +544,94 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
   compact_kernel<<<(unsigned)(P * ctas), kCompactWarps * 32, 0, stream>>>(a, (int)ctas);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
+}
+
+curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int32_t g_per_head,
+                              const curdkv_desc* desc, int32_t budget, const int32_t* head_budgets,
+                              int32_t num_sink, int32_t window, int32_t adaptive, double alpha,
+                              float* scores, float* head_sums, int32_t* idx, int32_t* head_counts,
+                              int32_t* head_offsets, void* K_out, void* V_out, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  curdkv_status st = check_desc(desc);
+  if (st != CURDKV_OK) return st;
+  if ((st = check_kv(K, V, desc)) != CURDKV_OK) return st;
+  if (scores == nullptr || head_sums == nullptr || idx == nullptr || head_counts == nullptr ||
+      K_out == nullptr || V_out == nullptr || workspace == nullptr)
+    return CURDKV_ERR_INVALID_ARG;
+  if (budget < 0 || num_sink < 0 || window < 0) return CURDKV_ERR_INVALID_ARG;
+  if (adaptive != 0 && adaptive != 1) return CURDKV_ERR_INVALID_ARG;
+  if (adaptive && head_offsets == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (!aligned16(K_out) || !aligned16(V_out)) return CURDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  const size_t score_bytes = curdkv_workspace_bytes(desc, 0, 0);
+  if (workspace_bytes < score_bytes + head_counter_bytes(desc)) return CURDKV_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t P = (int64_t)desc->batch * desc->kv_heads;
+  const int tiles = tiles_per_head(desc);
+
+  // One launch scores and selects when the tensor-core sketch applies and every head has its own
+  // budget; the selection then hides behind the K/V stream.  Otherwise the three steps follow
+  // one another.
+  const bool fused = !adaptive && budget > 0 && desc->use_projection && !g_per_head && !desc->whiten &&
+                     desc->d == 128 && desc->r >= 1 && desc->r <= 32 && desc->n_max >= kTileRows &&
+                     G != nullptr && P > 0 && P * tiles <= 0x7fffffffLL &&
+                     P * (int64_t)budget <= 0x7fffffffLL;
+  if (!fused) {
+    st = curdkv_score(K, V, G, g_per_head, desc, scores, head_sums, workspace, score_bytes, cuda_stream);
+    if (st == CURDKV_OK)
+      st = curdkv_select(scores, desc, budget, head_budgets, num_sink, window, adaptive, alpha, idx,
+                         head_counts, head_offsets, workspace, score_bytes, cuda_stream);
+  } else {
+    // workspace: status words, one tile counter per head (zero on entry), tile partial sums
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    const size_t counters = head_counter_bytes(desc);
+    if (cudaMemsetAsync(ws, 0, kStatusBytes + counters, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+    int32_t* head_done = reinterpret_cast<int32_t*>(ws + kStatusBytes);
+    float* tile_sums = reinterpret_cast<float*>(ws + kStatusBytes + counters);
+    const int slice = desc->seqlens != nullptr ? umma::kMaxRaggedBatchFused : desc->batch;
+    for (int b0 = 0; b0 < desc->batch; b0 += slice) {
+      curdkv_desc part = *desc;
+      part.batch = desc->batch - b0 < slice ? desc->batch - b0 : slice;
+      const __nv_bfloat16* Kb = static_cast<const __nv_bfloat16*>(K) + (int64_t)b0 * desc->k_stride_b;
+      const __nv_bfloat16* Vb = static_cast<const __nv_bfloat16*>(V) + (int64_t)b0 * desc->v_stride_b;
+      CUtensorMap mk, mv;
+      if (!make_tile_map(&mk, Kb, &part, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) ||
+          !make_tile_map(&mv, Vb, &part, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n))
+        return CURDKV_ERR_CUDA;
+      const size_t p0 = (size_t)b0 * desc->kv_heads;
+      umma::Args u;
+      u.G = G;
+      u.seqlens = desc->seqlens != nullptr ? desc->seqlens + b0 : nullptr;
+      u.batch = part.batch;
+      u.heads = desc->kv_heads;
+      u.n_max = desc->n_max;
+      u.r = desc->r;
+      u.tiles_per_head = tiles;
+      u.score_mode = desc->score_mode;
+      u.scores = scores + p0 * desc->n_max;
+      u.tile_sums = tile_sums + p0 * tiles * umma::kPartsPerTile;
+      u.status = static_cast<uint32_t*>(workspace);
+      u.head_sums = head_sums + p0;
+      u.head_done = head_done + p0;
+      u.head_budgets = head_budgets != nullptr ? head_budgets + p0 : nullptr;
+      u.idx = idx + p0 * budget;
+      u.counts = head_counts + p0;
+      u.offsets = head_offsets != nullptr ? head_offsets + p0 : nullptr;
+      u.budget = budget;
+      u.num_sink = num_sink;
+      u.window = window;
+      u.raw = desc->raw_scores;
+      u.first_head = (int)p0;
+      u.all_heads = (int)P;
+      if (launch_umma<32, true>(mk, mv, u, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+      if (!launch_ok()) return CURDKV_ERR_CUDA;
+    }
+    g_profile_start = g_profile_stop = nullptr;
+  }
+  if (st != CURDKV_OK) return st;
+  if (!adaptive && budget == 0) return CURDKV_OK;          // nothing is kept, nothing to gather
+  return curdkv_compact(K, V, desc, idx, adaptive ? 0 : budget, head_counts, head_offsets, K_out, V_out,
+                        adaptive ? 0 : budget, workspace, cuda_stream);
 }
 
 curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, void* cuda_stream) {

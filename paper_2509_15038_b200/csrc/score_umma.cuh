@@ -21,11 +21,19 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "select.cuh"
 
 namespace curdkv {
 namespace umma {
 
 constexpr int kThreads = 192;
+// The fused form adds a group of selection warps behind the six pipeline warps: whenever this CTA
+// writes the last tile of a head, they normalise that head's scores and select its tokens (Alg. 1
+// lines 6-9) while the pipeline goes on streaming.
+constexpr int kFusedSelThreads = 256;
+constexpr int kFusedThreads = kThreads + kFusedSelThreads;
+constexpr int kFusedListCap = 4096;                        // candidate list of the selection warps
+constexpr int kFusedQueue = 64;                            // finished heads waiting for the selection warps
 // Ring of tensor tiles.  Four 32 KB slots per SM keep HBM saturated; a deeper
 // ring measurably lowers the achieved read bandwidth on B200.
 constexpr int kSlots = 4;
@@ -45,6 +53,15 @@ struct Args {
   float* tile_sums;        // [batch*heads][tiles_per_head][kPartsPerTile]
   uint32_t* status;
   unsigned long long wait_ns = kWaitLimitNs;   // limit of each pipeline wait
+  // fused selection only (sketch_umma_kernel<R, true>); pointers are those of this launch's first head
+  float* head_sums = nullptr;          // [batch*heads]
+  int32_t* head_done = nullptr;        // [batch*heads] tiles written so far, zero on entry
+  const int32_t* head_budgets = nullptr;
+  int32_t* idx = nullptr;              // [batch*heads][budget]
+  int32_t* counts = nullptr;
+  int32_t* offsets = nullptr;          // or nullptr
+  int budget = 0, num_sink = 0, window = 0, raw = 0;
+  int first_head = 0, all_heads = 0;   // position of this launch's heads in the caller's batch
 };
 
 // Ragged batches: the kernel walks only the tiles that hold valid rows.  Every
@@ -52,15 +69,17 @@ struct Args {
 // memory and maps a running tile number to (sequence, head, tile) by binary
 // search, so all CTAs get the same number of real tiles.
 constexpr int kMaxRaggedBatch = 8192;                      // sequences per launch with seqlens
+constexpr int kMaxRaggedBatchFused = 4096;                 // ... when the candidate list shares the space
 
-template <int R>
+template <int R, bool FUSED = false>
 struct Smem {                                     // offsets from the 1024-aligned base
   static constexpr int kN = 2 * R;                // MMA N: [G_hi | G_lo]
   static constexpr int kGHalf = kN * 128;         // bytes per 64-channel span of G^T
   static constexpr int kG = 0;
   static constexpr int kSlot0 = 2 * kGHalf;
   static constexpr int kBar = kSlot0 + kSlots * kSlotBytes;
-  static constexpr int kPrefix = kBar + 256;      // int32 [batch + 1], ragged launches only
+  static constexpr int kList = kBar + 256;        // (key, index) pairs of the selection warps
+  static constexpr int kPrefix = kList + (FUSED ? kFusedListCap * 8 : 0);   // int32 [batch + 1], ragged launches only
   static constexpr int kFixed = kPrefix + 1024;   // + slack for manual alignment
   static constexpr int dynamic_bytes(int ragged_batch) {
     return kFixed + (ragged_batch > 0 ? (ragged_batch + 1) * 4 : 0);
@@ -212,12 +231,118 @@ __device__ __forceinline__ float sketch_row_norm(uint32_t taddr) {
   return acc;
 }
 
+// ---- fused selection ---------------------------------------------------------
+struct FusedSmem {
+  SelectSmem sel;
+  int queue[kFusedQueue];      // heads whose last tile this CTA wrote; -1 = empty slot
+  int reserved, taken;         // slots handed out to producers / consumed by the selection warps
+  int producers_done;          // epilogue warps that have left their loop
+  int tile_parts[4];           // epilogue warps that have written their quarter of a tile in flight
+  int current;                 // head the selection warps work on
+};
+
+// An epilogue warp's lane 0 hands a finished head to the selection warps of its CTA.
+__device__ __forceinline__ void fused_push(FusedSmem& fs, int p, const Args& a, volatile int* abort_flag) {
+  const int slot = atomicAdd(&fs.reserved, 1);
+  unsigned long long t0 = 0;
+  for (uint32_t spin = 1; slot - *(volatile int*)&fs.taken >= kFusedQueue; ++spin) {
+    if ((spin & 0xffu) == 0) {                             // a full queue: wait (bounded) for the consumers
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (*abort_flag || now - t0 > a.wait_ns) {
+        *abort_flag = 1;
+        flag_status(a.status, CURDKV_DEV_TIMEOUT);
+        return;
+      }
+    }
+  }
+  *(volatile int*)&fs.queue[slot % kFusedQueue] = p;
+}
+
+// Thread 0 of the selection warps: next finished head, or -1 when the epilogue warps have left and
+// the queue is empty.
+__device__ __forceinline__ int fused_pop(FusedSmem& fs, const Args& a) {
+  unsigned long long t0 = 0;
+  for (uint32_t spin = 1;; ++spin) {
+    const int at = fs.taken % kFusedQueue;
+    const int p = *(volatile int*)&fs.queue[at];
+    if (p >= 0) {
+      *(volatile int*)&fs.queue[at] = -1;
+      __threadfence_block();
+      *(volatile int*)&fs.taken = fs.taken + 1;
+      __threadfence();                                     // the head's scores were written by other CTAs
+      return p;
+    }
+    if (*(volatile int*)&fs.producers_done == 4 && *(volatile int*)&fs.reserved == fs.taken) return -1;
+    __nanosleep(200);
+    if ((spin & 0x3ffu) == 0) {
+      // the producers' own waits are bounded, so this ends; the limit is a second line of defence
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > 32ull * a.wait_ns) {
+        flag_status(a.status, CURDKV_DEV_TIMEOUT);
+        return -1;
+      }
+    }
+  }
+}
+
+// Alg. 1 lines 6-9 for head p by the selection warps (group G of kFusedSelThreads threads): the head
+// sum in the order normalise_kernel forms it, the division on the way into the leading-digit
+// histogram, then the fixed-budget selection of select_fixed_kernel on the normalised scores.
+template <class G>
+__device__ __forceinline__ void fused_select_head(const Args& a, int p, const KeyList& list, SelectSmem& sm) {
+  static_assert(kFusedSelThreads == 256, "the head sum follows normalise_kernel's 256-thread order");
+  const int tid = G::tid(), lane = tid & 31, warp = tid >> 5;
+  const int n = seq_len_of(a.seqlens, p / a.heads, a.n_max);
+  const int tiles = (n + kTileRows - 1) / kTileRows;
+  float* row = a.scores + (size_t)p * a.n_max;
+  const float* mine = a.tile_sums + (size_t)p * a.tiles_per_head * kPartsPerTile;
+  float part = 0.f;                                        // fixed order: thread, warp tree, warp order
+  for (int i = tid; i < tiles * kPartsPerTile; i += kFusedSelThreads) part += __ldcg(mine + i);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+  if (lane == 0) sm.warp_def[warp] = __float_as_uint(part);
+  clear_hist<G>(sm.hist);
+  G::sync();
+  float S = 0.f;
+#pragma unroll
+  for (int w = 0; w < kFusedSelThreads / 32; ++w) S += __uint_as_float(sm.warp_def[w]);
+  if (tid == 0) a.head_sums[p] = S;
+
+  int k = a.budget;
+  if (a.head_budgets != nullptr) k = max(0, min(a.head_budgets[p], a.budget));
+  const int k_eff = min(k, n);
+  const ForcedSet F = forced_set(n, k_eff, a.num_sink, a.window);
+  RowKeys keys = global_keys(row, n, F);
+  keys.written_here = true;
+  scale_row_and_histogram<G>(row, keys, a.n_max, tiles * kTileRows, S, a.raw != 0, sm.hist);
+  G::sync();
+  select_fixed_row<G>(keys, F, k_eff, a.budget, nullptr, 0, list, true, a.idx + (size_t)p * a.budget, sm);
+  if (tid == 0) {
+    a.counts[p] = k_eff;
+    if (a.offsets != nullptr) {                            // heads sit at multiples of `budget` rows
+      const int gp = a.first_head + p;
+      a.offsets[p] = gp * a.budget;
+      if (gp == a.all_heads - 1) a.offsets[p + 1] = (gp + 1) * a.budget;
+    }
+  }
+}
+
+template <bool FUSED>
+struct FusedState {
+  FusedSmem s;
+};
+template <>
+struct FusedState<false> {};
+
 // ---------------------------------------------------------------------------
-template <int R>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int R, bool FUSED = false>
+__global__ void __launch_bounds__(FUSED ? kFusedThreads : kThreads, 1)
 sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const Args a) {
-  using L = Smem<R>;
+  using L = Smem<R, FUSED>;
+  __shared__ FusedState<FUSED> fused;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -241,6 +366,13 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if constexpr (FUSED) {
+    if (tid < kFusedQueue) fused.s.queue[tid] = -1;
+    if (tid == 0) {
+      fused.s.reserved = fused.s.taken = fused.s.producers_done = 0;
+      fused.s.tile_parts[0] = fused.s.tile_parts[1] = fused.s.tile_parts[2] = fused.s.tile_parts[3] = 0;
+    }
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(tmem_holder)),
@@ -255,21 +387,25 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     uint32_t* chunk_tot = reinterpret_cast<uint32_t*>(base_ptr + L::kSlot0);   // ring not in use yet
     const int per = (a.batch + kThreads - 1) / kThreads;
     const int b0 = min(tid * per, a.batch), b1 = min(b0 + per, a.batch);
-    uint32_t sum = 0;
-    for (int b = b0; b < b1; ++b)
-      sum += (uint32_t)a.heads * (uint32_t)((seq_len_of(a.seqlens, b, a.n_max) + kTileRows - 1) / kTileRows);
-    chunk_tot[tid] = sum;
-    __syncthreads();
-    uint32_t before = 0;
-    for (int i = 0; i < tid; ++i) before += chunk_tot[i];
-    for (int b = b0; b < b1; ++b) {
-      pre[b] = before;
-      before += (uint32_t)a.heads * (uint32_t)((seq_len_of(a.seqlens, b, a.n_max) + kTileRows - 1) / kTileRows);
+    if (tid < kThreads) {                                  // the pipeline warps (all, unless fused)
+      uint32_t sum = 0;
+      for (int b = b0; b < b1; ++b)
+        sum += (uint32_t)a.heads * (uint32_t)((seq_len_of(a.seqlens, b, a.n_max) + kTileRows - 1) / kTileRows);
+      chunk_tot[tid] = sum;
     }
-    if (tid == kThreads - 1) pre[a.batch] = before;
+    __syncthreads();
+    if (tid < kThreads) {
+      uint32_t before = 0;
+      for (int i = 0; i < tid; ++i) before += chunk_tot[i];
+      for (int b = b0; b < b1; ++b) {
+        pre[b] = before;
+        before += (uint32_t)a.heads * (uint32_t)((seq_len_of(a.seqlens, b, a.n_max) + kTileRows - 1) / kTileRows);
+      }
+      if (tid == kThreads - 1) pre[a.batch] = before;
+    }
     // made visible to every role by the barrier at the end of the set-up
   }
-  for (int i = tid; i < 128 * R; i += kThreads) {
+  for (int i = tid; i < 128 * R; i += (int)blockDim.x) {
     const int t = i / R, c = i % R;                        // channel t, sketch column c
     const float g = c < a.r ? __ldg(a.G + (size_t)t * a.r + c) : 0.f;
     const __nv_bfloat16 hi = __float2bfloat16_rn(g);
@@ -384,7 +520,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
         while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < a.wait_ns) {}
       }
     }
-  } else {
+  } else if (warp < kThreads / 32) {
     // ------------------------------------------------------------ epilogue
     const int quarter = warp & 3;                          // TMEM lanes this warp may read
     // scores are read again by the normaliser and the selection: ask L2 to keep them over
@@ -419,6 +555,47 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
       if (lane == 0)
         a.tile_sums[((size_t)p * a.tiles_per_head + row0 / kTileRows) * kPartsPerTile + quarter] = s;
+      if constexpr (FUSED) {
+        // Count the tile once all four quarters are out; the warp that completes a head's last
+        // tile hands the head to the selection warps of this CTA.  The epilogue warps are never
+        // more than two tiles apart (the accumulator stages see to that): four counters do.
+        __threadfence();                                   // scores and partial sum before the count
+        __syncwarp();
+        if (lane == 0) {
+          int* parts_done = &fused.s.tile_parts[(tile_it - 1) & 3];
+          if (atomicAdd(parts_done, 1) == 3) {
+            *parts_done = 0;
+            __threadfence();
+            const int tiles_of_head = (n + kTileRows - 1) / kTileRows;
+            if (atomicAdd(a.head_done + p, 1) + 1 == tiles_of_head) {
+              __threadfence();
+              fused_push(fused.s, p, a, abort_flag);
+            }
+          }
+        }
+      }
+    }
+    if constexpr (FUSED) {
+      __threadfence_block();
+      if (lane == 0) atomicAdd(&fused.s.producers_done, 1);
+    }
+  } else if constexpr (FUSED) {
+    // ------------------------------------------------------------ selection (Alg. 1 lines 6-9)
+    using G = WarpRange<kThreads, kFusedSelThreads, 1>;
+    const KeyList list{reinterpret_cast<uint2*>(base_ptr + L::kList), &fused.s.sel.list_count[0],
+                       (uint32_t)kFusedListCap};
+    // heads without rows never complete a tile: they are dealt out by CTA
+    if (a.seqlens != nullptr) {
+      for (int p = (int)blockIdx.x; p < a.batch * a.heads; p += (int)gridDim.x)
+        if (seq_len_of(a.seqlens, p / a.heads, a.n_max) == 0) fused_select_head<G>(a, p, list, fused.s.sel);
+    }
+    for (;;) {
+      if (G::tid() == 0) fused.s.current = fused_pop(fused.s, a);
+      G::sync();
+      const int p = fused.s.current;
+      G::sync();
+      if (p < 0) break;
+      fused_select_head<G>(a, p, list, fused.s.sel);
     }
   }
 

@@ -82,11 +82,28 @@ struct KeyList {
   __device__ __forceinline__ int size() const { return (int)min(*count, cap); }
 };
 
-// The CTA-wide helpers below work for CTAs of 1024 threads (four histogram bins per thread) and
-// of 512 threads (eight): short rows run as two 512-thread CTAs per SM, which hides more of the
-// latency of their many short phases.
+// The helpers below are written for a group G of threads that works on one row together: a whole
+// CTA, or a run of warps inside a larger, warp-specialised CTA (the fused score + select kernel).
+// G supplies the thread's rank in the group, the group's size and its barrier.  Sizes: 1024 threads
+// (four histogram bins per thread), 512 (eight; short rows run as two such CTAs per SM, which hides
+// more of the latency of their many short phases) or 256 (sixteen).
+struct WholeCta {
+  static __device__ __forceinline__ int tid() { return (int)threadIdx.x; }
+  static __device__ __forceinline__ int size() { return (int)blockDim.x; }
+  static __device__ __forceinline__ void sync() { __syncthreads(); }
+};
+// Threads [FIRST, FIRST + N) of the CTA, synchronised by the named hardware barrier BAR.
+template <int FIRST, int N, int BAR>
+struct WarpRange {
+  static_assert(N % 32 == 0 && FIRST % 32 == 0 && BAR >= 1 && BAR <= 15, "whole warps, a free barrier");
+  static __device__ __forceinline__ int tid() { return (int)threadIdx.x - FIRST; }
+  static __device__ __forceinline__ int size() { return N; }
+  static __device__ __forceinline__ void sync() { asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(N) : "memory"); }
+};
+
+template <class G>
 __device__ __forceinline__ void clear_hist(uint32_t* hist) {
-  for (int i = threadIdx.x; i < kSelBins / 4; i += blockDim.x)
+  for (int i = G::tid(); i < kSelBins / 4; i += G::size())
     reinterpret_cast<uint4*>(hist)[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
@@ -95,10 +112,10 @@ __device__ __forceinline__ void clear_hist(uint32_t* hist) {
 // inside that digit's bucket in sm.remaining and the number of keys in higher
 // bins in sm.above.  Whole CTA (B consecutive bins per thread); the results are
 // readable after the call.
-template <int B>
+template <class G, int B>
 __device__ __forceinline__ void pick_digit_impl(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
   constexpr int kWarps = kSelBins / (32 * B);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = G::tid(), lane = tid & 31, warp = tid >> 5;
   uint32_t c[B];
 #pragma unroll
   for (int q = 0; q < B / 4; ++q) {
@@ -116,7 +133,7 @@ __device__ __forceinline__ void pick_digit_impl(const uint32_t* hist, uint32_t r
   }
   if (lane == 0) sm.warp_def[warp] = suffix;
   if (tid == 0) { sm.digit = 0; sm.remaining = 0; sm.above = 0; }
-  __syncthreads();
+  G::sync();
   uint32_t w = lane < kWarps ? sm.warp_def[lane] : 0u, wsuf = w;   // inclusive suffix sum over the warps
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -133,19 +150,20 @@ __device__ __forceinline__ void pick_digit_impl(const uint32_t* hist, uint32_t r
     }
     above += c[u];
   }
-  __syncthreads();
+  G::sync();
 }
+template <class G>
 __device__ __forceinline__ void pick_digit(const uint32_t* hist, uint32_t remaining, SelectSmem& sm) {
-  if (blockDim.x == 1024) pick_digit_impl<4>(hist, remaining, sm);
-  else if (blockDim.x == 512) pick_digit_impl<8>(hist, remaining, sm);
-  else pick_digit_impl<16>(hist, remaining, sm);
+  if (G::size() == 1024) pick_digit_impl<G, 4>(hist, remaining, sm);
+  else if (G::size() == 512) pick_digit_impl<G, 8>(hist, remaining, sm);
+  else pick_digit_impl<G, 16>(hist, remaining, sm);
 }
 
 // Number of keys of `hist` in bins above `digit`.  Whole CTA; every thread gets the sum.
-template <int B>
+template <class G, int B>
 __device__ __forceinline__ uint32_t count_above_impl(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
   constexpr int kWarps = kSelBins / (32 * B);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = G::tid(), lane = tid & 31, warp = tid >> 5;
   uint32_t v = 0;
 #pragma unroll
   for (int u = 0; u < B; ++u)
@@ -153,17 +171,18 @@ __device__ __forceinline__ uint32_t count_above_impl(const uint32_t* hist, uint3
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   if (lane == 0) sm.warp_eq[warp] = v;
-  __syncthreads();
+  G::sync();
   uint32_t t = lane < kWarps ? sm.warp_eq[lane] : 0u;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-  __syncthreads();
+  G::sync();
   return t;
 }
+template <class G>
 __device__ __forceinline__ uint32_t count_above(const uint32_t* hist, uint32_t digit, SelectSmem& sm) {
-  if (blockDim.x == 1024) return count_above_impl<4>(hist, digit, sm);
-  if (blockDim.x == 512) return count_above_impl<8>(hist, digit, sm);
-  return count_above_impl<16>(hist, digit, sm);
+  if (G::size() == 1024) return count_above_impl<G, 4>(hist, digit, sm);
+  if (G::size() == 512) return count_above_impl<G, 8>(hist, digit, sm);
+  return count_above_impl<G, 16>(hist, digit, sm);
 }
 
 // Rank keys of one row, four tokens at a time ("quad" q holds tokens
@@ -175,6 +194,8 @@ struct RowKeys {
   const uint4* staged;                                     // nullptr: read global memory
   int n, sinks, hi;                                        // candidates are [sinks, hi)
   bool vec;                                                // row is 16-byte aligned
+  bool written_here = false;                               // the row was written by this kernel: read it
+                                                           // from L2, never through the read-only path
 
   __device__ __forceinline__ int quads() const { return (n + 3) >> 2; }
 
@@ -188,18 +209,19 @@ struct RowKeys {
     if (staged != nullptr) return staged[q];
     const int j = 4 * q;
     if (vec && j >= sinks && j + 3 < hi) {                 // interior quad: four candidates
-      const float4 f = __ldg(reinterpret_cast<const float4*>(row) + q);
+      const float4* at = reinterpret_cast<const float4*>(row) + q;
+      const float4 f = written_here ? __ldcg(at) : __ldg(at);
       return make_uint4(score_key(f.x), score_key(f.y), score_key(f.z), score_key(f.w));
     }
     float f[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = j + i < n ? __ldg(row + j + i) : 0.f;
+    for (int i = 0; i < 4; ++i) f[i] = j + i < n ? (written_here ? __ldcg(row + j + i) : __ldg(row + j + i)) : 0.f;
     return make_uint4(key_of(f[0], j), key_of(f[1], j + 1), key_of(f[2], j + 2), key_of(f[3], j + 3));
   }
 };
 
 __device__ __forceinline__ RowKeys global_keys(const float* row, int n, const ForcedSet& F) {
-  return RowKeys{row, nullptr, n, F.sinks, F.hi, (reinterpret_cast<uintptr_t>(row) & 15u) == 0};
+  return RowKeys{row, nullptr, n, F.sinks, F.hi, (reinterpret_cast<uintptr_t>(row) & 15u) == 0, false};
 }
 
 // Running (digit, count) pair of one thread: equal neighbouring digits are
@@ -224,13 +246,14 @@ constexpr int kSelUnroll = 4;                              // quads in flight pe
 
 // Adds the keys <= ceiling whose bits under `mask` equal `prefix` to the
 // histogram of this pass's digit.  Whole CTA.
+template <class G>
 __device__ __forceinline__ void digit_histogram(const RowKeys& keys, uint32_t ceiling, uint32_t mask,
                                                 uint32_t prefix, int pass, uint32_t* hist) {
-  const int quads = keys.quads(), step = (int)blockDim.x;
+  const int quads = keys.quads(), step = (int)G::size();
   const int shift = pass_shift(pass);
   const uint32_t dmask = pass_digit_mask(pass);
   DigitRun run;
-  for (int q0 = (int)threadIdx.x; q0 < quads; q0 += kSelUnroll * step) {
+  for (int q0 = (int)G::tid(); q0 < quads; q0 += kSelUnroll * step) {
     uint4 v[kSelUnroll];
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u)
@@ -256,10 +279,11 @@ __device__ __forceinline__ void digit_histogram(const RowKeys& keys, uint32_t ce
 
 // Copies the rank keys of a row into shared memory and, on the way, builds the
 // histogram of their leading digit.  Whole CTA; hist must be zero on entry.
+template <class G>
 __device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, uint32_t* hist) {
-  const int quads = src.quads(), step = (int)blockDim.x;
+  const int quads = src.quads(), step = (int)G::size();
   DigitRun run;
-  for (int q0 = (int)threadIdx.x; q0 < quads; q0 += kSelUnroll * step) {
+  for (int q0 = (int)G::tid(); q0 < quads; q0 += kSelUnroll * step) {
     uint4 v[kSelUnroll];
 #pragma unroll
     for (int u = 0; u < kSelUnroll; ++u)
@@ -282,8 +306,7 @@ __device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, ui
 // tokens of warp w precede those of warp w + 1 in token order.
 struct Segments {
   int per_warp, quads;
-  __device__ __forceinline__ explicit Segments(int quads_) : quads(quads_) {
-    const int warps = (int)blockDim.x >> 5;
+  __device__ __forceinline__ Segments(int quads_, int warps) : quads(quads_) {
     per_warp = ((quads_ + warps - 1) / warps + 31) & ~31;  // whole-warp sweeps
   }
   __device__ __forceinline__ int begin(int warp) const { return min(warp * per_warp, quads); }
@@ -299,9 +322,10 @@ __device__ __forceinline__ uint32_t classify(const uint4& v, uint32_t T) {
 
 // Per-segment numbers of keys above / equal to the cut, by sweeping the row.  Whole CTA;
 // the totals land in sm.seg_def / sm.seg_eq (visible after the caller's next barrier).
+template <class G>
 __device__ __forceinline__ void count_sweep(const RowKeys& keys, const Cut& cut, SelectSmem& sm) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const Segments seg(keys.quads());
+  const int lane = G::tid() & 31, warp = G::tid() >> 5;
+  const Segments seg(keys.quads(), G::size() >> 5);
   const int q_end = seg.end(warp);
   uint32_t def_cnt = 0, eq_cnt = 0;
   for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += kSelUnroll * 32) {
@@ -330,11 +354,12 @@ __device__ __forceinline__ void count_sweep(const RowKeys& keys, const Cut& cut,
 // leading digit is above `d_cut` (they are kept whatever the rest of the cut turns out to be) and
 // copies the keys with leading digit d_a (and d_b, if use_b) into the lists.  Whole CTA; totals in
 // sm.seg_def (sm.seg_eq is cleared); list counters must be zero on entry.
+template <class G>
 __device__ __forceinline__ void collect_sweep(const RowKeys& keys, uint32_t d_cut, uint32_t d_a,
                                               const KeyList& list_a, bool use_b, uint32_t d_b,
                                               const KeyList& list_b, SelectSmem& sm) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const Segments seg(keys.quads());
+  const int lane = G::tid() & 31, warp = G::tid() >> 5;
+  const Segments seg(keys.quads(), G::size() >> 5);
   const int q_end = seg.end(warp);
   uint32_t def_cnt = 0;
   for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += kSelUnroll * 32) {
@@ -368,11 +393,12 @@ __device__ __forceinline__ void collect_sweep(const RowKeys& keys, uint32_t d_cu
 }
 
 // digit_histogram over a (complete) list instead of the row.
+template <class G>
 __device__ __forceinline__ void list_histogram(const KeyList& list, uint32_t ceiling, uint32_t mask,
                                                uint32_t prefix, int pass, uint32_t* hist) {
   const int shift = pass_shift(pass), n = list.size();
   const uint32_t dmask = pass_digit_mask(pass);
-  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+  for (int e = G::tid(); e < n; e += G::size()) {
     const uint32_t key = list.items[e].x;
     if ((key & mask) == prefix && key <= ceiling) atomicAdd(&hist[(key >> shift) & dmask], 1u);
   }
@@ -380,10 +406,11 @@ __device__ __forceinline__ void list_histogram(const KeyList& list, uint32_t cei
 
 // Adds the list's keys above / equal to the cut to the per-segment totals (the list holds every
 // key whose leading digit equals the cut's; keys with a higher digit were counted by collect_sweep).
+template <class G>
 __device__ __forceinline__ void count_from_list(const KeyList& list, const Cut& cut, const Segments& seg,
                                                 SelectSmem& sm) {
   const int n = list.size();
-  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+  for (int e = G::tid(); e < n; e += G::size()) {
     const uint2 it = list.items[e];
     if (it.x > cut.T) atomicAdd(&sm.seg_def[seg.of_token(it.y)], 1u);
     else if (it.x == cut.T) atomicAdd(&sm.seg_eq[seg.of_token(it.y)], 1u);
@@ -392,6 +419,7 @@ __device__ __forceinline__ void count_from_list(const KeyList& list, const Cut& 
 
 // Remaining digits of a cut whose leading digit `d0` is known: the `rank`-th largest key (1-based)
 // among the keys of leading digit d0.  Uses the list if it is complete, else sweeps the row.  Whole CTA.
+template <class G>
 __device__ __forceinline__ Cut finish_cut(const RowKeys& keys, const KeyList& list, uint32_t d0,
                                           uint32_t rank, SelectSmem& sm) {
   uint32_t prefix = d0 << 20, mask = 0xfffu << 20, remaining = rank;
@@ -400,8 +428,8 @@ __device__ __forceinline__ Cut finish_cut(const RowKeys& keys, const KeyList& li
     // a short list is ranked directly: thread t counts the keys above and equal to key t (equal
     // keys find the same cut, so it does not matter which of their threads writes it)
     const int L = list.size();
-    if ((int)threadIdx.x < L) {
-      const uint32_t key = list.items[threadIdx.x].x;
+    if ((int)G::tid() < L) {
+      const uint32_t key = list.items[G::tid()].x;
       uint32_t gt = 0, eq = 0;
       for (int e = 0; e < L; ++e) {
         const uint32_t other = list.items[e].x;
@@ -413,22 +441,22 @@ __device__ __forceinline__ Cut finish_cut(const RowKeys& keys, const KeyList& li
         sm.remaining = rank - gt;
       }
     }
-    __syncthreads();
+    G::sync();
     const Cut cut{sm.digit, sm.remaining};
-    __syncthreads();                                       // sm.digit may be rewritten
+    G::sync();                                       // sm.digit may be rewritten
     return cut;
   }
   for (int pass = 1; pass < kSelPasses; ++pass) {
-    clear_hist(sm.hist);
-    __syncthreads();
-    if (from_list) list_histogram(list, 0xffffffffu, mask, prefix, pass, sm.hist);
-    else digit_histogram(keys, 0xffffffffu, mask, prefix, pass, sm.hist);
-    __syncthreads();
-    pick_digit(sm.hist, remaining, sm);
+    clear_hist<G>(sm.hist);
+    G::sync();
+    if (from_list) list_histogram<G>(list, 0xffffffffu, mask, prefix, pass, sm.hist);
+    else digit_histogram<G>(keys, 0xffffffffu, mask, prefix, pass, sm.hist);
+    G::sync();
+    pick_digit<G>(sm.hist, remaining, sm);
     prefix |= sm.digit << pass_shift(pass);
     mask |= pass_digit_mask(pass) << pass_shift(pass);
     remaining = sm.remaining;
-    __syncthreads();
+    G::sync();
   }
   return Cut{prefix, remaining};
 }
@@ -436,15 +464,16 @@ __device__ __forceinline__ Cut finish_cut(const RowKeys& keys, const KeyList& li
 // Ordered write of one row: the tokens whose key is above cut.T and the first cut.eq_take tokens
 // whose key equals cut.T go to `out` in ascending token order.  The per-segment totals must be in
 // sm.seg_def / sm.seg_eq (from count_sweep, or collect_sweep + count_from_list).  Whole CTA.
+template <class G>
 __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut, int32_t* out,
                                             SelectSmem& sm) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const Segments seg(keys.quads());
+  const int lane = G::tid() & 31, warp = G::tid() >> 5;
+  const Segments seg(keys.quads(), G::size() >> 5);
   const int q_begin = seg.begin(warp), q_end = seg.end(warp);
-  __syncthreads();
+  G::sync();
   uint32_t def_before = 0, eq_before = 0;                  // kept / equal tokens of earlier warps
   {
-    const bool live = lane < ((int)blockDim.x >> 5);       // one segment per warp of the CTA
+    const bool live = lane < ((int)G::size() >> 5);       // one segment per warp of the CTA
     const uint32_t d = live ? sm.seg_def[lane] : 0u, e = live ? sm.seg_eq[lane] : 0u;
     uint32_t di = d, ei = e;
 #pragma unroll
@@ -492,31 +521,67 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
     def_before += dtot;
     eq_before += etot;
   }
-  __syncthreads();                                         // sm.warp_* may be reused
+  G::sync();                                         // sm.warp_* may be reused
+}
+
+// Alg. 1 line 6 for one row, on the way to the selection: row[j] <- row[j] / S for j < n (0 when the
+// sum is not positive; left as it is with `raw`), row[j] <- 0 for first_unwritten <= j < n_max, and
+// the leading-digit histogram of the resulting rank keys in `hist` (zero on entry).  The row was
+// written by other CTAs of this kernel: it is read from L2.  Group G.
+template <class G>
+__device__ __forceinline__ void scale_row_and_histogram(float* row, const RowKeys& keys, int n_max,
+                                                        int first_unwritten, float S, bool raw,
+                                                        uint32_t* hist) {
+  const int n = keys.n, step = G::size();
+  const bool live = S > 0.f;
+  auto scaled = [&](float x) { return raw ? x : (live ? __fdiv_rn(x, S) : 0.f); };
+  DigitRun run;
+  int done = 0;
+  if (keys.vec) {
+    const int quads = n >> 2;                              // whole quads of valid tokens
+    for (int q0 = G::tid(); q0 < quads; q0 += kSelUnroll * step) {
+      float4 f[kSelUnroll];
+#pragma unroll
+      for (int u = 0; u < kSelUnroll; ++u)
+        if (q0 + u * step < quads) f[u] = __ldcg(reinterpret_cast<const float4*>(row) + q0 + u * step);
+#pragma unroll
+      for (int u = 0; u < kSelUnroll; ++u) {
+        const int q = q0 + u * step;
+        if (q < quads) {
+          const float4 o = make_float4(scaled(f[u].x), scaled(f[u].y), scaled(f[u].z), scaled(f[u].w));
+          if (!raw) reinterpret_cast<float4*>(row)[q] = o;
+          run.add(keys.key_of(o.x, 4 * q) >> 20, hist);
+          run.add(keys.key_of(o.y, 4 * q + 1) >> 20, hist);
+          run.add(keys.key_of(o.z, 4 * q + 2) >> 20, hist);
+          run.add(keys.key_of(o.w, 4 * q + 3) >> 20, hist);
+        }
+      }
+    }
+    done = quads << 2;
+  }
+  for (int j = done + G::tid(); j < n; j += step) {
+    const float o = scaled(__ldcg(row + j));
+    if (!raw) row[j] = o;
+    run.add(keys.key_of(o, j) >> 20, hist);
+  }
+  run.flush(hist);
+  for (int j = first_unwritten + G::tid(); j < n_max; j += step) row[j] = 0.f;
 }
 
 // ---------------------------------------------------------------------------
-// Fixed per-head budget.  grid = batch*heads, block = 1024, 512 or 256, dynamic shared
-// memory = 16 * stage_quads bytes (0: rows are read from global memory) followed
-// by one candidate list of list_cap entries.
+// Fixed per-head budget, one row, by the group G: Alg. 1 lines 7-9 on the scores `keys` describes.
+// k_eff = min(k, n) rows are kept; their ascending indices go to out[0, k_eff), -1 to
+// out[k_eff, budget).  `staged` (stage_quads quads, or nothing) may hold a copy of the keys;
+// `hist_ready` says that sm.hist already holds the leading-digit histogram of the row's keys (the
+// caller built it while it had the scores in hand).
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
-    const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
-    int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window, int stage_quads,
-    int list_cap, int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
-  __shared__ SelectSmem sm;
-  extern __shared__ uint4 staged_keys[];                   // stage_quads quads, or nothing
-  const int p = blockIdx.x, b = p / heads, tid = threadIdx.x;
-  const int n = seq_len_of(seqlens, b, n_max);
-  int k = budget;
-  if (head_budgets != nullptr) k = max(0, min(head_budgets[p], budget));
-  const int k_eff = min(k, n);
-  const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
-  int32_t* out = idx + (size_t)p * budget;
-
+template <class G>
+__device__ __forceinline__ void select_fixed_row(RowKeys keys, const ForcedSet& F, int k_eff, int budget,
+                                                 uint4* staged, int stage_quads, const KeyList& list,
+                                                 bool hist_ready, int32_t* out, SelectSmem& sm) {
+  const int tid = G::tid(), n = keys.n;
   Cut cut;
-  bool counted = false;                                    // per-segment totals already in sm.warp_*
+  bool counted = false;                                    // per-segment totals already in sm.seg_*
   if (k_eff == 0) {
     cut = keep_nothing();
   } else if (k_eff == n) {
@@ -525,34 +590,56 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     cut = keep_forced_only();
   } else {
     // sweep 1: leading-digit histogram (staging the keys on the way if the row fits)
-    clear_hist(sm.hist);
-    if (tid == 0) sm.list_count[0] = 0;
-    __syncthreads();
-    if (keys.quads() <= stage_quads) {
-      stage_keys(keys, staged_keys, sm.hist);
-      keys.staged = staged_keys;
-    } else {
-      digit_histogram(keys, 0xffffffffu, 0u, 0u, 0, sm.hist);
+    if (!hist_ready) {
+      clear_hist<G>(sm.hist);
+      if (tid == 0) *list.count = 0;
+      G::sync();
+      if (keys.quads() <= stage_quads) {
+        stage_keys<G>(keys, staged, sm.hist);
+        keys.staged = staged;
+      } else {
+        digit_histogram<G>(keys, 0xffffffffu, 0u, 0u, 0, sm.hist);
+      }
+    } else if (tid == 0) {
+      *list.count = 0;
     }
-    __syncthreads();
-    pick_digit(sm.hist, (uint32_t)k_eff, sm);
+    G::sync();
+    pick_digit<G>(sm.hist, (uint32_t)k_eff, sm);
     const uint32_t d0 = sm.digit, rank = sm.remaining;
-    __syncthreads();
+    G::sync();
     // sweep 2: keys above the digit are counted per segment, keys of the digit go to the list
-    const KeyList list{reinterpret_cast<uint2*>(staged_keys + stage_quads), &sm.list_count[0],
-                       (uint32_t)list_cap};
-    collect_sweep(keys, d0, d0, list, false, 0u, list, sm);
-    __syncthreads();
-    cut = finish_cut(keys, list, d0, rank, sm);
+    collect_sweep<G>(keys, d0, d0, list, false, 0u, list, sm);
+    G::sync();
+    cut = finish_cut<G>(keys, list, d0, rank, sm);
     if (list.complete()) {
-      count_from_list(list, cut, Segments(keys.quads()), sm);
+      count_from_list<G>(list, cut, Segments(keys.quads(), G::size() >> 5), sm);
       counted = true;
     }
   }
-  if (!counted) count_sweep(keys, cut, sm);
-  write_sweep(keys, cut, out, sm);
-  for (int t = k_eff + tid; t < budget; t += (int)blockDim.x) out[t] = -1;
-  if (tid == 0) {
+  if (!counted) count_sweep<G>(keys, cut, sm);
+  write_sweep<G>(keys, cut, out, sm);
+  for (int t = k_eff + tid; t < budget; t += G::size()) out[t] = -1;
+}
+
+// grid = batch*heads, block = 1024, 512 or 256, dynamic shared memory = 16 * stage_quads bytes
+// (0: rows are read from global memory) followed by one candidate list of list_cap entries.
+__global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
+    const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
+    int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window, int stage_quads,
+    int list_cap, int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+  __shared__ SelectSmem sm;
+  extern __shared__ uint4 staged_keys[];                   // stage_quads quads, or nothing
+  using G = WholeCta;
+  const int p = blockIdx.x, b = p / heads;
+  const int n = seq_len_of(seqlens, b, n_max);
+  int k = budget;
+  if (head_budgets != nullptr) k = max(0, min(head_budgets[p], budget));
+  const int k_eff = min(k, n);
+  const ForcedSet F = forced_set(n, k_eff, num_sink, window);
+  const RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
+  const KeyList list{reinterpret_cast<uint2*>(staged_keys + stage_quads), &sm.list_count[0], (uint32_t)list_cap};
+  select_fixed_row<G>(keys, F, k_eff, budget, staged_keys, stage_quads, list, false, idx + (size_t)p * budget, sm);
+  if (threadIdx.x == 0) {
     counts[p] = k_eff;
     if (offsets != nullptr) {                              // heads sit at multiples of `budget` rows
       offsets[p] = p * budget;
@@ -588,6 +675,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
     int budget, int num_sink, int window, int min_protected, int32_t* __restrict__ idx,
     int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   __shared__ AdaptiveSmem sm;
+  using G = WholeCta;
   extern __shared__ uint4 adaptive_dyn[];
   uint32_t* hist_all = reinterpret_cast<uint32_t*>(adaptive_dyn);          // leading digits of all keys
   constexpr int B = kSelBins / THREADS, Q = B / 4;         // histogram bins (quads of bins) per thread
@@ -609,14 +697,14 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
 
   // ---- sweep 1: leading-digit histogram of the row; leading digit of this head's safeguard cut
   // (its `prot` largest keys) and how many keys of that digit the cut takes
-  clear_hist(hist_all);
+  clear_hist<G>(hist_all);
   if (tid == 0) sm.s.list_count[0] = sm.s.list_count[1] = 0;
   __syncthreads();
-  if (!all) digit_histogram(keys, 0xffffffffu, 0u, 0u, 0, hist_all);
+  if (!all) digit_histogram<G>(keys, 0xffffffffu, 0u, 0u, 0, hist_all);
   __syncthreads();
   uint32_t d0 = 0xffffffffu, rank_own = 0;
   if (!none && !all) {
-    pick_digit_impl<B>(hist_all, (uint32_t)prot, sm.s);
+    pick_digit_impl<G, B>(hist_all, (uint32_t)prot, sm.s);
     d0 = sm.s.digit;
     rank_own = sm.s.remaining;
     __syncthreads();
@@ -651,10 +739,10 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
       reinterpret_cast<uint4*>(sm.s.hist)[tid * Q + q] = acc;
     }
     __syncthreads();
-    pick_digit_impl<B>(sm.s.hist, remaining, sm.s);
+    pick_digit_impl<G, B>(sm.s.hist, remaining, sm.s);
     dg = sm.s.digit;
     remaining = sm.s.remaining;
-    local_gt = count_above_impl<B>(sm.hist_local, dg, sm.s);
+    local_gt = count_above_impl<G, B>(sm.hist_local, dg, sm.s);
     cluster.sync();                                        // peers are done reading hist_local
   }
 
@@ -666,13 +754,13 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
   const uint32_t d_cut = global_lower ? dg : d0;
   const bool share = !none && dg == d0;                    // one list serves both cuts
   const bool swept = !all && (pool > 0 || !none);
-  if (swept) collect_sweep(keys, d_cut, d0, list_a, pool > 0 && !share, dg, list_b, sm.s);
+  if (swept) collect_sweep<G>(keys, d_cut, d0, list_a, pool > 0 && !share, dg, list_b, sm.s);
   __syncthreads();
 
   // ---- this head's safeguard cut
   Cut own = keep_nothing();
   if (all) own = keep_every_token();
-  else if (!none) own = finish_cut(keys, list_a, d0, rank_own, sm.s);
+  else if (!none) own = finish_cut<G>(keys, list_a, d0, rank_own, sm.s);
   // unprotected keys: those <= own.T, minus the first own.eq_take equal to it
   const uint32_t ceiling = own.T;
 
@@ -683,11 +771,11 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
     uint32_t prefix = dg << 20, mask = 0xfffu << 20;
     for (int pass = 1; pass < kSelPasses; ++pass) {
       const int shift = pass_shift(pass);
-      clear_hist(sm.hist_local);
+      clear_hist<G>(sm.hist_local);
       __syncthreads();
       if (!all) {
-        if (list_g.complete()) list_histogram(list_g, ceiling, mask, prefix, pass, sm.hist_local);
-        else digit_histogram(keys, ceiling, mask, prefix, pass, sm.hist_local);
+        if (list_g.complete()) list_histogram<G>(list_g, ceiling, mask, prefix, pass, sm.hist_local);
+        else digit_histogram<G>(keys, ceiling, mask, prefix, pass, sm.hist_local);
       }
       __syncthreads();
       if (tid == 0 && own.eq_take > 0 && (own.T & mask) == prefix)
@@ -704,12 +792,12 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
         reinterpret_cast<uint4*>(sm.s.hist)[tid * Q + q] = acc;
       }
       __syncthreads();
-      pick_digit_impl<B>(sm.s.hist, remaining, sm.s);
+      pick_digit_impl<G, B>(sm.s.hist, remaining, sm.s);
       const uint32_t dgt = sm.s.digit;
       remaining = sm.s.remaining;
       prefix |= dgt << shift;
       mask |= pass_digit_mask(pass) << shift;
-      local_gt += count_above_impl<B>(sm.hist_local, dgt, sm.s);
+      local_gt += count_above_impl<G, B>(sm.hist_local, dgt, sm.s);
       if (pass == kSelPasses - 1) local_eq = sm.hist_local[dgt];
       cluster.sync();                                      // peers are done reading hist_local
     }
@@ -748,9 +836,9 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
 
   // ---- per-segment totals, then the ordered write (sweep 3)
   const KeyList& list_c = global_lower ? list_b : list_a;  // holds the keys of the cut's leading digit
-  if (swept && list_c.complete()) count_from_list(list_c, cut, Segments(keys.quads()), sm.s);
-  else count_sweep(keys, cut, sm.s);
-  write_sweep(keys, cut, idx + off, sm.s);
+  if (swept && list_c.complete()) count_from_list<G>(list_c, cut, Segments(keys.quads(), THREADS >> 5), sm.s);
+  else count_sweep<G>(keys, cut, sm.s);
+  write_sweep<G>(keys, cut, idx + off, sm.s);
   if (tid == 0) {
     counts[p] = (int32_t)kept;
     offsets[p] = (int32_t)off;
