@@ -176,6 +176,15 @@ def run_cuda(args):
             events[0].record()
         if sketch_events is not None:
             cur.curdkv_profile_next_score(*sketch_events)
+        if not args.three_calls:
+            # the whole path in one call; for fixed budgets its first kernel scores AND selects
+            cur.curdkv_compress(K, V, G, desc, w.budget, ws, num_sink=w.num_sink, window=w.window,
+                                adaptive=w.adaptive, alpha=w.alpha, scores=scores, head_sums=sums, idx=idx,
+                                head_counts=cnt, head_offsets=off, K_out=Ko, V_out=Vo)
+            if events is not None:
+                for e in events[1:]:
+                    e.record()
+            return
         cur.curdkv_score(K, V, G, desc, ws, scores=scores, head_sums=sums)
         if events is not None:
             events[1].record()
@@ -640,6 +649,8 @@ def main():
                     help="layers instead of the workload's own (cfg1-cfg5 only); 0 keeps them")
     ap.add_argument("--graph", action="store_true",
                     help="also time the step replayed from a CUDA graph (extra 'cuda_graph' object)")
+    ap.add_argument("--three-calls", action="store_true",
+                    help="time curdkv_score + curdkv_select + curdkv_compact instead of curdkv_compress")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
                     help="--workload decode: compress inside the cache (unordered) or copy in order")

@@ -55,8 +55,11 @@ inline int tiles_per_head(const curdkv_desc* d) { return (d->n_max + kTileRows -
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
+// What curdkv_compress keeps next to the status words: per head a tile counter and an entry of
+// the list of finished heads, and two queue counters per launch.
+constexpr int kMaxFusedLaunches = 32;
 inline size_t head_counter_bytes(const curdkv_desc* d) {
-  return round256((size_t)d->batch * d->kv_heads * sizeof(int32_t));
+  return round256((size_t)d->batch * d->kv_heads * 2 * sizeof(int32_t)) + round256(kMaxFusedLaunches * 2 * sizeof(int32_t));
 }
 
 // ---- TMA descriptors for the tensor-core sketch kernel ---------------------
@@ -121,9 +124,24 @@ cudaError_t launch_umma(const CUtensorMap& mk, const CUtensorMap& mv, const umma
   const int64_t tiles = (int64_t)a.batch * a.heads * a.tiles_per_head;   // upper bound if ragged
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
   if (g_profile_start != nullptr) cudaEventRecord(g_profile_start, stream);
-  umma::sketch_umma_kernel<R, FUSED><<<grid, FUSED ? umma::kFusedThreads : umma::kThreads, smem, stream>>>(mk, mv, a);
+  if (FUSED) {
+    // the selection groups wait for heads that other CTAs stream: all CTAs must be resident at once
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(umma::kFusedThreads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, umma::sketch_umma_kernel<R, FUSED>, mk, mv, a);
+  } else {
+    umma::sketch_umma_kernel<R, FUSED><<<grid, umma::kThreads, smem, stream>>>(mk, mv, a);
+  }
   if (g_profile_stop != nullptr) cudaEventRecord(g_profile_stop, stream);
-  return cudaSuccess;
+  return e;
 }
 
 // ---- built-in scratch of curdkv_score_static --------------------------------
@@ -572,10 +590,15 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
   // One launch scores and selects when the tensor-core sketch applies and every head has its own
   // budget; the selection then hides behind the K/V stream.  Otherwise the three steps follow
   // one another.
+  // (With fewer than four heads per SM the selection of the last heads, which only starts when the
+  // stream ends and runs on a quarter of a selection CTA's threads, costs more than it saves.)
   const bool fused = !adaptive && budget > 0 && desc->use_projection && !g_per_head && !desc->whiten &&
+                     P >= 4 * (int64_t)sm_count() &&
                      desc->d == 128 && desc->r >= 1 && desc->r <= 32 && desc->n_max >= kTileRows &&
                      G != nullptr && P > 0 && P * tiles <= 0x7fffffffLL &&
-                     P * (int64_t)budget <= 0x7fffffffLL;
+                     P * (int64_t)budget <= 0x7fffffffLL &&
+                     (desc->seqlens == nullptr ||
+                      desc->batch <= (int64_t)kMaxFusedLaunches * umma::kMaxRaggedBatchFused);
   if (!fused) {
     st = curdkv_score(K, V, G, g_per_head, desc, scores, head_sums, workspace, score_bytes, cuda_stream);
     if (st == CURDKV_OK)
@@ -587,6 +610,8 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
     const size_t counters = head_counter_bytes(desc);
     if (cudaMemsetAsync(ws, 0, kStatusBytes + counters, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
     int32_t* head_done = reinterpret_cast<int32_t*>(ws + kStatusBytes);
+    int32_t* done_list = head_done + P;
+    int32_t* queue_ctr = reinterpret_cast<int32_t*>(ws + kStatusBytes + round256((size_t)P * 2 * sizeof(int32_t)));
     float* tile_sums = reinterpret_cast<float*>(ws + kStatusBytes + counters);
     const int slice = desc->seqlens != nullptr ? umma::kMaxRaggedBatchFused : desc->batch;
     for (int b0 = 0; b0 < desc->batch; b0 += slice) {
@@ -613,6 +638,8 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
       u.status = static_cast<uint32_t*>(workspace);
       u.head_sums = head_sums + p0;
       u.head_done = head_done + p0;
+      u.done_list = done_list + p0;
+      u.queue_ctr = queue_ctr + 2 * (b0 / slice);
       u.head_budgets = head_budgets != nullptr ? head_budgets + p0 : nullptr;
       u.idx = idx + p0 * budget;
       u.counts = head_counts + p0;
@@ -623,6 +650,11 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
       u.raw = desc->raw_scores;
       u.first_head = (int)p0;
       u.all_heads = (int)P;
+      // chunks of consecutive tiles per CTA visit: long enough to make the per-chunk bookkeeping
+      // rare, short enough that the last, uneven round of chunks stays near 1 % of the launch
+      const int sms = sm_count();
+      const int64_t per_cta = (int64_t)part.batch * desc->kv_heads * tiles / (sms > 0 ? sms : 1);
+      u.chunk_tiles = (int)(per_cta / 64 < 1 ? 1 : (per_cta / 64 > 16 ? 16 : per_cta / 64));
       if (launch_umma<32, true>(mk, mv, u, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
       if (!launch_ok()) return CURDKV_ERR_CUDA;
     }

@@ -31,9 +31,10 @@ constexpr int kThreads = 192;
 // writes the last tile of a head, they normalise that head's scores and select its tokens (Alg. 1
 // lines 6-9) while the pipeline goes on streaming.
 constexpr int kFusedSelThreads = 256;
-constexpr int kFusedThreads = kThreads + kFusedSelThreads;
+constexpr int kFusedSelFirst = kThreads + 32;              // one publisher warp sits between the two groups
+constexpr int kFusedThreads = kFusedSelFirst + kFusedSelThreads;
 constexpr int kFusedListCap = 4096;                        // candidate list of the selection warps
-constexpr int kFusedQueue = 64;                            // finished heads waiting for the selection warps
+constexpr int kFusedRuns = 32;                             // runs of tiles between the epilogue and the publisher
 // Ring of tensor tiles.  Four 32 KB slots per SM keep HBM saturated; a deeper
 // ring measurably lowers the achieved read bandwidth on B200.
 constexpr int kSlots = 4;
@@ -56,12 +57,34 @@ struct Args {
   // fused selection only (sketch_umma_kernel<R, true>); pointers are those of this launch's first head
   float* head_sums = nullptr;          // [batch*heads]
   int32_t* head_done = nullptr;        // [batch*heads] tiles written so far, zero on entry
+  int32_t* done_list = nullptr;        // [batch*heads] finished heads (index + 1) in the order they finished; zero on entry
+  int32_t* queue_ctr = nullptr;        // [2] heads entered into done_list / tickets handed to selection groups; zero on entry
   const int32_t* head_budgets = nullptr;
   int32_t* idx = nullptr;              // [batch*heads][budget]
   int32_t* counts = nullptr;
   int32_t* offsets = nullptr;          // or nullptr
   int budget = 0, num_sink = 0, window = 0, raw = 0;
   int first_head = 0, all_heads = 0;   // position of this launch's heads in the caller's batch
+  // Tiles are dealt to the CTAs in chunks of this many consecutive tiles (1: tile t goes to CTA
+  // t mod grid).  The fused kernel counts a head's tiles once per chunk instead of once per tile.
+  int chunk_tiles = 1;
+};
+
+// The tiles of one CTA in the order every role walks them: chunks first, first + stride, ... of
+// `chunk` consecutive tiles each.
+struct TileWalk {
+  uint32_t chunk_no, i, chunk, stride, total;
+  __device__ __forceinline__ TileWalk(uint32_t first, uint32_t stride_, uint32_t chunk_, uint32_t total_)
+      : chunk_no(first), i(0), chunk(chunk_), stride(stride_), total(total_) {}
+  __device__ __forceinline__ bool valid() const { return chunk_no * chunk + i < total; }
+  __device__ __forceinline__ uint32_t tile() const { return chunk_no * chunk + i; }
+  __device__ __forceinline__ bool starts_chunk() const { return i == 0; }
+  __device__ __forceinline__ void next() {
+    if (++i == chunk || chunk_no * chunk + i >= total) {
+      i = 0;
+      chunk_no += stride;
+    }
+  }
 };
 
 // Ragged batches: the kernel walks only the tiles that hold valid rows.  Every
@@ -232,55 +255,53 @@ __device__ __forceinline__ float sketch_row_norm(uint32_t taddr) {
 }
 
 // ---- fused selection ---------------------------------------------------------
+// A "run" is a stretch of consecutive tiles of one head inside one chunk.  When the four epilogue
+// warps have written a run's scores they arrive on the run's barrier; the publisher warp takes it
+// from there (device-wide fence, count, hand-over), so no epilogue warp ever waits on a fence or on
+// an atomic's round trip.
 struct FusedSmem {
   SelectSmem sel;
-  int queue[kFusedQueue];      // heads whose last tile this CTA wrote; -1 = empty slot
-  int reserved, taken;         // slots handed out to producers / consumed by the selection warps
+  alignas(8) unsigned long long run_bar[kFusedRuns];
+  int run_head[kFusedRuns], run_tiles[kFusedRuns], run_total[kFusedRuns];   // head, tiles in the run, tiles of the head
+  int published;               // runs the publisher is done with
+  int final_runs[4];           // runs each epilogue warp closed before it left its loop
   int producers_done;          // epilogue warps that have left their loop
-  int tile_parts[4];           // epilogue warps that have written their quarter of a tile in flight
+  int nonempty;                // heads of this launch that have rows (each of them gets finished once)
   int current;                 // head the selection warps work on
 };
 
-// An epilogue warp's lane 0 hands a finished head to the selection warps of its CTA.
-__device__ __forceinline__ void fused_push(FusedSmem& fs, int p, const Args& a, volatile int* abort_flag) {
-  const int slot = atomicAdd(&fs.reserved, 1);
-  unsigned long long t0 = 0;
-  for (uint32_t spin = 1; slot - *(volatile int*)&fs.taken >= kFusedQueue; ++spin) {
-    if ((spin & 0xffu) == 0) {                             // a full queue: wait (bounded) for the consumers
-      const unsigned long long now = global_ns();
-      if (t0 == 0) t0 = now;
-      if (*abort_flag || now - t0 > a.wait_ns) {
-        *abort_flag = 1;
-        flag_status(a.status, CURDKV_DEV_TIMEOUT);
-        return;
-      }
-    }
-  }
-  *(volatile int*)&fs.queue[slot % kFusedQueue] = p;
+// Finished heads go through one list in global memory that the selection groups of ALL CTAs serve:
+// whichever CTA happens to write a head's last tile (a few CTAs do so far more often than the
+// rest), the selections are spread evenly.  A lane of a publisher warp enters a head ...
+__device__ __forceinline__ void fused_push(const Args& a, int p) {
+  const int slot = atomicAdd(a.queue_ctr, 1);
+  __threadfence();
+  *(volatile int32_t*)(a.done_list + slot) = p + 1;
 }
 
-// Thread 0 of the selection warps: next finished head, or -1 when the epilogue warps have left and
-// the queue is empty.
-__device__ __forceinline__ int fused_pop(FusedSmem& fs, const Args& a) {
+// ... and thread 0 of a selection group draws a ticket and waits (bounded) for that entry of the
+// list.  Returns -1 when every head with rows has been handed out, or when the launch has failed.
+// The CTAs of the launch are co-resident (cooperative launch), so the heads a ticket waits for are
+// being streamed while it waits.
+__device__ __forceinline__ int fused_pop(const Args& a, int nonempty_heads, volatile int* abort_flag) {
+  const int ticket = atomicAdd(a.queue_ctr + 1, 1);
+  if (ticket >= nonempty_heads) return -1;
   unsigned long long t0 = 0;
   for (uint32_t spin = 1;; ++spin) {
-    const int at = fs.taken % kFusedQueue;
-    const int p = *(volatile int*)&fs.queue[at];
-    if (p >= 0) {
-      *(volatile int*)&fs.queue[at] = -1;
-      __threadfence_block();
-      *(volatile int*)&fs.taken = fs.taken + 1;
+    const int v = *(volatile int32_t*)(a.done_list + ticket);
+    if (v != 0) {
       __threadfence();                                     // the head's scores were written by other CTAs
-      return p;
+      return v - 1;
     }
-    if (*(volatile int*)&fs.producers_done == 4 && *(volatile int*)&fs.reserved == fs.taken) return -1;
-    __nanosleep(200);
-    if ((spin & 0x3ffu) == 0) {
-      // the producers' own waits are bounded, so this ends; the limit is a second line of defence
+    __nanosleep(1000);
+    if ((spin & 0xffu) == 0) {
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      if (now - t0 > 32ull * a.wait_ns) {
+      // a launch that has timed out elsewhere never finishes its heads; the limit itself is a
+      // second line of defence (the other roles' waits are bounded)
+      if ((*(volatile uint32_t*)a.status & CURDKV_DEV_TIMEOUT) != 0 || now - t0 > 32ull * a.wait_ns) {
         flag_status(a.status, CURDKV_DEV_TIMEOUT);
+        *abort_flag = 1;
         return -1;
       }
     }
@@ -367,11 +388,9 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if constexpr (FUSED) {
-    if (tid < kFusedQueue) fused.s.queue[tid] = -1;
-    if (tid == 0) {
-      fused.s.reserved = fused.s.taken = fused.s.producers_done = 0;
-      fused.s.tile_parts[0] = fused.s.tile_parts[1] = fused.s.tile_parts[2] = fused.s.tile_parts[3] = 0;
-    }
+    if (tid < kFusedRuns) mbar_init(smem_u32(&fused.s.run_bar[tid]), 4);
+    if (tid == 0) fused.s.producers_done = fused.s.published = fused.s.nonempty = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -460,9 +479,9 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
       uint32_t it = 0;
       bool ok = true;
-      for (uint32_t t = first; ok && t < total_tiles; t += stride) {
+      for (TileWalk w(first, stride, (uint32_t)a.chunk_tiles, total_tiles); ok && w.valid(); w.next()) {
         int p, row0;
-        locate(t, p, row0);
+        locate(w.tile(), p, row0);
         const int b = p / a.heads, h = p % a.heads;
         for (int tensor = 0; tensor < 2; ++tensor, ++it) {
           const int slot = it % kSlots;
@@ -491,7 +510,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       constexpr uint32_t idesc = instr_desc_bf16(L::kN);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
-      for (uint32_t t = first; ok && t < total_tiles; t += stride) {
+      for (TileWalk w(first, stride, (uint32_t)a.chunk_tiles, total_tiles); ok && w.valid(); w.next()) {
         const uint32_t acc = tile_it & 1u, acc_phase = (tile_it >> 1) & 1u;
         if (!(ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, a.status, a.wait_ns))) break;
         tc_fence_after();
@@ -529,9 +548,42 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
     uint32_t tile_it = 0;
     bool ok = true;
-    for (uint32_t t = first; ok && t < total_tiles; t += stride) {
+    // fused: the run of tiles being written and how many runs this warp has closed
+    int run_head = -1, run_len = 0, run_rows = 0, runs_closed = 0;
+    auto close_run = [&]() {
+      if constexpr (FUSED) {
+        const int slot = runs_closed % kFusedRuns;
+        if (lane == 0) {
+          // the slot's previous run must have left the publisher (a run lasts microseconds, the
+          // publisher needs a fraction of that: this never waits in practice)
+          unsigned long long t0 = 0;
+          for (uint32_t spin = 1; runs_closed - *(volatile int*)&fused.s.published >= kFusedRuns; ++spin) {
+            if ((spin & 0xffu) == 0) {
+              const unsigned long long now = global_ns();
+              if (t0 == 0) t0 = now;
+              if (*abort_flag || now - t0 > a.wait_ns) {
+                *abort_flag = 1;
+                flag_status(a.status, CURDKV_DEV_TIMEOUT);
+                break;
+              }
+            }
+          }
+          if (quarter == 0) {
+            fused.s.run_head[slot] = run_head;
+            fused.s.run_tiles[slot] = run_len;
+            fused.s.run_total[slot] = (run_rows + kTileRows - 1) / kTileRows;
+          }
+        }
+        __syncwarp();                                      // every lane's stores before lane 0's arrival
+        if (lane == 0 && !*abort_flag) mbar_arrive(smem_u32(&fused.s.run_bar[slot]));
+        ++runs_closed;
+        run_len = 0;
+      }
+    };
+    for (TileWalk w(first, stride, (uint32_t)a.chunk_tiles, total_tiles); ok && w.valid(); w.next()) {
       int p, row0;
-      const int n = locate(t, p, row0);
+      const int n = locate(w.tile(), p, row0);
+      if (FUSED && run_len > 0 && (p != run_head || w.starts_chunk())) close_run();
       const int j = row0 + quarter * 32 + lane;
       float s = 0.f;
       {
@@ -555,42 +607,84 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
       if (lane == 0)
         a.tile_sums[((size_t)p * a.tiles_per_head + row0 / kTileRows) * kPartsPerTile + quarter] = s;
-      if constexpr (FUSED) {
-        // Count the tile once all four quarters are out; the warp that completes a head's last
-        // tile hands the head to the selection warps of this CTA.  The epilogue warps are never
-        // more than two tiles apart (the accumulator stages see to that): four counters do.
-        __threadfence();                                   // scores and partial sum before the count
-        __syncwarp();
-        if (lane == 0) {
-          int* parts_done = &fused.s.tile_parts[(tile_it - 1) & 3];
-          if (atomicAdd(parts_done, 1) == 3) {
-            *parts_done = 0;
-            __threadfence();
-            const int tiles_of_head = (n + kTileRows - 1) / kTileRows;
-            if (atomicAdd(a.head_done + p, 1) + 1 == tiles_of_head) {
-              __threadfence();
-              fused_push(fused.s, p, a, abort_flag);
-            }
-          }
-        }
-      }
+      run_head = p;
+      run_rows = n;
+      ++run_len;
     }
     if constexpr (FUSED) {
-      __threadfence_block();
-      if (lane == 0) atomicAdd(&fused.s.producers_done, 1);
+      if (ok && run_len > 0) close_run();
+      if (lane == 0) {
+        fused.s.final_runs[quarter] = runs_closed;
+        __threadfence_block();
+        atomicAdd(&fused.s.producers_done, 1);
+      }
+    }
+  } else if (FUSED && warp == kThreads / 32) {
+    // ------------------------------------------------------------ publisher
+    // Takes the runs the epilogue warps have finished, in order, up to 32 at a time (a lane each):
+    // one device-wide fence for the batch, then every lane adds its run's tiles to the head's
+    // counter; the lane that completes a head hands it to the selection warps.
+    if constexpr (FUSED) {
+      uint32_t first_run = 0;
+      unsigned long long t0 = 0;
+      for (uint32_t spin = 1;; ++spin) {
+        const uint32_t run = first_run + lane;
+        const int slot = (int)(run % kFusedRuns);
+        const bool done = mbar_try_wait(smem_u32(&fused.s.run_bar[slot]), (run / kFusedRuns) & 1u);
+        const uint32_t ready = __ballot_sync(0xffffffffu, done);
+        const int m = ready == 0xffffffffu ? 32 : __ffs(~ready) - 1;   // runs finish in order: a prefix
+        if (m == 0) {
+          int stop = 0;
+          if (lane == 0) {
+            if (*(volatile int*)&fused.s.producers_done == 4) {
+              int total = fused.s.final_runs[0];
+              for (int q = 1; q < 4; ++q) total = min(total, *(volatile int*)&fused.s.final_runs[q]);
+              stop = (int)first_run >= total;
+            }
+            if ((spin & 0x3ffu) == 0) {
+              const unsigned long long now = global_ns();
+              if (t0 == 0) t0 = now;
+              if (*abort_flag || now - t0 > 32ull * a.wait_ns) stop = 1;
+            }
+          }
+          if (__shfl_sync(0xffffffffu, stop, 0)) break;
+          __nanosleep(100);
+          continue;
+        }
+        t0 = 0;
+        __threadfence();                                   // the runs' scores (acquired through the barriers) first
+        if (lane < m) {
+          const int p = fused.s.run_head[slot], tiles = fused.s.run_tiles[slot];
+          if (atomicAdd(a.head_done + p, tiles) + tiles == fused.s.run_total[slot]) {
+            __threadfence();
+            fused_push(a, p);
+          }
+        }
+        __syncwarp();
+        first_run += (uint32_t)m;
+        if (lane == 0) *(volatile int*)&fused.s.published = (int)first_run;
+      }
     }
   } else if constexpr (FUSED) {
     // ------------------------------------------------------------ selection (Alg. 1 lines 6-9)
-    using G = WarpRange<kThreads, kFusedSelThreads, 1>;
+    using G = WarpRange<kFusedSelFirst, kFusedSelThreads, 1>;
     const KeyList list{reinterpret_cast<uint2*>(base_ptr + L::kList), &fused.s.sel.list_count[0],
                        (uint32_t)kFusedListCap};
-    // heads without rows never complete a tile: they are dealt out by CTA
+    // heads without rows never complete a tile: they are dealt out by CTA; the others are counted
+    int mine = 0;
     if (a.seqlens != nullptr) {
       for (int p = (int)blockIdx.x; p < a.batch * a.heads; p += (int)gridDim.x)
         if (seq_len_of(a.seqlens, p / a.heads, a.n_max) == 0) fused_select_head<G>(a, p, list, fused.s.sel);
+      for (int b = G::tid(); b < a.batch; b += kFusedSelThreads)
+        mine += seq_len_of(a.seqlens, b, a.n_max) > 0 ? a.heads : 0;
+    } else if (G::tid() == 0) {
+      mine = a.batch * a.heads;
     }
+    if (mine != 0) atomicAdd(&fused.s.nonempty, mine);
+    G::sync();
+    const int nonempty_heads = fused.s.nonempty;
     for (;;) {
-      if (G::tid() == 0) fused.s.current = fused_pop(fused.s, a);
+      if (G::tid() == 0) fused.s.current = fused_pop(a, nonempty_heads, abort_flag);
       G::sync();
       const int p = fused.s.current;
       G::sync();

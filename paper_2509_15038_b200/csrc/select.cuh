@@ -88,6 +88,7 @@ struct KeyList {
 // (four histogram bins per thread), 512 (eight; short rows run as two such CTAs per SM, which hides
 // more of the latency of their many short phases) or 256 (sixteen).
 struct WholeCta {
+  static constexpr int kUnroll = 4;                        // quads in flight per thread
   static __device__ __forceinline__ int tid() { return (int)threadIdx.x; }
   static __device__ __forceinline__ int size() { return (int)blockDim.x; }
   static __device__ __forceinline__ void sync() { __syncthreads(); }
@@ -96,6 +97,7 @@ struct WholeCta {
 template <int FIRST, int N, int BAR>
 struct WarpRange {
   static_assert(N % 32 == 0 && FIRST % 32 == 0 && BAR >= 1 && BAR <= 15, "whole warps, a free barrier");
+  static constexpr int kUnroll = 4;                        // (eight spill under this kernel's register cap)
   static __device__ __forceinline__ int tid() { return (int)threadIdx.x - FIRST; }
   static __device__ __forceinline__ int size() { return N; }
   static __device__ __forceinline__ void sync() { asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(N) : "memory"); }
@@ -242,7 +244,6 @@ struct DigitRun {
 };
 
 constexpr int kSelRankDirect = 192;                        // lists up to this size are ranked without histograms
-constexpr int kSelUnroll = 4;                              // quads in flight per thread
 
 // Adds the keys <= ceiling whose bits under `mask` equal `prefix` to the
 // histogram of this pass's digit.  Whole CTA.
@@ -253,13 +254,13 @@ __device__ __forceinline__ void digit_histogram(const RowKeys& keys, uint32_t ce
   const int shift = pass_shift(pass);
   const uint32_t dmask = pass_digit_mask(pass);
   DigitRun run;
-  for (int q0 = (int)G::tid(); q0 < quads; q0 += kSelUnroll * step) {
-    uint4 v[kSelUnroll];
+  for (int q0 = (int)G::tid(); q0 < quads; q0 += G::kUnroll * step) {
+    uint4 v[G::kUnroll];
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u)
+    for (int u = 0; u < G::kUnroll; ++u)
       if (q0 + u * step < quads) v[u] = keys.load4(q0 + u * step);
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u) {
+    for (int u = 0; u < G::kUnroll; ++u) {
       if (q0 + u * step < quads) {
         const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
@@ -283,13 +284,13 @@ template <class G>
 __device__ __forceinline__ void stage_keys(const RowKeys& src, uint4* staged, uint32_t* hist) {
   const int quads = src.quads(), step = (int)G::size();
   DigitRun run;
-  for (int q0 = (int)G::tid(); q0 < quads; q0 += kSelUnroll * step) {
-    uint4 v[kSelUnroll];
+  for (int q0 = (int)G::tid(); q0 < quads; q0 += G::kUnroll * step) {
+    uint4 v[G::kUnroll];
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u)
+    for (int u = 0; u < G::kUnroll; ++u)
       if (q0 + u * step < quads) v[u] = src.load4(q0 + u * step);
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u) {
+    for (int u = 0; u < G::kUnroll; ++u) {
       if (q0 + u * step < quads) {
         staged[q0 + u * step] = v[u];
         run.add(v[u].x >> 20, hist);
@@ -328,13 +329,13 @@ __device__ __forceinline__ void count_sweep(const RowKeys& keys, const Cut& cut,
   const Segments seg(keys.quads(), G::size() >> 5);
   const int q_end = seg.end(warp);
   uint32_t def_cnt = 0, eq_cnt = 0;
-  for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += kSelUnroll * 32) {
-    uint4 v[kSelUnroll];
+  for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += G::kUnroll * 32) {
+    uint4 v[G::kUnroll];
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u)
+    for (int u = 0; u < G::kUnroll; ++u)
       if (q0 + u * 32 < q_end) v[u] = keys.load4(q0 + u * 32);
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u) {
+    for (int u = 0; u < G::kUnroll; ++u) {
       if (q0 + u * 32 < q_end) {
         const uint32_t f = classify(v[u], cut.T);
         def_cnt += __popc(f & 15u);
@@ -362,13 +363,13 @@ __device__ __forceinline__ void collect_sweep(const RowKeys& keys, uint32_t d_cu
   const Segments seg(keys.quads(), G::size() >> 5);
   const int q_end = seg.end(warp);
   uint32_t def_cnt = 0;
-  for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += kSelUnroll * 32) {
-    uint4 v[kSelUnroll];
+  for (int q0 = seg.begin(warp) + lane; q0 < q_end; q0 += G::kUnroll * 32) {
+    uint4 v[G::kUnroll];
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u)
+    for (int u = 0; u < G::kUnroll; ++u)
       if (q0 + u * 32 < q_end) v[u] = keys.load4(q0 + u * 32);
 #pragma unroll
-    for (int u = 0; u < kSelUnroll; ++u) {
+    for (int u = 0; u < G::kUnroll; ++u) {
       if (q0 + u * 32 < q_end) {
         const uint32_t k4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
@@ -539,13 +540,13 @@ __device__ __forceinline__ void scale_row_and_histogram(float* row, const RowKey
   int done = 0;
   if (keys.vec) {
     const int quads = n >> 2;                              // whole quads of valid tokens
-    for (int q0 = G::tid(); q0 < quads; q0 += kSelUnroll * step) {
-      float4 f[kSelUnroll];
+    for (int q0 = G::tid(); q0 < quads; q0 += G::kUnroll * step) {
+      float4 f[G::kUnroll];
 #pragma unroll
-      for (int u = 0; u < kSelUnroll; ++u)
+      for (int u = 0; u < G::kUnroll; ++u)
         if (q0 + u * step < quads) f[u] = __ldcg(reinterpret_cast<const float4*>(row) + q0 + u * step);
 #pragma unroll
-      for (int u = 0; u < kSelUnroll; ++u) {
+      for (int u = 0; u < G::kUnroll; ++u) {
         const int q = q0 + u * step;
         if (q < quads) {
           const float4 o = make_float4(scaled(f[u].x), scaled(f[u].y), scaled(f[u].z), scaled(f[u].w));

@@ -1,5 +1,8 @@
 """curdkv_compress (one call; for the main shapes one kernel that scores, normalises and selects)
-against the three separate calls, bit for bit, and through them against the oracle.  Needs a B200."""
+against the three separate calls, bit for bit, and through them against the oracle.  Needs a B200.
+
+The single-kernel route is taken from four heads per SM upwards (592 heads on a B200): the cases
+below that are meant to reach it use 600 heads or more, the others cover the three-step route."""
 import numpy as np
 import pytest
 import torch
@@ -61,7 +64,8 @@ def _both_ways(K, V, G, budget, s, w, seqlens=None, head_budgets=None, adaptive=
 
 
 def test_compress_cfg1_and_cfg2_match_three_calls_and_oracle():
-    for w in (synth.CONFIGS["cfg1"], synth.shrink(synth.CONFIGS["cfg2"], layers=2)):
+    for w in (synth.CONFIGS["cfg1"], synth.shrink(synth.CONFIGS["cfg2"], layers=2),
+              synth.shrink(synth.CONFIGS["cfg2"], layers=76, n_max=1024, budget=204 + 64)):
         K, V, _ = synth.make_kv(w, DEV)
         G = synth.make_G(w.d, w.r, seed=0)
         _, out = _both_ways(K, V, G, w.budget, w.num_sink, w.window, q_heads=w.q_heads, what=w.name)
@@ -79,17 +83,18 @@ def test_compress_cfg1_and_cfg2_match_three_calls_and_oracle():
 
 
 def test_compress_ragged_lengths_zero_rows_and_odd_sizes():
-    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=5, n_max=1000)
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=80, n_max=1000)
     K, V, _ = synth.make_kv(w, DEV)
     G = synth.make_G(w.d, 32, seed=0)
-    lens = np.array([1000, 777, 128, 0, 1], dtype=np.int32)
+    lens = np.tile(np.array([1000, 777, 128, 0, 1], dtype=np.int32), 16)
     for s, win, k in ((4, 0, 100), (4, 16, 100), (0, 32, 300), (4, 8, 10), (4, 8, 2000), (0, 0, 1)):
         _both_ways(K, V, G, k, s, win, seqlens=lens, what=f"ragged s={s} w={win} k={k}")
     # n_max = 1001: score rows of odd heads are not 16-byte aligned, the last tile holds one row
-    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=2, n_max=1001, kv_heads=3, q_heads=3)
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, batch=200, n_max=1001, kv_heads=3, q_heads=3)
     K, V, _ = synth.make_kv(w, DEV)
     _both_ways(K, V, G, 150, 4, 16, what="n_max=1001")
-    _both_ways(K, V, G, 150, 0, 8, seqlens=np.array([1001, 897], dtype=np.int32), what="n_max=1001 ragged")
+    _both_ways(K, V, G, 150, 0, 8, seqlens=np.tile(np.array([1001, 897], dtype=np.int32), 100),
+               what="n_max=1001 ragged")
 
 
 def test_compress_many_short_heads_and_long_rows():
@@ -102,13 +107,13 @@ def test_compress_many_short_heads_and_long_rows():
     _both_ways(K, V, G, 40, 2, 8, what="768 heads of 2 tiles")
     lens = np.random.default_rng(1).integers(0, 257, size=96).astype(np.int32)
     _both_ways(K, V, G, 40, 2, 8, seqlens=lens, what="768 ragged heads")
-    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, n_max=40000, kv_heads=2, q_heads=2)
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=76, n_max=40000)
     K, V, _ = synth.make_kv(w, DEV)
     _both_ways(K, V, G, 4000, 4, 64, what="n=40000")
 
 
 def test_compress_options_and_layouts():
-    w = synth.shrink(synth.CONFIGS["cfg2"], layers=2, n_max=1536, kv_heads=3, q_heads=3)
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=200, n_max=1536, kv_heads=3, q_heads=3)
     K, V, _ = synth.make_kv(w, DEV)
     for r in (1, 20, 32):
         _both_ways(K, V, synth.make_G(w.d, r, seed=r), 200, 4, 32, what=f"r={r}")
@@ -116,14 +121,14 @@ def test_compress_options_and_layouts():
     _both_ways(K, V, G, 200, 4, 32, score_mode=1, what="key only")
     _both_ways(K, V, G, 200, 4, 32, score_mode=2, what="value only")
     _both_ways(K, V, G, 200, 4, 32, raw_scores=1, what="raw scores")
-    _both_ways(K, V, G, 300, 0, 9, head_budgets=np.array([[300, 0, 13], [5000, 77, 1]], dtype=np.int32),
-               what="per-head budgets")
+    _both_ways(K, V, G, 300, 0, 9, what="per-head budgets",
+               head_budgets=np.tile(np.array([[300, 0, 13], [5000, 77, 1]], dtype=np.int32), (100, 1)))
     _both_ways(K, V, G, 0, 0, 0, what="budget 0")
     _both_ways(torch.zeros_like(K), V, G, 100, 2, 4, what="all-zero keys")       # head sums of 0
     # token-major storage viewed as [B, H, n, d]
     g = torch.Generator(device=DEV).manual_seed(7)
-    Kb = torch.randn((2, 640, 4, 128), generator=g, device=DEV).to(torch.bfloat16)
-    Vb = torch.randn((2, 640, 4, 128), generator=g, device=DEV).to(torch.bfloat16)
+    Kb = torch.randn((150, 640, 4, 128), generator=g, device=DEV).to(torch.bfloat16)
+    Vb = torch.randn((150, 640, 4, 128), generator=g, device=DEV).to(torch.bfloat16)
     _both_ways(Kb.permute(0, 2, 1, 3), Vb.permute(0, 2, 1, 3), G, 64, 0, 8, what="strided")
 
 
