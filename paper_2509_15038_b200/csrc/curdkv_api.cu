@@ -56,10 +56,9 @@ inline int tiles_per_head(const curdkv_desc* d) { return (d->n_max + kTileRows -
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
 // What curdkv_compress keeps next to the status words: per head a tile counter and an entry of
-// the list of finished heads, and two queue counters per launch.
-constexpr int kMaxFusedLaunches = 32;
+// the list of finished heads, and two queue counters.
 inline size_t head_counter_bytes(const curdkv_desc* d) {
-  return round256((size_t)d->batch * d->kv_heads * 2 * sizeof(int32_t)) + round256(kMaxFusedLaunches * 2 * sizeof(int32_t));
+  return round256((size_t)d->batch * d->kv_heads * 2 * sizeof(int32_t)) + 256;
 }
 
 // ---- TMA descriptors for the tensor-core sketch kernel ---------------------
@@ -117,7 +116,7 @@ cudaError_t launch_umma(const CUtensorMap& mk, const CUtensorMap& mv, const umma
   const int smem = L::dynamic_bytes(a.seqlens != nullptr ? a.batch : 0);
   cudaError_t e = cudaFuncSetAttribute(umma::sketch_umma_kernel<R, FUSED>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       L::dynamic_bytes(FUSED ? umma::kMaxRaggedBatchFused : umma::kMaxRaggedBatch));
+                                       L::dynamic_bytes(FUSED ? 0 : umma::kMaxRaggedBatch));
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
@@ -234,9 +233,16 @@ size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32
   return score + (max_budget > 0 ? head_counter_bytes(desc) : 0);
 }
 
-curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
-                           const curdkv_desc* desc, float* scores, float* head_sums,
-                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// curdkv_score; with normalise = false the scores stay as the score kernels leave them
+// (unnormalised, one or four partial sums per tile in the workspace: *parts_per_tile) for a
+// selection kernel that finishes Alg. 1 line 6 itself.
+curdkv_status score_impl(const void* K, const void* V, const float* G, int32_t g_per_head,
+                         const curdkv_desc* desc, float* scores, float* head_sums, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream, bool normalise, int* parts_per_tile) {
   curdkv_status st = check_desc(desc);
   if (st != CURDKV_OK) return st;
   if ((st = check_kv(K, V, desc)) != CURDKV_OK) return st;
@@ -437,6 +443,8 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
     if (!launch_ok()) return CURDKV_ERR_CUDA;
   }
 
+  if (parts_per_tile != nullptr) *parts_per_tile = parts;
+  if (!normalise) return CURDKV_OK;
   const int chunks = (desc->n_max + kNormChunk - 1) / kNormChunk;
   normalise_kernel<<<(unsigned)(P * chunks), 256, 0, stream>>>(scores, a.tile_sums, head_sums,
                                                               desc->seqlens, desc->kv_heads,
@@ -446,13 +454,11 @@ curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t
   return CURDKV_OK;
 }
 
-curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_t budget,
-                            const int32_t* head_budgets, int32_t num_sink, int32_t window,
-                            int32_t adaptive, double alpha, int32_t* idx, int32_t* head_counts,
-                            int32_t* head_offsets, void* workspace, size_t workspace_bytes,
-                            void* cuda_stream) {
-  (void)workspace;
-  (void)workspace_bytes;
+// curdkv_select; with norm.tile_sums the selection kernel normalises `scores` first
+curdkv_status select_impl(float* scores, const curdkv_desc* desc, int32_t budget,
+                          const int32_t* head_budgets, int32_t num_sink, int32_t window,
+                          int32_t adaptive, double alpha, int32_t* idx, int32_t* head_counts,
+                          int32_t* head_offsets, void* cuda_stream, const Normaliser& norm) {
   curdkv_status st = check_desc(desc);
   if (st != CURDKV_OK) return st;
   if (scores == nullptr || idx == nullptr || head_counts == nullptr) return CURDKV_ERR_INVALID_ARG;
@@ -494,7 +500,7 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
       cfg.numAttrs = 1;
       return cudaLaunchKernelEx(&cfg, kernel, scores, desc->seqlens, (int)desc->kv_heads, (int)desc->n_max,
                                 (int)budget, (int)num_sink, (int)window, min_protected, idx, head_counts,
-                                head_offsets);
+                                head_offsets, norm);
     };
     const cudaError_t e = small_ctas ? launch(select_adaptive_kernel<512>, 512)
                                      : launch(select_adaptive_kernel<1024>, 1024);
@@ -515,9 +521,32 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
   else if (desc->n_max <= 16384) { sel_threads = 512; list_cap = kSelListCap / 2; }
   select_fixed_kernel<<<(unsigned)P, sel_threads, stage_bytes + (size_t)list_cap * 8, stream>>>(
       scores, desc->seqlens, desc->kv_heads, desc->n_max, budget, head_budgets, num_sink, window,
-      (int)(stage_bytes / sizeof(uint4)), list_cap, idx, head_counts, head_offsets);
+      (int)(stage_bytes / sizeof(uint4)), list_cap, idx, head_counts, head_offsets, norm);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+curdkv_status curdkv_score(const void* K, const void* V, const float* G, int32_t g_per_head,
+                           const curdkv_desc* desc, float* scores, float* head_sums,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return score_impl(K, V, G, g_per_head, desc, scores, head_sums, workspace, workspace_bytes, cuda_stream,
+                    true, nullptr);
+}
+
+curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_t budget,
+                            const int32_t* head_budgets, int32_t num_sink, int32_t window,
+                            int32_t adaptive, double alpha, int32_t* idx, int32_t* head_counts,
+                            int32_t* head_offsets, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  // the kernels only write the scores when they are asked to normalise them
+  return select_impl(const_cast<float*>(scores), desc, budget, head_budgets, num_sink, window, adaptive,
+                     alpha, idx, head_counts, head_offsets, cuda_stream, Normaliser{nullptr, nullptr, 0, 0, 0});
 }
 
 curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* desc,
@@ -592,18 +621,25 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
   // one another.
   // (With fewer than four heads per SM the selection of the last heads, which only starts when the
   // stream ends and runs on a quarter of a selection CTA's threads, costs more than it saves.)
+  // Ragged batches keep the three-step route as well: their many short heads make the
+  // selection warps busy enough to slow the stream by more than the hidden selection saves.
   const bool fused = !adaptive && budget > 0 && desc->use_projection && !g_per_head && !desc->whiten &&
-                     P >= 4 * (int64_t)sm_count() &&
+                     P >= 4 * (int64_t)sm_count() && desc->seqlens == nullptr &&
                      desc->d == 128 && desc->r >= 1 && desc->r <= 32 && desc->n_max >= kTileRows &&
                      G != nullptr && P > 0 && P * tiles <= 0x7fffffffLL &&
-                     P * (int64_t)budget <= 0x7fffffffLL &&
-                     (desc->seqlens == nullptr ||
-                      desc->batch <= (int64_t)kMaxFusedLaunches * umma::kMaxRaggedBatchFused);
+                     P * (int64_t)budget <= 0x7fffffffLL;
   if (!fused) {
-    st = curdkv_score(K, V, G, g_per_head, desc, scores, head_sums, workspace, score_bytes, cuda_stream);
-    if (st == CURDKV_OK)
-      st = curdkv_select(scores, desc, budget, head_budgets, num_sink, window, adaptive, alpha, idx,
-                         head_counts, head_offsets, workspace, score_bytes, cuda_stream);
+    // the selection kernel forms the head sums and divides on its first sweep over the scores:
+    // no separate normalisation pass
+    int parts = 1;
+    st = score_impl(K, V, G, g_per_head, desc, scores, head_sums, workspace, score_bytes, cuda_stream, false,
+                    &parts);
+    if (st == CURDKV_OK && P > 0) {
+      const Normaliser norm{reinterpret_cast<const float*>(static_cast<unsigned char*>(workspace) + kStatusBytes),
+                            head_sums, tiles, parts, desc->raw_scores};
+      st = select_impl(scores, desc, budget, head_budgets, num_sink, window, adaptive, alpha, idx, head_counts,
+                       head_offsets, cuda_stream, tiles > 0 ? norm : Normaliser{nullptr, nullptr, 0, 0, 0});
+    }
   } else {
     // workspace: status words, one tile counter per head (zero on entry), tile partial sums
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -613,51 +649,43 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
     int32_t* done_list = head_done + P;
     int32_t* queue_ctr = reinterpret_cast<int32_t*>(ws + kStatusBytes + round256((size_t)P * 2 * sizeof(int32_t)));
     float* tile_sums = reinterpret_cast<float*>(ws + kStatusBytes + counters);
-    const int slice = desc->seqlens != nullptr ? umma::kMaxRaggedBatchFused : desc->batch;
-    for (int b0 = 0; b0 < desc->batch; b0 += slice) {
-      curdkv_desc part = *desc;
-      part.batch = desc->batch - b0 < slice ? desc->batch - b0 : slice;
-      const __nv_bfloat16* Kb = static_cast<const __nv_bfloat16*>(K) + (int64_t)b0 * desc->k_stride_b;
-      const __nv_bfloat16* Vb = static_cast<const __nv_bfloat16*>(V) + (int64_t)b0 * desc->v_stride_b;
-      CUtensorMap mk, mv;
-      if (!make_tile_map(&mk, Kb, &part, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) ||
-          !make_tile_map(&mv, Vb, &part, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n))
-        return CURDKV_ERR_CUDA;
-      const size_t p0 = (size_t)b0 * desc->kv_heads;
-      umma::Args u;
-      u.G = G;
-      u.seqlens = desc->seqlens != nullptr ? desc->seqlens + b0 : nullptr;
-      u.batch = part.batch;
-      u.heads = desc->kv_heads;
-      u.n_max = desc->n_max;
-      u.r = desc->r;
-      u.tiles_per_head = tiles;
-      u.score_mode = desc->score_mode;
-      u.scores = scores + p0 * desc->n_max;
-      u.tile_sums = tile_sums + p0 * tiles * umma::kPartsPerTile;
-      u.status = static_cast<uint32_t*>(workspace);
-      u.head_sums = head_sums + p0;
-      u.head_done = head_done + p0;
-      u.done_list = done_list + p0;
-      u.queue_ctr = queue_ctr + 2 * (b0 / slice);
-      u.head_budgets = head_budgets != nullptr ? head_budgets + p0 : nullptr;
-      u.idx = idx + p0 * budget;
-      u.counts = head_counts + p0;
-      u.offsets = head_offsets != nullptr ? head_offsets + p0 : nullptr;
-      u.budget = budget;
-      u.num_sink = num_sink;
-      u.window = window;
-      u.raw = desc->raw_scores;
-      u.first_head = (int)p0;
-      u.all_heads = (int)P;
-      // chunks of consecutive tiles per CTA visit: long enough to make the per-chunk bookkeeping
-      // rare, short enough that the last, uneven round of chunks stays near 1 % of the launch
-      const int sms = sm_count();
-      const int64_t per_cta = (int64_t)part.batch * desc->kv_heads * tiles / (sms > 0 ? sms : 1);
-      u.chunk_tiles = (int)(per_cta / 64 < 1 ? 1 : (per_cta / 64 > 16 ? 16 : per_cta / 64));
-      if (launch_umma<32, true>(mk, mv, u, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
-      if (!launch_ok()) return CURDKV_ERR_CUDA;
-    }
+    CUtensorMap mk, mv;
+    if (!make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) ||
+        !make_tile_map(&mv, V, desc, desc->v_stride_b, desc->v_stride_h, desc->v_stride_n))
+      return CURDKV_ERR_CUDA;
+    umma::Args u;
+    u.G = G;
+    u.seqlens = nullptr;
+    u.batch = desc->batch;
+    u.heads = desc->kv_heads;
+    u.n_max = desc->n_max;
+    u.r = desc->r;
+    u.tiles_per_head = tiles;
+    u.score_mode = desc->score_mode;
+    u.scores = scores;
+    u.tile_sums = tile_sums;
+    u.status = static_cast<uint32_t*>(workspace);
+    u.head_sums = head_sums;
+    u.head_done = head_done;
+    u.done_list = done_list;
+    u.queue_ctr = queue_ctr;
+    u.head_budgets = head_budgets;
+    u.idx = idx;
+    u.counts = head_counts;
+    u.offsets = head_offsets;
+    u.budget = budget;
+    u.num_sink = num_sink;
+    u.window = window;
+    u.raw = desc->raw_scores;
+    u.first_head = 0;
+    u.all_heads = (int)P;
+    // chunks of consecutive tiles per CTA visit: long enough to make the per-chunk bookkeeping
+    // rare, short enough that the last, uneven round of chunks stays near 1 % of the launch
+    const int sms = sm_count();
+    const int64_t per_cta = P * tiles / (sms > 0 ? sms : 1);
+    u.chunk_tiles = (int)(per_cta / 64 < 1 ? 1 : (per_cta / 64 > 16 ? 16 : per_cta / 64));
+    if (launch_umma<32, true>(mk, mv, u, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+    if (!launch_ok()) return CURDKV_ERR_CUDA;
     g_profile_start = g_profile_stop = nullptr;
   }
   if (st != CURDKV_OK) return st;

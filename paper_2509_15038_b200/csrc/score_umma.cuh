@@ -92,7 +92,6 @@ struct TileWalk {
 // memory and maps a running tile number to (sequence, head, tile) by binary
 // search, so all CTAs get the same number of real tiles.
 constexpr int kMaxRaggedBatch = 8192;                      // sequences per launch with seqlens
-constexpr int kMaxRaggedBatchFused = 4096;                 // ... when the candidate list shares the space
 
 template <int R, bool FUSED = false>
 struct Smem {                                     // offsets from the 1024-aligned base
@@ -266,7 +265,6 @@ struct FusedSmem {
   int published;               // runs the publisher is done with
   int final_runs[4];           // runs each epilogue warp closed before it left its loop
   int producers_done;          // epilogue warps that have left their loop
-  int nonempty;                // heads of this launch that have rows (each of them gets finished once)
   int current;                 // head the selection warps work on
 };
 
@@ -313,22 +311,13 @@ __device__ __forceinline__ int fused_pop(const Args& a, int nonempty_heads, vola
 // histogram, then the fixed-budget selection of select_fixed_kernel on the normalised scores.
 template <class G>
 __device__ __forceinline__ void fused_select_head(const Args& a, int p, const KeyList& list, SelectSmem& sm) {
-  static_assert(kFusedSelThreads == 256, "the head sum follows normalise_kernel's 256-thread order");
-  const int tid = G::tid(), lane = tid & 31, warp = tid >> 5;
+  const int tid = G::tid();
   const int n = seq_len_of(a.seqlens, p / a.heads, a.n_max);
   const int tiles = (n + kTileRows - 1) / kTileRows;
   float* row = a.scores + (size_t)p * a.n_max;
-  const float* mine = a.tile_sums + (size_t)p * a.tiles_per_head * kPartsPerTile;
-  float part = 0.f;                                        // fixed order: thread, warp tree, warp order
-  for (int i = tid; i < tiles * kPartsPerTile; i += kFusedSelThreads) part += __ldcg(mine + i);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-  if (lane == 0) sm.warp_def[warp] = __float_as_uint(part);
   clear_hist<G>(sm.hist);
-  G::sync();
-  float S = 0.f;
-#pragma unroll
-  for (int w = 0; w < kFusedSelThreads / 32; ++w) S += __uint_as_float(sm.warp_def[w]);
+  const float S = head_sum_fixed_order<G>(a.tile_sums + (size_t)p * a.tiles_per_head * kPartsPerTile,
+                                          tiles * kPartsPerTile, sm);
   if (tid == 0) a.head_sums[p] = S;
 
   int k = a.budget;
@@ -337,7 +326,7 @@ __device__ __forceinline__ void fused_select_head(const Args& a, int p, const Ke
   const ForcedSet F = forced_set(n, k_eff, a.num_sink, a.window);
   RowKeys keys = global_keys(row, n, F);
   keys.written_here = true;
-  scale_row_and_histogram<G>(row, keys, a.n_max, tiles * kTileRows, S, a.raw != 0, sm.hist);
+  scale_row_and_histogram<G>(row, keys, a.n_max, tiles * kTileRows, S, a.raw != 0, sm.hist, nullptr);
   G::sync();
   select_fixed_row<G>(keys, F, k_eff, a.budget, nullptr, 0, list, true, a.idx + (size_t)p * a.budget, sm);
   if (tid == 0) {
@@ -389,7 +378,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
   }
   if constexpr (FUSED) {
     if (tid < kFusedRuns) mbar_init(smem_u32(&fused.s.run_bar[tid]), 4);
-    if (tid == 0) fused.s.producers_done = fused.s.published = fused.s.nonempty = 0;
+    if (tid == 0) fused.s.producers_done = fused.s.published = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -670,19 +659,9 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     using G = WarpRange<kFusedSelFirst, kFusedSelThreads, 1>;
     const KeyList list{reinterpret_cast<uint2*>(base_ptr + L::kList), &fused.s.sel.list_count[0],
                        (uint32_t)kFusedListCap};
-    // heads without rows never complete a tile: they are dealt out by CTA; the others are counted
-    int mine = 0;
-    if (a.seqlens != nullptr) {
-      for (int p = (int)blockIdx.x; p < a.batch * a.heads; p += (int)gridDim.x)
-        if (seq_len_of(a.seqlens, p / a.heads, a.n_max) == 0) fused_select_head<G>(a, p, list, fused.s.sel);
-      for (int b = G::tid(); b < a.batch; b += kFusedSelThreads)
-        mine += seq_len_of(a.seqlens, b, a.n_max) > 0 ? a.heads : 0;
-    } else if (G::tid() == 0) {
-      mine = a.batch * a.heads;
-    }
-    if (mine != 0) atomicAdd(&fused.s.nonempty, mine);
-    G::sync();
-    const int nonempty_heads = fused.s.nonempty;
+    // (the fused form is launched for batches without per-sequence lengths only: every head has
+    // rows and gets finished exactly once)
+    const int nonempty_heads = a.batch * a.heads;
     for (;;) {
       if (G::tid() == 0) fused.s.current = fused_pop(a, nonempty_heads, abort_flag);
       G::sync();

@@ -525,19 +525,39 @@ __device__ __forceinline__ void write_sweep(const RowKeys& keys, const Cut& cut,
   G::sync();                                         // sm.warp_* may be reused
 }
 
+// The head normaliser S = sum_j lK_j lV_j from the per-tile partial sums, in the one order every
+// kernel of this library uses (256 threads: thread t adds partials t, t + 256, ...; a shuffle tree
+// per warp; the eight warp sums in warp order), so that S is the same bit pattern wherever it is
+// formed.  Group G of at least 256 threads; the partials may have been written by this launch.
+template <class G>
+__device__ __forceinline__ float head_sum_fixed_order(const float* partials, int count, SelectSmem& sm) {
+  const int tid = G::tid(), lane = tid & 31, warp = tid >> 5;
+  float part = 0.f;
+  if (tid < 256)
+    for (int i = tid; i < count; i += 256) part += __ldcg(partials + i);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+  if (lane == 0 && warp < 8) sm.warp_def[warp] = __float_as_uint(part);
+  G::sync();
+  float S = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) S += __uint_as_float(sm.warp_def[w]);
+  return S;
+}
+
 // Alg. 1 line 6 for one row, on the way to the selection: row[j] <- row[j] / S for j < n (0 when the
 // sum is not positive; left as it is with `raw`), row[j] <- 0 for first_unwritten <= j < n_max, and
-// the leading-digit histogram of the resulting rank keys in `hist` (zero on entry).  The row was
-// written by other CTAs of this kernel: it is read from L2.  Group G.
+// the leading-digit histogram of the resulting rank keys in `hist` (zero on entry).  With `staged`
+// (16-byte aligned rows only) the rank keys are also left there, a quad per four tokens.  The row
+// may have been written by other CTAs of this launch: it is read from L2.  Group G.
 template <class G>
 __device__ __forceinline__ void scale_row_and_histogram(float* row, const RowKeys& keys, int n_max,
                                                         int first_unwritten, float S, bool raw,
-                                                        uint32_t* hist) {
+                                                        uint32_t* hist, uint4* staged) {
   const int n = keys.n, step = G::size();
   const bool live = S > 0.f;
   auto scaled = [&](float x) { return raw ? x : (live ? __fdiv_rn(x, S) : 0.f); };
   DigitRun run;
-  int done = 0;
   if (keys.vec) {
     const int quads = n >> 2;                              // whole quads of valid tokens
     for (int q0 = G::tid(); q0 < quads; q0 += G::kUnroll * step) {
@@ -551,23 +571,45 @@ __device__ __forceinline__ void scale_row_and_histogram(float* row, const RowKey
         if (q < quads) {
           const float4 o = make_float4(scaled(f[u].x), scaled(f[u].y), scaled(f[u].z), scaled(f[u].w));
           if (!raw) reinterpret_cast<float4*>(row)[q] = o;
-          run.add(keys.key_of(o.x, 4 * q) >> 20, hist);
-          run.add(keys.key_of(o.y, 4 * q + 1) >> 20, hist);
-          run.add(keys.key_of(o.z, 4 * q + 2) >> 20, hist);
-          run.add(keys.key_of(o.w, 4 * q + 3) >> 20, hist);
+          const uint4 k4 = make_uint4(keys.key_of(o.x, 4 * q), keys.key_of(o.y, 4 * q + 1),
+                                      keys.key_of(o.z, 4 * q + 2), keys.key_of(o.w, 4 * q + 3));
+          if (staged != nullptr) staged[q] = k4;
+          run.add(k4.x >> 20, hist);
+          run.add(k4.y >> 20, hist);
+          run.add(k4.z >> 20, hist);
+          run.add(k4.w >> 20, hist);
         }
       }
     }
-    done = quads << 2;
-  }
-  for (int j = done + G::tid(); j < n; j += step) {
-    const float o = scaled(__ldcg(row + j));
-    if (!raw) row[j] = o;
-    run.add(keys.key_of(o, j) >> 20, hist);
+    if (G::tid() == 0 && (n & 3) != 0) {                   // the last, partial quad
+      uint32_t k4[4] = {0u, 0u, 0u, 0u};
+      for (int j = quads << 2; j < n; ++j) {
+        const float o = scaled(__ldcg(row + j));
+        if (!raw) row[j] = o;
+        k4[j & 3] = keys.key_of(o, j);
+        run.add(k4[j & 3] >> 20, hist);
+      }
+      if (staged != nullptr) staged[quads] = make_uint4(k4[0], k4[1], k4[2], k4[3]);
+    }
+  } else {
+    for (int j = G::tid(); j < n; j += step) {
+      const float o = scaled(__ldcg(row + j));
+      if (!raw) row[j] = o;
+      run.add(keys.key_of(o, j) >> 20, hist);
+    }
   }
   run.flush(hist);
   for (int j = first_unwritten + G::tid(); j < n_max; j += step) row[j] = 0.f;
 }
+
+// What a selection kernel needs to finish Alg. 1 line 6 itself (the scores then arrive as the
+// score kernels leave them: unnormalised, with per-tile partial sums).  tile_sums = nullptr: the
+// scores are final already.
+struct Normaliser {
+  const float* tile_sums;  // [heads][tiles_per_head][parts_per_tile]
+  float* head_sums;        // [heads]
+  int tiles_per_head, parts_per_tile, raw;
+};
 
 // ---------------------------------------------------------------------------
 // Fixed per-head budget, one row, by the group G: Alg. 1 lines 7-9 on the scores `keys` describes.
@@ -624,10 +666,13 @@ __device__ __forceinline__ void select_fixed_row(RowKeys keys, const ForcedSet& 
 
 // grid = batch*heads, block = 1024, 512 or 256, dynamic shared memory = 16 * stage_quads bytes
 // (0: rows are read from global memory) followed by one candidate list of list_cap entries.
+// With norm.tile_sums the kernel first finishes Alg. 1 line 6 for its row (head sum, division on the
+// way into the staged keys) and `scores` is written.
 __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
-    const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
+    float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
     int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window, int stage_quads,
-    int list_cap, int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+    int list_cap, int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+    const Normaliser norm) {
   __shared__ SelectSmem sm;
   extern __shared__ uint4 staged_keys[];                   // stage_quads quads, or nothing
   using G = WholeCta;
@@ -637,9 +682,27 @@ __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
   if (head_budgets != nullptr) k = max(0, min(head_budgets[p], budget));
   const int k_eff = min(k, n);
   const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  const RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
+  float* row = scores + (size_t)p * n_max;
+  RowKeys keys = global_keys(row, n, F);
   const KeyList list{reinterpret_cast<uint2*>(staged_keys + stage_quads), &sm.list_count[0], (uint32_t)list_cap};
-  select_fixed_row<G>(keys, F, k_eff, budget, staged_keys, stage_quads, list, false, idx + (size_t)p * budget, sm);
+  bool hist_ready = false;
+  if (norm.tile_sums != nullptr) {
+    const int tiles = (n + kTileRows - 1) / kTileRows;
+    const float S = head_sum_fixed_order<G>(
+        norm.tile_sums + (size_t)p * norm.tiles_per_head * norm.parts_per_tile, tiles * norm.parts_per_tile, sm);
+    if (threadIdx.x == 0) norm.head_sums[p] = S;
+    clear_hist<G>(sm.hist);
+    G::sync();
+    const bool stage = keys.vec && keys.quads() <= stage_quads;
+    scale_row_and_histogram<G>(row, keys, n_max, tiles * kTileRows, S, norm.raw != 0, sm.hist,
+                               stage ? staged_keys : nullptr);
+    keys.written_here = true;
+    if (stage) keys.staged = staged_keys;
+    hist_ready = true;
+    G::sync();
+  }
+  select_fixed_row<G>(keys, F, k_eff, budget, staged_keys, stage_quads, list, hist_ready,
+                      idx + (size_t)p * budget, sm);
   if (threadIdx.x == 0) {
     counts[p] = k_eff;
     if (offsets != nullptr) {                              // heads sit at multiples of `budget` rows
@@ -672,9 +735,9 @@ __host__ __device__ constexpr int adaptive_dynamic_bytes(int threads) { return k
 
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kernel(
-    const float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
+    float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
     int budget, int num_sink, int window, int min_protected, int32_t* __restrict__ idx,
-    int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+    int32_t* __restrict__ counts, int32_t* __restrict__ offsets, const Normaliser norm) {
   __shared__ AdaptiveSmem sm;
   using G = WholeCta;
   extern __shared__ uint4 adaptive_dyn[];
@@ -690,7 +753,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
   const int n = seq_len_of(seqlens, b, n_max);
   const int k_eff = min(budget, n);
   const ForcedSet F = forced_set(n, k_eff, num_sink, window);
-  const RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
+  RowKeys keys = global_keys(scores + (size_t)p * n_max, n, F);
   const int forced = k_eff - F.free_slots;
   const int prot = min(max(min_protected, forced), k_eff);  // protected rows per head, forced included
   const bool none = prot == 0, all = prot >= n;             // nothing / everything is protected
@@ -700,8 +763,19 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
   // (its `prot` largest keys) and how many keys of that digit the cut takes
   clear_hist<G>(hist_all);
   if (tid == 0) sm.s.list_count[0] = sm.s.list_count[1] = 0;
-  __syncthreads();
-  if (!all) digit_histogram<G>(keys, 0xffffffffu, 0u, 0u, 0, hist_all);
+  if (norm.tile_sums != nullptr) {
+    // Alg. 1 line 6 first: the scores arrive unnormalised, with per-tile partial sums
+    const int tiles = (n + kTileRows - 1) / kTileRows;
+    const float S = head_sum_fixed_order<G>(
+        norm.tile_sums + (size_t)p * norm.tiles_per_head * norm.parts_per_tile, tiles * norm.parts_per_tile, sm.s);
+    if (tid == 0) norm.head_sums[p] = S;
+    scale_row_and_histogram<G>(scores + (size_t)p * n_max, keys, n_max, tiles * kTileRows, S, norm.raw != 0,
+                               hist_all, nullptr);
+    keys.written_here = true;
+  } else {
+    __syncthreads();
+    if (!all) digit_histogram<G>(keys, 0xffffffffu, 0u, 0u, 0, hist_all);
+  }
   __syncthreads();
   uint32_t d0 = 0xffffffffu, rank_own = 0;
   if (!none && !all) {
