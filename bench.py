@@ -26,9 +26,6 @@ METRIC = "kv_head_tokens_compressed_per_s"
 UNIT = "head-tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126 << 20
-# dram__bytes_read.sum + dram__bytes_write.sum of one sketch-kernel launch, from the ncu
-# capture summarised under profiles/ (None: not captured for the kernel as it stands)
-TRAFFIC_BYTES = {"cfg2": 1.0787e9, "cfg3": 16 * 1.0787e9}   # cfg3 = cfg2's capture x 16 head-tokens
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -132,6 +129,246 @@ def job_throughput(units_per_rank, world, seconds):
 
 # --------------------------------------------------------------------------- CUDA arm
 
+class Case:
+    """One workload resident in HBM with its output buffers; ``step()`` runs the whole hot path once."""
+
+    def __init__(self, cur, w, dev, whiten=False, three_calls=False, kv=None):
+        self.cur, self.w, self.dev, self.whiten, self.three_calls = cur, w, dev, whiten, three_calls
+        self.K, self.V, self.seqlens = kv if kv is not None else synth.make_kv(w, dev)
+        self.G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
+        self.sl = None if self.seqlens is None else torch.as_tensor(self.seqlens, device=dev)
+        self.desc = cur.make_desc(self.K, self.V, w.r, q_heads=w.q_heads, seqlens=self.sl, whiten=int(whiten),
+                                  ridge=1e-4 if whiten else 0.0)
+        self.ws = cur.alloc_workspace(self.desc, max(w.budget, 1), w.adaptive)
+        LB, H = w.folded_batch, w.kv_heads
+        P, cap = LB * H, min(w.budget, w.n_max)
+        self.scores = torch.empty((LB, H, w.n_max), dtype=torch.float32, device=dev)
+        self.sums = torch.empty((LB, H), dtype=torch.float32, device=dev)
+        if w.adaptive:
+            self.idx = torch.empty((P * cap,), dtype=torch.int32, device=dev)
+            self.Ko = torch.empty((P * cap, w.d), dtype=torch.bfloat16, device=dev)
+        else:
+            self.idx = torch.empty((LB, H, w.budget), dtype=torch.int32, device=dev)
+            self.Ko = torch.empty((LB, H, w.budget, w.d), dtype=torch.bfloat16, device=dev)
+        self.Vo = torch.empty_like(self.Ko)
+        self.cnt = torch.empty((LB, H), dtype=torch.int32, device=dev)
+        self.off = torch.empty((P + 1,), dtype=torch.int32, device=dev)
+        # inputs that fit in the 126 MB L2 are evicted between steps by writing a larger buffer
+        self.small = 2 * self.K.numel() * self.K.element_size() < 2 * L2_BYTES
+        self.flush = torch.empty((2 * L2_BYTES,), dtype=torch.uint8, device=dev) if self.small else None
+
+    def step(self, events=None, kernel_events=None):
+        cur, w = self.cur, self.w
+        if events is not None:
+            events[0].record()
+        if kernel_events is not None:
+            cur.curdkv_profile_next_score(*kernel_events)
+        if not self.three_calls:
+            # the whole path in one call; for fixed budgets its first kernel scores AND selects
+            cur.curdkv_compress(self.K, self.V, self.G, self.desc, w.budget, self.ws, num_sink=w.num_sink,
+                                window=w.window, adaptive=w.adaptive, alpha=w.alpha, scores=self.scores,
+                                head_sums=self.sums, idx=self.idx, head_counts=self.cnt,
+                                head_offsets=self.off, K_out=self.Ko, V_out=self.Vo)
+        else:
+            cur.curdkv_score(self.K, self.V, self.G, self.desc, self.ws, scores=self.scores, head_sums=self.sums)
+            if events is not None:
+                events[1].record()
+            cur.curdkv_select(self.scores, self.desc, w.budget, num_sink=w.num_sink, window=w.window,
+                              adaptive=w.adaptive, alpha=w.alpha, workspace=self.ws, idx=self.idx,
+                              head_counts=self.cnt, head_offsets=self.off)
+            if events is not None:
+                events[2].record()
+            cur.curdkv_compact(self.K, self.V, self.desc, self.idx, self.cnt, self.off, packed=w.adaptive,
+                               K_out=self.Ko, V_out=self.Vo, workspace=self.ws)
+        if events is not None:
+            events[3].record()
+
+    def timed(self, steps, warmup, barrier=None, flush=True):
+        """CUDA-event timing of `steps` steps after `warmup`; returns a dict of per-step figures."""
+        cur = self.cur
+        sync = barrier or torch.cuda.synchronize
+        for _ in range(max(warmup, 3)):
+            self.step()
+        sync()
+        flags = cur.curdkv_device_status(self.ws)
+        if flags:
+            raise RuntimeError(f"device status flags {flags:#x} after warm-up ({self.w.name})")
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+        # events the library records right around its streaming kernel (the dominant kernel); their
+        # handles only exist once they have been recorded
+        kv = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for pair in kv:
+            for e in pair:
+                e.record()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        use_flush = self.flush is not None and flush
+        sync()
+        launches0 = cur.launch_count()
+        t0.record()
+        for i in range(steps):
+            if use_flush:
+                self.flush.zero_()                 # sits between the per-step event pairs: not timed
+            self.step(ev[i], kv[i])
+        t1.record()
+        sync()
+        per_step = np.array([e[0].elapsed_time(e[3]) for e in ev])
+        out = {"ms_whole": t0.elapsed_time(t1) / steps, "ms_events": float(per_step.mean()),
+               "per_step": per_step, "kernel_ms": float(np.mean([a.elapsed_time(b) for a, b in kv])),
+               "launches": cur.launch_count() - launches0, "flushed": use_flush}
+        if self.three_calls:
+            st = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in ev]).mean(0)
+            out["stage_ms"] = {"score": float(st[0]), "select": float(st[1]), "compact": float(st[2])}
+        else:
+            out["stage_ms"] = {"score+select (streaming kernel, library events)": out["kernel_ms"],
+                               "rest of the call (gather; for AdaCurDKV also the selection kernel)":
+                                   float(per_step.mean()) - out["kernel_ms"]}
+        return out
+
+    def free(self):
+        for name in ("K", "V", "scores", "idx", "Ko", "Vo", "flush", "ws"):
+            setattr(self, name, None)
+        torch.cuda.empty_cache()
+
+
+def workload_text(w, whiten=False):
+    return (f"{w.name}: {w.layers} layers x batch {w.batch} x {w.kv_heads} KV heads "
+            f"(GQA {w.q_heads}:{w.kv_heads}), n={w.n_max}, d={w.d}, r={w.r}, "
+            f"budget {w.budget} incl. window {w.window}, sinks {w.num_sink}, "
+            + ("AdaCurDKV alpha=%.2f" % w.alpha if w.adaptive else "fixed per-head budget")
+            + (", whitened sketch (leverage scores, ridge 1e-4)" if whiten else "")
+            + (f", ragged lengths {w.ragged}" if w.ragged else ""))
+
+
+def kernel_traffic(kernel, tokens):
+    """DRAM bytes of one launch of `kernel`, from the ncu capture summarised under profiles/ (scaled by
+    head-tokens: the kernel streams every row once, so its traffic grows in proportion), or None when
+    no capture of the kernel as it stands is on file."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "streaming_kernel_traffic.json")) as f:
+            rec = json.load(f)["kernels"][kernel]
+        return rec["dram_bytes_per_launch"] * tokens / rec["head_tokens_per_launch"], rec["capture"]
+    except Exception:
+        return None, None
+
+
+def streaming_kernel_name(w, whiten, three_calls, sms=148):
+    if whiten:
+        return "sketch_items_kernel<%d>" % (32 if w.r <= 32 else 64)
+    fused = (not three_calls and not w.adaptive and w.ragged is None and w.r <= 32 and w.n_max >= 128
+             and w.folded_batch * w.kv_heads >= 4 * sms)
+    return "sketch_umma_kernel<%d, %s>" % (32 if w.r <= 32 else 64, "true" if fused else "false")
+
+
+def case_summary(case, t, world=1):
+    """Throughput and roofline figures of one timed case."""
+    w = case.w
+    tokens, read_bytes, write_bytes = workload_bytes(w, case.seqlens)
+    ms = t["ms_events"] if t["flushed"] else t["ms_whole"]
+    gbs = (read_bytes + write_bytes) / (ms * 1e-3) / 1e9
+    peak, _ = measured_peak()
+    return {"ms_per_step": ms, "stage_ms": t["stage_ms"], "head_tokens_per_step": tokens,
+            "head_tokens_per_s": tokens / (ms * 1e-3), "gb_per_s": gbs,
+            "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS, "frac_of_measured_copy": gbs / peak,
+            "streaming_kernel": streaming_kernel_name(w, case.whiten, case.three_calls),
+            "streaming_kernel_ms": t["kernel_ms"],
+            "streaming_kernel_gb_per_s": read_bytes / (t["kernel_ms"] * 1e-3) / 1e9,
+            "gpu_launches_per_step": t["launches"] / len(t["per_step"]),
+            "l2": "flushed between steps" if t["flushed"] else
+                  ("inputs fit in L2, not flushed" if case.small else "inputs exceed L2")}
+
+
+def oracle_check(case, lb):
+    """Part of the cpu-baseline leg: the fp64 oracle on ONE (layer, sequence) group of the case (all its
+    heads for AdaCurDKV, the first head otherwise), timed, and compared with what the GPU produced:
+    scores within 1e-3 relative, selection equal outside the 1e-4 tie band of a cut, gathered rows
+    byte-identical to the source rows at the GPU's indices."""
+    from oracle import curdkv_oracle as orc
+
+    w = case.w
+    heads = range(w.kv_heads) if w.adaptive else range(1)
+    n = w.n_max if case.seqlens is None else int(case.seqlens[lb])
+    Ku = synth.to_u16(case.K[lb, list(heads)])[None]
+    Vu = synth.to_u16(case.V[lb, list(heads)])[None]
+    G = synth.make_G(w.d, w.r, seed=0)
+    sl = None if case.seqlens is None else np.array([n], dtype=np.int32)
+    t0 = time.perf_counter()
+    rs, _ = orc.score(Ku, Vu, G, seqlens=sl)
+    if w.adaptive:
+        ridx, rcnt, roff = orc.select_adaptive(rs, w.budget, w.num_sink, w.window, w.alpha, seqlens=sl)
+    else:
+        ridx, rcnt = orc.select_fixed(rs, w.budget, w.num_sink, w.window, seqlens=sl)
+    dt = time.perf_counter() - t0
+    got = case.scores[lb, list(heads)].cpu().numpy().astype(np.float64)[None]
+    tol = 1e-3 * np.abs(rs) + 1e-6 * np.abs(rs).max(-1, keepdims=True)
+    ok = bool(np.all(np.abs(got - rs) <= tol))
+    H = w.kv_heads
+    off = case.off.cpu().numpy()
+    cnt = case.cnt.cpu().numpy()
+    gi = case.idx.cpu().numpy()
+    cuts, pairs = [], []
+    for j, h in enumerate(heads):
+        if w.adaptive:
+            g = gi[off[lb * H + h]: off[lb * H + h] + cnt[lb, h]]
+            r = ridx[roff[j]: roff[j + 1]]
+        else:
+            g, r = gi[lb, h, : cnt[lb, h]], ridx[0, j, : rcnt[0, j]]
+        forced_lo = n - min(w.window, n)
+        cand = [t for t in r.tolist() if w.num_sink <= t < forced_lo]
+        cuts.append(min(rs[0, j][t] for t in cand) if cand else np.inf)
+        pairs.append((j, h, g, r))
+        ok &= bool(np.all(np.diff(g) > 0)) and (len(g) == 0 or (g.min() >= 0 and g.max() < n))
+        rows = torch.as_tensor(g.astype(np.int64), device=case.K.device)
+        if w.adaptive:
+            base = int(off[lb * H + h])
+            ok &= bool(torch.equal(case.Ko[base: base + len(g)], case.K[lb, h][rows]))
+            ok &= bool(torch.equal(case.Vo[base: base + len(g)], case.V[lb, h][rows]))
+        else:
+            ok &= bool(torch.equal(case.Ko[lb, h, : len(g)], case.K[lb, h][rows]))
+            ok &= bool(torch.equal(case.Vo[lb, h, : len(g)], case.V[lb, h][rows]))
+    ok &= sum(len(g) for _, _, g, _ in pairs) == sum(len(r) for _, _, _, r in pairs)
+    lo_cut = min(cuts)
+    for j, h, g, r in pairs:
+        if not w.adaptive:
+            ok &= len(g) == len(r)
+        for t in set(g.tolist()) ^ set(r.tolist()):
+            rel = min(abs(rs[0, j][t] / c - 1.0) for c in (lo_cut, cuts[j]) if np.isfinite(c) and c > 0)
+            ok &= bool(rel < 1e-4)
+    return {"parity": bool(ok), "group": int(lb), "heads_checked": len(list(heads)), "oracle_seconds": dt,
+            "oracle_head_tokens_per_s": len(list(heads)) * n / dt}
+
+
+ALL_CONFIGS = ("cfg1", "cfg2", "cfg3_b1", "cfg4", "cfg5")
+
+
+def run_all_configs(cur, dev, steps, check):
+    """The other benchmark configurations, a few steps each, one after the other (each cache is freed
+    before the next is built): cfg1 with and without an L2-evicting write between steps, cfg2, the
+    headline shape at batch 1, cfg4 (AdaCurDKV, r = 64, 128K tokens) and cfg5 at three budgets."""
+    out = {}
+    for name in ALL_CONFIGS:
+        base = synth.CONFIGS[name]
+        kv = synth.make_kv(base, dev)
+        budgets = (128, 512, 2048) if name == "cfg5" else (base.budget,)
+        for k in budgets:
+            w = synth.shrink(base, budget=k)
+            case = Case(cur, w, dev, kv=kv)
+            key = name if len(budgets) == 1 else f"{name}_k{k}"
+            t = case.timed(steps, 3)
+            entry = case_summary(case, t)
+            entry["workload"] = workload_text(w)
+            if check:
+                entry["oracle_check"] = oracle_check(case, w.folded_batch // 2)
+            out[key if name != "cfg1" else "cfg1_l2_flushed"] = entry
+            if name == "cfg1":                             # the same 4 MiB cache left in L2 between steps
+                hot = case_summary(case, case.timed(steps, 3, flush=False))
+                hot["workload"] = entry["workload"]
+                out["cfg1_l2_resident"] = hot
+            case.free()
+        del kv
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args):
     from paper_2509_15038_b200 import binding as cur
 
@@ -151,125 +388,44 @@ def run_cuda(args):
         w = synth.shrink(w, batch=args.batch)
     if args.layers > 0:                                    # ... or with fewer layers (small profiling cases)
         w = synth.shrink(w, layers=args.layers)
-    K, V, seqlens = synth.make_kv(w, dev)
-    G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=dev)
-    sl = None if seqlens is None else torch.as_tensor(seqlens, device=dev)
-    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads, seqlens=sl, whiten=int(args.whiten),
-                         ridge=1e-4 if args.whiten else 0.0)
-    ws = cur.alloc_workspace(desc, w.budget, w.adaptive)
-    P = w.folded_batch * w.kv_heads
-    scores = torch.empty((w.folded_batch, w.kv_heads, w.n_max), dtype=torch.float32, device=dev)
-    sums = torch.empty((w.folded_batch, w.kv_heads), dtype=torch.float32, device=dev)
-    cap = min(w.budget, w.n_max)
-    if w.adaptive:
-        idx = torch.empty((P * cap,), dtype=torch.int32, device=dev)
-        Ko = torch.empty((P * cap, w.d), dtype=torch.bfloat16, device=dev)
-    else:
-        idx = torch.empty((w.folded_batch, w.kv_heads, w.budget), dtype=torch.int32, device=dev)
-        Ko = torch.empty((w.folded_batch, w.kv_heads, w.budget, w.d), dtype=torch.bfloat16, device=dev)
-    Vo = torch.empty_like(Ko)
-    cnt = torch.empty((w.folded_batch, w.kv_heads), dtype=torch.int32, device=dev)
-    off = torch.empty((P + 1,), dtype=torch.int32, device=dev)
-
-    def step(events=None, sketch_events=None):
-        if events is not None:
-            events[0].record()
-        if sketch_events is not None:
-            cur.curdkv_profile_next_score(*sketch_events)
-        if not args.three_calls:
-            # the whole path in one call; for fixed budgets its first kernel scores AND selects
-            cur.curdkv_compress(K, V, G, desc, w.budget, ws, num_sink=w.num_sink, window=w.window,
-                                adaptive=w.adaptive, alpha=w.alpha, scores=scores, head_sums=sums, idx=idx,
-                                head_counts=cnt, head_offsets=off, K_out=Ko, V_out=Vo)
-            if events is not None:
-                for e in events[1:]:
-                    e.record()
-            return
-        cur.curdkv_score(K, V, G, desc, ws, scores=scores, head_sums=sums)
-        if events is not None:
-            events[1].record()
-        cur.curdkv_select(scores, desc, w.budget, num_sink=w.num_sink, window=w.window,
-                          adaptive=w.adaptive, alpha=w.alpha, workspace=ws, idx=idx,
-                          head_counts=cnt, head_offsets=off)
-        if events is not None:
-            events[2].record()
-        cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=w.adaptive, K_out=Ko, V_out=Vo,
-                           workspace=ws)
-        if events is not None:
-            events[3].record()
+    case = Case(cur, w, dev, whiten=args.whiten, three_calls=args.three_calls)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    flags = cur.curdkv_device_status(ws)
-    if flags:
-        raise RuntimeError(f"device status flags {flags:#x} after warm-up")
-
     sampler = ClockSampler(local)
+    for _ in range(max(args.warmup, 3)):
+        case.step()
+    barrier()
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    barrier()
-    launches0 = cur.launch_count()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    # events the library records right around its sketch kernel (the dominant kernel); their
-    # handles only exist once they have been recorded
-    sk = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
-    for pair in sk:
-        for e in pair:
-            e.record()
-    t0 = torch.cuda.Event(enable_timing=True)
-    t1 = torch.cuda.Event(enable_timing=True)
-    # inputs that fit in the 126 MB L2 are evicted between steps by writing a larger buffer; the
-    # flushes then sit between the per-step event pairs and are not timed
-    small = 2 * K.numel() * K.element_size() < 2 * L2_BYTES
-    flush = torch.empty((2 * L2_BYTES,), dtype=torch.uint8, device=dev) if small else None
-    barrier()
-    t0.record()
-    for i in range(args.steps):
-        if flush is not None:
-            flush.zero_()
-        step(ev[i], sk[i])
-    t1.record()
-    barrier()
-    launches = cur.launch_count() - launches0
+    t = case.timed(args.steps, 0, barrier=barrier)
     clocks = sampler.stop() if rank == 0 else None
-    if small:
-        ms_step = max_over_ranks(sum(e[0].elapsed_time(e[3]) for e in ev), dev, world) / args.steps
-    else:
-        ms_step = max_over_ranks(t0.elapsed_time(t1), dev, world) / args.steps
-    stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in ev]).mean(0)
-    per_step = np.array([e[0].elapsed_time(e[3]) for e in ev])      # this rank's steps, one by one
+    ms_step = max_over_ranks(t["ms_events"] if t["flushed"] else t["ms_whole"], dev, world)
+    per_step = t["per_step"]
 
-    tokens, read_bytes, write_bytes = workload_bytes(w, seqlens)
+    tokens, read_bytes, write_bytes = workload_bytes(w, case.seqlens)
     pass_bytes = read_bytes                  # K + V once: what one streaming kernel reads
-    if args.whiten:
-        read_bytes *= 2                      # Gram pass + sketch pass
     value = job_throughput(tokens, world, ms_step * 1e-3)
     gbs = job_throughput(read_bytes + write_bytes, world, ms_step * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
-    sketch_ms = float(np.mean([a.elapsed_time(b) for a, b in sk]))
-    sketch_gbs = pass_bytes / (sketch_ms * 1e-3) / 1e9
+    kernel = streaming_kernel_name(w, args.whiten, args.three_calls)
+    kernel_gbs = pass_bytes / (t["kernel_ms"] * 1e-3) / 1e9
+    traffic, capture = kernel_traffic(kernel, tokens)
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": f"{w.name}: {w.layers} layers x batch {w.batch} x {w.kv_heads} KV heads "
-                        f"(GQA {w.q_heads}:{w.kv_heads}), n={w.n_max}, d={w.d}, r={w.r}, "
-                        f"budget {w.budget} incl. window {w.window}, sinks {w.num_sink}, "
-                        + ("AdaCurDKV alpha=%.2f" % w.alpha if w.adaptive else "fixed per-head budget")
-                        + (", whitened sketch (leverage scores, ridge 1e-4)" if args.whiten else "")
-                        + (f", ragged lengths {w.ragged}" if w.ragged else ""),
+            "workload": workload_text(w, args.whiten),
             "head_tokens_per_step": tokens, "seq_tokens_per_step": tokens // (w.layers * w.kv_heads),
+            "api": ("curdkv_score + curdkv_select + curdkv_compact" if args.three_calls else "curdkv_compress"),
             "l2": ("inputs (%.3f GB) fit in the 126 MB L2: a 252 MB buffer is written between steps "
-                   "(outside the timed event pairs)" % (read_bytes / 1e9)) if small else
+                   "(outside the timed event pairs)" % (read_bytes / 1e9)) if case.small else
                   ("inputs (%.1f GB) exceed the 126 MB L2, no flush between steps" % (read_bytes / 1e9)),
             "sharding": "independent replicas per rank, no collective",
         },
@@ -277,47 +433,61 @@ def run_cuda(args):
         "pct_of_nominal_8000": 100 * gbs / world / NOMINAL_HBM_GBS,
         "pct_of_measured_copy": 100 * gbs / world / peak,
         "seq_tokens_per_s": value / (w.layers * w.kv_heads),
-        "stage_ms": {"score": float(stage_ms[0]), "select": float(stage_ms[1]),
-                     "compact": float(stage_ms[2])},
+        "stage_ms": t["stage_ms"],
         "ms_per_step_median": float(np.median(per_step)), "ms_per_step_best": float(per_step.min()),
         "clocks": clocks,
-        "gpu_launches": int(launches),
+        "gpu_launches": int(t["launches"]),
         "roofline": {
-            "bound": "hbm",
-            "kernel": ("sketch_items_kernel" if args.whiten else "sketch_umma_kernel") + " (inside curdkv_score)",
-            "achieved": sketch_gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
-            "unit": "GB/s", "frac": sketch_gbs / peak,
-            "traffic": None if (args.whiten or args.batch > 0 or args.layers > 0) else TRAFFIC_BYTES.get(w.name),
-            "algorithmic_bytes_per_launch": pass_bytes, "ms_per_launch": sketch_ms,
+            "bound": "hbm", "kernel": kernel + " (inside " + ("curdkv_score" if args.three_calls else "curdkv_compress") + ")",
+            "achieved": kernel_gbs, "peak": peak,
+            "peak_kind": peak_kind + " copy bandwidth (a read+write mix; this kernel only reads, "
+                                     "which is why the fraction can exceed 1)",
+            "unit": "GB/s", "frac": kernel_gbs / peak, "frac_of_nominal_8000": kernel_gbs / NOMINAL_HBM_GBS,
+            "traffic": traffic, "traffic_source": capture,
+            "algorithmic_bytes_per_launch": pass_bytes, "ms_per_launch": t["kernel_ms"],
             "timer": "CUDA events recorded by the library around the kernel, mean over the timed steps",
         },
     }
     if args.graph and world == 1:
         # the same step captured once into a CUDA graph and replayed: what a caller that runs the
-        # three calls back to back saves in launch overhead (only visible on small workloads)
+        # calls back to back saves in launch overhead (only visible on small workloads)
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            step()
+            case.step()
         torch.cuda.current_stream().wait_stream(side)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            step()
+            case.step()
         gev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
         for i in range(args.steps):
-            if flush is not None:
-                flush.zero_()
+            if case.flush is not None:
+                case.flush.zero_()
             gev[i][0].record()
             graph.replay()
             gev[i][1].record()
         torch.cuda.synchronize()
         out["cuda_graph"] = {"ms_per_step": float(np.mean([a_.elapsed_time(b_) for a_, b_ in gev])),
                              "eager_ms_per_step": ms_step}
-    out["e2e"] = run_e2e(cur, w, K, V, seqlens, value_tokens=tokens, world=world, dev=dev,
+    if not args.three_calls and world == 1 and not args.no_all_configs:
+        # the separate calls on the same cache, for the stage split and the comparison
+        ref = Case(cur, w, dev, whiten=args.whiten, three_calls=True, kv=(case.K, case.V, case.seqlens))
+        rt = ref.timed(min(args.steps, 10), 3)
+        out["three_calls"] = {"ms_per_step": rt["ms_events"] if rt["flushed"] else rt["ms_whole"],
+                              "stage_ms": rt["stage_ms"], "streaming_kernel_ms": rt["kernel_ms"]}
+        ref.K = ref.V = None
+        ref.free()
+    out["e2e"] = run_e2e(cur, w, case.K, case.V, case.seqlens, value_tokens=tokens, world=world, dev=dev,
                          steps=min(args.steps, args.e2e_steps))
-    if rank == 0:
-        if not args.no_cpu_baseline and world == 1:
+    if rank == 0 and world == 1:
+        if not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(w, core_seconds=20.0)
+            out["cpu_baseline"]["headline_check"] = oracle_check(case, w.folded_batch // 2)
+        case.free()
+        if not args.no_all_configs and args.workload == "cfg3" and args.batch == 0 and args.layers == 0:
+            out["all_configs"] = run_all_configs(cur, dev, steps=min(args.steps, 10),
+                                                 check=not args.no_cpu_baseline)
+    if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -636,6 +806,48 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_dry(args):
+    """Host logic of the N-rank run without a GPU (gloo): every rank takes its own replica of the
+    workload description, "times" a fake step of 1 + rank/10 ms, the slowest rank's time is agreed
+    on and rank 0 prints the line.  What the real run does around its kernels, and nothing else."""
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    w = rank_workload(synth.CONFIGS[args.workload], rank)
+    tokens, read_bytes, write_bytes = workload_bytes(w, synth.make_seqlens(w))
+    ms_step = max_over_ranks(1.0 + rank / 10.0, torch.device("cpu"), world)
+    seeds = [None] * world
+    if world > 1:
+        dist.all_gather_object(seeds, w.data_seed)
+        dist.barrier()
+    else:
+        seeds = [w.data_seed]
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": job_throughput(tokens, world, ms_step * 1e-3), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+                          "higher_is_better": True, "scaling": "weak", "data": "none (dry run of the host logic)",
+                          "config": {"workload": workload_text(w), "head_tokens_per_step": tokens,
+                                     "data_seeds": seeds}}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def spawn_ranks(n):
+    """`bench.py --gpus N` started by hand: re-launch this command as N ranks, one per GPU, the way
+    the driver does (torch.distributed.run on 127.0.0.1); rank 0 prints the one line."""
+    import socket
+
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -652,6 +864,10 @@ def main():
     ap.add_argument("--three-calls", action="store_true",
                     help="time curdkv_score + curdkv_select + curdkv_compact instead of curdkv_compress")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-all-configs", action="store_true",
+                    help="skip the other configurations (all_configs) and the three-call comparison")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="host logic of the multi-rank path only (gloo, no CUDA): for tests on a CPU box")
     ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
                     help="--workload decode: compress inside the cache (unordered) or copy in order")
     ap.add_argument("--whiten", action="store_true",
@@ -659,7 +875,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3,
                     help="steps of the host-buffer end-to-end leg (0 disables it)")
     args = ap.parse_args()
-    if args.workload in ("decode", "evict"):
+    if args.gpus > 1 and "RANK" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
+    if args.dry_run:
+        run_dry(args)
+    elif args.workload in ("decode", "evict"):
         if args.impl == "reference":
             raise SystemExit("the reference arm times the prefill workloads only")
         run_decode(args) if args.workload == "decode" else run_evict(args)

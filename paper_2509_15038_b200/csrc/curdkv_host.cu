@@ -2,7 +2,7 @@
 // Chunks of batch elements are copied to the device, scored, selected and
 // gathered, and the results copied back, on two internal streams so that the
 // copies of one chunk overlap the kernels and the copies of the next.  Built
-// only on the public device entry points of curdkv.h.
+// only on the public device entry point curdkv_compress.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -25,7 +25,7 @@ inline int64_t cap_rows(const curdkv_desc* d, int32_t budget) {
 bool slot_layout(const curdkv_desc* d, int32_t budget, int32_t adaptive, int32_t cb, SlotLayout* L) {
   curdkv_desc c = *d;
   c.batch = cb;
-  const size_t ws = curdkv_workspace_bytes(&c, budget, adaptive);
+  const size_t ws = curdkv_workspace_bytes(&c, budget > 0 ? budget : 1, adaptive);
   if (ws == 0) return false;
   const size_t P = (size_t)cb * d->kv_heads;
   const size_t kv = P * (size_t)d->n_max * d->d * 2;
@@ -155,15 +155,10 @@ curdkv_status curdkv_compress_host(const void* K_host, const void* V_host, const
     int32_t* idx = reinterpret_cast<int32_t*>(sb + L.idx);
     int32_t* counts = reinterpret_cast<int32_t*>(sb + L.counts);
     int32_t* offsets = reinterpret_cast<int32_t*>(sb + L.offsets);
-    curdkv_status stt = curdkv_score(sb + L.K, sb + L.V, G_dev, g_per_head, &c, scores,
-                                     reinterpret_cast<float*>(sb + L.sums), sb + L.workspace,
-                                     L.total - L.workspace, stream);
-    if (stt == CURDKV_OK)
-      stt = curdkv_select(scores, &c, budget, nullptr, num_sink, window, adaptive, alpha, idx, counts,
-                          offsets, sb + L.workspace, L.total - L.workspace, stream);
-    if (stt == CURDKV_OK)
-      stt = curdkv_compact(sb + L.K, sb + L.V, &c, idx, adaptive ? 0 : budget, counts, offsets,
-                           sb + L.K_out, sb + L.V_out, adaptive ? 0 : budget, sb + L.workspace, stream);
+    const curdkv_status stt =
+        curdkv_compress(sb + L.K, sb + L.V, G_dev, g_per_head, &c, budget, nullptr, num_sink, window, adaptive,
+                        alpha, scores, reinterpret_cast<float*>(sb + L.sums), idx, counts, offsets,
+                        sb + L.K_out, sb + L.V_out, sb + L.workspace, L.total - L.workspace, stream);
     if (stt != CURDKV_OK) { fail(stt); break; }
 
     copy(counts_host + (size_t)b0 * H, counts, P * 4, cudaMemcpyDeviceToHost);

@@ -56,3 +56,24 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["gpu_launches"] == 0
+
+
+def test_gpus_flag_spawns_one_rank_per_gpu_dry_run():
+    """`bench.py --gpus 2` started without a launcher re-launches itself as two ranks; with --dry-run
+    they run the host logic on gloo: the line says n_gpus 2, carries the slowest rank's time and the
+    whole-job rate, and every rank drew its own data seed."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run",
+                          "--workload", "cfg2"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak"
+    assert line["ms_per_step"] == 1.1                        # max over ranks of 1.0 and 1.1
+    tokens = 32 * 8 * 8192
+    assert line["value"] == 2 * tokens / 1.1e-3
+    assert len(set(line["config"]["data_seeds"])) == 2
+    one = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--dry-run", "--workload", "cfg2"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert json.loads(one.stdout.strip().splitlines()[-1])["n_gpus"] == 1
