@@ -251,7 +251,8 @@ def kernel_traffic(kernel, tokens):
         return None, None
 
 
-def streaming_kernel_name(w, whiten, three_calls, sms=148):
+def streaming_kernel_name(w, whiten, three_calls):
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
     if whiten:
         return "sketch_items_kernel<%d>" % (32 if w.r <= 32 else 64)
     fused = (not three_calls and not w.adaptive and w.ragged is None and w.r <= 32 and w.n_max >= 128
@@ -571,9 +572,13 @@ def run_decode(args):
 
     def step():
         nonlocal live
+        if inplace:       # one call: new rows copied and heads selected in one launch, survivors stay
+            cur.curdkv_cache_step(caches[live], K_new, V_new, G, k, ws, num_sink=c["num_sink"],
+                                  window=c["window"])                    # put, at most `chunk` rows move
+            return
         cur.curdkv_cache_append(caches[live], K_new, V_new, G, ws)
-        if inplace:       # survivors stay put, at most `chunk` rows per head move into the holes
-            cur.curdkv_cache_compress_inplace(caches[live], k, ws, num_sink=c["num_sink"], window=c["window"])
+        if False:
+            pass
         else:             # ordered copy of all survivors into the other cache
             cur.curdkv_cache_compress(caches[live], caches[1 - live], k, ws, num_sink=c["num_sink"],
                                       window=c["window"])

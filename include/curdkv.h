@@ -226,8 +226,8 @@ curdkv_status curdkv_compress_host(const void* K_host, const void* V_host, const
                                    int32_t* counts_host, int32_t* offsets_host, void* arena,
                                    size_t arena_bytes, int32_t chunk_batch, uint32_t* status_flags_host);
 
-/* ---- Generation phase (Sec. 3.2: "can be applied during the pre-filling as well as
- * the token generation phase"; the paper leaves the procedure open).  Reading used:
+/* ---- Generation phase.  Sec. 3.2 notes that the method also applies while tokens are
+ * generated, not only at prefill, and gives no procedure for it.  Reading used:
  * a cache holds, per (sequence, KV head), up to `capacity` rows of K and V with their
  * original token positions and their unnormalised scores l^KV (Alg. 1 lines 2-5).
  * curdkv_cache_append scores newly generated rows and appends them;
@@ -264,7 +264,11 @@ curdkv_status curdkv_cache_append(const curdkv_cache* cache, const void* K_new, 
 /* Alg. 1 lines 6-10 on the rows held in `in`; the kept rows, scores and positions go
  * to `out` (a different cache with capacity >= min(budget, in->capacity); the two
  * must not overlap), which also receives the counters.  Sequences holding at most
- * `budget` rows are copied unchanged.  desc supplies batch, kv_heads and d. */
+ * `budget` rows are copied unchanged.  desc supplies batch, kv_heads and d.
+ * Forced rows are found by their POSITIONS (below num_sink; among the most recent
+ * `window`), so the call also works on a cache that curdkv_cache_compress_inplace has
+ * left unordered; the kept rows come out in the order of their slots in `in`, which is
+ * ascending position order when `in` was ordered.  Requires num_sink + window <= budget. */
 curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* out,
                                     const curdkv_desc* desc, int32_t budget, int32_t num_sink,
                                     int32_t window, void* workspace, size_t workspace_bytes,
@@ -316,6 +320,18 @@ curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compresse
 curdkv_status curdkv_cache_compress_inplace(const curdkv_cache* cache, const curdkv_desc* desc,
                                             int32_t budget, int32_t num_sink, int32_t window,
                                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* One generation step in two launches after the scoring of the new rows: what
+ * curdkv_cache_append followed by curdkv_cache_compress_inplace does (same arguments, same
+ * resulting cache bit for bit, same status flags).  The selection needs only scores and
+ * positions, so one kernel copies the new rows into the cache and, beside those copies,
+ * selects for every head from the held rows' scores and the new rows' fresh ones; a second
+ * kernel moves the survivors into the holes and sets the counters.  Requires budget >= 1 and
+ * num_sink + window <= budget; capacities above 36,864 rows run as the two calls. */
+curdkv_status curdkv_cache_step(const curdkv_cache* cache, const void* K_new, const void* V_new,
+                                const float* G, int32_t g_per_head, const curdkv_desc* desc_new,
+                                int32_t budget, int32_t num_sink, int32_t window, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream);
 
 /* GQA (Sec. 3.2): query head q uses KV head q / (q_heads / kv_heads).  Writes
  * kv_head_of_q int32 [q_heads] (device) so that attention consumers can index

@@ -29,7 +29,7 @@ EXPORTS = (
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
     "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
     "curdkv_eviction_loss", "curdkv_gqa_expand", "curdkv_cache_compress_inplace",
-    "curdkv_selftest_bounded_wait", "curdkv_compress",
+    "curdkv_selftest_bounded_wait", "curdkv_compress", "curdkv_cache_step",
 )
 
 
@@ -114,6 +114,8 @@ def load():
     lib.curdkv_cache_compress.argtypes = [cp, cp, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
     lib.curdkv_cache_compress_inplace.restype = ctypes.c_int
     lib.curdkv_cache_compress_inplace.argtypes = [cp, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
+    lib.curdkv_cache_step.restype = ctypes.c_int
+    lib.curdkv_cache_step.argtypes = [cp, vp, vp, vp, i32, dp, i32, i32, i32, vp, ctypes.c_size_t, vp]
     lib.curdkv_attention_workspace_bytes.restype = ctypes.c_size_t
     lib.curdkv_attention_workspace_bytes.argtypes = [dp]
     lib.curdkv_attention_out.restype = ctypes.c_int
@@ -400,6 +402,16 @@ def curdkv_cache_compress_inplace(cache: DeviceCache, budget: int, workspace: to
                                                 int(num_sink), int(window), _ptr(workspace),
                                                 workspace.numel(), _stream())
     _check(code, "curdkv_cache_compress_inplace")
+
+
+def curdkv_cache_step(cache: DeviceCache, K_new, V_new, G, budget: int, workspace: torch.Tensor, *,
+                      num_sink: int = 0, window: int = 0, t_new: Optional[torch.Tensor] = None) -> None:
+    """One generation step: append K_new, V_new ``[B, Hkv, t, d]`` and compress in place to ``budget``."""
+    desc = make_desc(K_new, V_new, G.shape[-1], seqlens=t_new)
+    code = load().curdkv_cache_step(ctypes.byref(cache.c), _ptr(K_new), _ptr(V_new), _ptr(G), int(G.dim() == 3),
+                                    ctypes.byref(desc), int(budget), int(num_sink), int(window),
+                                    _ptr(workspace), workspace.numel(), _stream())
+    _check(code, "curdkv_cache_step")
 
 
 def curdkv_attention_out(Q, K, V, desc: Desc, *, scale: float = 1.0, head_rows=None, head_offsets=None,

@@ -4,6 +4,7 @@
 // compression step carries scores and positions along with the gathered rows.
 #pragma once
 #include "common.cuh"
+#include "select.cuh"
 
 namespace curdkv {
 
@@ -149,13 +150,23 @@ __global__ void __launch_bounds__(256) cache_keyed_scores_kernel(const CacheView
 // are copied into the slots < kept that were not kept ("holes"), so that the survivors occupy
 // slots [0, kept) again.  At most min(kept, held - kept) rows move.  grid = batch*heads,
 // block = 256, dynamic shared memory = capacity bytes (slot flags); holes: int32 [problems][capacity].
+// With set_counters the CTA of a sequence's first head also leaves count[b] = rows kept and adds
+// `appended` rows (t_new[b], or t) to total[b]: no kernel of this launch reads either.
 __global__ void __launch_bounds__(256) cache_fill_holes_kernel(const CacheView c, const int32_t* idx,
                                                                int budget, const int32_t* counts, int heads,
-                                                               int d, int32_t* holes, uint32_t* status) {
+                                                               int d, int32_t* holes, uint32_t* status,
+                                                               int set_counters, const int32_t* t_new, int t) {
   extern __shared__ unsigned char slot_kept[];
   __shared__ int s_first_mover, s_base, s_warp_tot[8];
   const int p = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int kept = min(counts[p], c.capacity);
+  if (set_counters && tid == 0 && p % heads == 0) {
+    const int b = p / heads;
+    int tb = t_new != nullptr ? t_new[b] : t;
+    tb = tb < 0 ? 0 : (tb > t ? t : tb);
+    c.count[b] = kept;
+    c.total[b] += tb;
+  }
   const int32_t* ix = idx + (size_t)p * budget;
   int32_t* my_holes = holes + (size_t)p * c.capacity;
   for (int s = tid; s < kept; s += 256) slot_kept[s] = 0;
@@ -238,10 +249,106 @@ __global__ void __launch_bounds__(256) cache_fill_holes_kernel(const CacheView c
   }
 }
 
-// count[b] = rows kept (the same for every head of a sequence).  grid = ceil(batch / 256).
-__global__ void cache_set_count_kernel(CacheView cache, const int32_t* counts, int heads, int batch) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < batch) cache.count[b] = min(counts[b * heads], cache.capacity);
+// ---- one generation step: append the new rows AND select in place, in one launch -------------
+// The selection of a head only needs the scores and positions of its rows, not the rows
+// themselves, so it runs beside the copies of the new rows: of every (chunks + 1) consecutive CTAs
+// the first selects for one head (keys staged in shared memory from the held rows' scores and
+// positions and from the new rows' fresh scores; it also files the new rows' scores and
+// positions in the cache), the others copy 32 new rows of that head each.  The counters are
+// only read here; cache_fill_holes_kernel sets them afterwards.
+struct StepArgs {
+  AppendArgs append;
+  int budget, num_sink, window;
+  int stage_quads, list_cap;       // shared-memory copy of a head's keys, candidate list
+  int32_t* idx;                    // [batch*heads][budget]
+  int32_t* counts;                 // [batch*heads]
+};
+
+__global__ void __launch_bounds__(256) cache_step_kernel(const StepArgs s) {
+  __shared__ SelectSmem sm;
+  extern __shared__ uint4 step_keys[];                     // stage_quads quads, then the list
+  const AppendArgs& a = s.append;
+  const int chunks_per_head = (a.t + kAppendRowsPerCta - 1) / kAppendRowsPerCta;
+  const int p = blockIdx.x / (chunks_per_head + 1), role = blockIdx.x % (chunks_per_head + 1);
+  const int b = p / a.heads, h = p % a.heads;
+  int tb = a.t_new != nullptr ? a.t_new[b] : a.t;
+  tb = tb < 0 ? 0 : (tb > a.t ? a.t : tb);
+  int held = a.cache.count[b];
+  if (held < 0 || held > a.cache.capacity) {               // counters the caller never set up
+    if (threadIdx.x == 0 && role == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+    held = held < 0 ? 0 : a.cache.capacity;
+  }
+  const int first_pos = a.cache.total[b], offered = tb;
+  if (tb > a.cache.capacity - held) {
+    if (threadIdx.x == 0 && role == 0) flag_status(a.status, CURDKV_DEV_CACHE_FULL);
+    tb = a.cache.capacity - held;
+  }
+  if (role > 0) {
+    // ------------------------------------------------------------ copy 32 new rows
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+    const KvView& T = half ? a.V_new : a.K_new;
+    const __nv_bfloat16* src = T.base + b * T.stride_b + h * T.stride_h;
+    __nv_bfloat16* dst = (half ? a.cache.V : a.cache.K) + ((size_t)p * a.cache.capacity + held) * a.d;
+    const int chunks = a.d >> 3;
+    const int row0 = (role - 1) * kAppendRowsPerCta + warp;
+    for (int c = l16; c < chunks; c += 16) {
+      uint4 v[kAppendRowsPerCta / kAppendWarps];
+#pragma unroll
+      for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
+        const int i = row0 + j * kAppendWarps;
+        if (i < tb) v[j] = __ldg(reinterpret_cast<const uint4*>(src + i * T.stride_n) + c);
+      }
+#pragma unroll
+      for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
+        const int i = row0 + j * kAppendWarps;
+        if (i < tb) reinterpret_cast<uint4*>(dst + (size_t)i * a.d)[c] = v[j];
+      }
+    }
+    return;
+  }
+  // -------------------------------------------------------------- select for head p (Alg. 1 lines 7-9)
+  using G = WholeCta;
+  const int n = held + tb;                                 // rows the head holds after the append
+  const int k_eff = min(s.budget, n);
+  const int recent = first_pos + offered - s.window;       // positions from here on are the window
+  float* raw_row = a.cache.raw + (size_t)p * a.cache.capacity;
+  int32_t* pos_row = a.cache.pos + (size_t)p * a.cache.capacity;
+  const float* raw_new = a.raw_new + (size_t)p * a.t;
+  clear_hist<G>(sm.hist);
+  if (threadIdx.x == 0) sm.list_count[0] = 0;
+  __syncthreads();
+  {
+    DigitRun run;
+    uint32_t* keys32 = reinterpret_cast<uint32_t*>(step_keys);
+    const int padded = ((n + 3) >> 2) << 2;
+    for (int j = threadIdx.x; j < padded; j += 256) {
+      uint32_t key = 0u;                                   // beyond the rows held: never kept
+      if (j < n) {
+        float raw;
+        int pos;
+        if (j < held) {
+          raw = raw_row[j];
+          pos = pos_row[j];
+        } else {                                           // a new row: file its score and position
+          raw = raw_new[j - held];
+          pos = first_pos + (j - held);
+          raw_row[j] = raw;
+          pos_row[j] = pos;
+        }
+        key = (pos < s.num_sink || pos >= recent) ? kForcedKey : score_key(raw);
+        run.add(key >> 20, sm.hist);
+      }
+      keys32[j] = key;
+    }
+    run.flush(sm.hist);
+  }
+  __syncthreads();
+  const ForcedSet F = forced_set(n, k_eff, 0, 0);          // forced rows carry the top key already
+  RowKeys keys{nullptr, step_keys, n, 0, n, true, false};
+  const KeyList list{reinterpret_cast<uint2*>(step_keys + s.stage_quads), &sm.list_count[0], (uint32_t)s.list_cap};
+  select_fixed_row<G>(keys, F, k_eff, s.budget, step_keys, s.stage_quads, list, true,
+                      s.idx + (size_t)p * s.budget, sm);
+  if (threadIdx.x == 0) s.counts[p] = k_eff;
 }
 
 }  // namespace curdkv

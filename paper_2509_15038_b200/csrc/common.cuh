@@ -18,6 +18,13 @@ constexpr size_t kStatusBytes = 256;
 // Adds one to the library's launch counter (defined beside the C ABI).
 void count_launch();
 
+// curdkv_score without its last step: `scores` receive l^K l^V (Alg. 1 line 5) as the score
+// kernels leave them, entries at or beyond a sequence's length are unspecified, head sums are not
+// formed.  For callers that read the valid entries only (defined beside the C ABI).
+curdkv_status score_unnormalised(const void* K, const void* V, const float* G, int32_t g_per_head,
+                                 const curdkv_desc* desc, float* scores, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
+
 struct KvView {          // one bf16 tensor [batch][heads][n_max][d], strides in elements
   const __nv_bfloat16* base;
   int64_t stride_b, stride_h, stride_n;

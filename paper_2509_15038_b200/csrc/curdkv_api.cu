@@ -105,6 +105,13 @@ int sm_count() {
   return n;
 }
 
+// SMs the host-side heuristics plan for: the current device's, or a B200's where no device can be
+// asked (workspace sizes are also queried on machines without a GPU).
+int planning_sm_count() {
+  const int n = sm_count();
+  return n > 0 ? n : 148;
+}
+
 // Events a caller asked to have recorded around the next sketch kernel of this
 // host thread (curdkv_profile_next_score).
 thread_local cudaEvent_t g_profile_start = nullptr, g_profile_stop = nullptr;
@@ -170,7 +177,7 @@ void* static_scratch_ptr() {
 
 // Whitened scoring cuts every head into this many runs of tiles (the work items of the two
 // streaming kernels).  An item costs its tiles plus a fixed part (staging W, draining and storing
-// a partial Gram matrix: about ten tiles' worth, measured), and every CTA walks ceil(P s / 148)
+// a partial Gram matrix: about ten tiles' worth, measured), and every CTA walks ceil(P s / SMs)
 // items, so the count that minimises rounds x (tiles per item + fixed part) is taken: many
 // segments balance the SMs, few keep the fixed part small.
 int whiten_segments(const curdkv_desc* d) {
@@ -178,10 +185,11 @@ int whiten_segments(const curdkv_desc* d) {
   if (P <= 0) return 1;
   const int tiles = tiles_per_head(d);
   constexpr int64_t kItemOverheadTiles = 10;
+  const int64_t sms = planning_sm_count();
   int best = 1;
   int64_t best_cost = -1;
   for (int s = 1; s <= tiles && s <= 1024; ++s) {
-    const int64_t rounds = (P * s + 147) / 148;
+    const int64_t rounds = (P * s + sms - 1) / sms;
     const int64_t cost = rounds * ((tiles + s - 1) / s + kItemOverheadTiles);
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
@@ -217,8 +225,22 @@ KvView view_of(const void* base, int64_t sb, int64_t sh, int64_t sn) {
 
 }  // namespace
 
+namespace {
+curdkv_status score_impl(const void* K, const void* V, const float* G, int32_t g_per_head,
+                         const curdkv_desc* desc, float* scores, float* head_sums, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream, bool normalise, int* parts_per_tile);
+}  // namespace
+
 namespace curdkv {
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+curdkv_status score_unnormalised(const void* K, const void* V, const float* G, int32_t g_per_head,
+                                 const curdkv_desc* desc, float* scores, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  float unused_sums = 0.f;                                 // only checked for NULL
+  return score_impl(K, V, G, g_per_head, desc, scores, &unused_sums, workspace, workspace_bytes, cuda_stream,
+                    false, nullptr);
+}
 }  // namespace curdkv
 
 extern "C" {
@@ -474,10 +496,10 @@ curdkv_status select_impl(float* scores, const curdkv_desc* desc, int32_t budget
     if (P * (int64_t)(budget < desc->n_max ? budget : desc->n_max) > 0x7fffffffLL)
       return CURDKV_ERR_UNSUPPORTED;
     const int min_protected = (int)floor(alpha * (double)budget);
-    // With one CTA of 1024 threads per SM, floor(148 / heads) clusters run at a time.  When the
+    // With one CTA of 1024 threads per SM, floor(SMs / heads) clusters run at a time.  When the
     // batch needs more than one such round, CTAs of 512 threads (two per SM) keep all clusters
     // resident instead.
-    const int64_t one_round = 148 / (desc->kv_heads > 0 ? desc->kv_heads : 1);
+    const int64_t one_round = planning_sm_count() / (desc->kv_heads > 0 ? desc->kv_heads : 1);
     const bool small_ctas = desc->batch > one_round;
     auto launch = [&](auto kernel, int threads) -> cudaError_t {
       if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

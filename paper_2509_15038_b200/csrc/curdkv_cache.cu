@@ -78,9 +78,9 @@ curdkv_status curdkv_cache_append(const curdkv_cache* cache, const void* K_new, 
   d.raw_scores = 1;
   d.score_mode = 0;
   d.whiten = 0;                       // a row's score must not depend on the rows it arrives with
-  curdkv_status st = curdkv_score(K_new, V_new, G, g_per_head, &d, raw_new,
-                                  reinterpret_cast<float*>(ws + L.sums), ws + L.score_ws,
-                                  L.raw_new - L.score_ws, cuda_stream);
+  // only the real rows' scores are read below: no normalisation pass, no head sums
+  curdkv_status st = score_unnormalised(K_new, V_new, G, g_per_head, &d, raw_new, ws + L.score_ws,
+                                        L.raw_new - L.score_ws, cuda_stream);
   if (st != CURDKV_OK) return st;
   const int64_t P = (int64_t)d.batch * d.kv_heads;
   if (P == 0 || d.n_max == 0) return CURDKV_OK;
@@ -115,6 +115,7 @@ curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* 
   if (!cache_ok(in) || !cache_ok(out) || desc == nullptr || workspace == nullptr)
     return CURDKV_ERR_INVALID_ARG;
   if (budget < 0 || num_sink < 0 || window < 0) return CURDKV_ERR_INVALID_ARG;
+  if ((int64_t)num_sink + window > budget) return CURDKV_ERR_INVALID_ARG;   // forced rows must fit
   if (in->K == out->K || in->V == out->V || in->raw == out->raw || in->pos == out->pos)
     return CURDKV_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
@@ -140,8 +141,16 @@ curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* 
   d.score_mode = 0;
   d.use_projection = 1;
   d.raw_scores = 0;
-  curdkv_status st = curdkv_select(in->raw, &d, budget, nullptr, num_sink, window, 0, 0.0, idx, counts,
-                                   nullptr, ws + L.score_ws, L.raw_new - L.score_ws, cuda_stream);
+  // Forced rows are found by POSITION (sinks: positions below num_sink; window: the most recent
+  // positions), whatever slots they sit in: a cache that curdkv_cache_compress_inplace has left
+  // unordered is handled like an ordered one.  They enter the selection with an infinite key.
+  float* keyed = reinterpret_cast<float*>(ws + L.keyed);
+  cache_keyed_scores_kernel<<<(unsigned)P, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      view_of(in), desc->kv_heads, num_sink, window, keyed);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  curdkv_status st = curdkv_select(keyed, &d, budget, nullptr, 0, 0, 0, 0.0, idx, counts, nullptr,
+                                   ws + L.score_ws, L.raw_new - L.score_ws, cuda_stream);
   if (st != CURDKV_OK) return st;
   if (budget > 0) {
     st = curdkv_compact(in->K, in->V, &d, idx, budget, counts, nullptr, out->K, out->V, out->capacity,
@@ -196,11 +205,79 @@ curdkv_status curdkv_cache_compress_inplace(const curdkv_cache* cache, const cur
     return CURDKV_ERR_CUDA;
   cache_fill_holes_kernel<<<(unsigned)P, 256, (size_t)cache->capacity, stream>>>(
       view, idx, budget, counts, d.kv_heads, d.d, reinterpret_cast<int32_t*>(ws + L.holes),
-      reinterpret_cast<uint32_t*>(ws + L.score_ws));
+      reinterpret_cast<uint32_t*>(ws + L.score_ws), 1, nullptr, 0);      // sets count[b]; total[b] += 0
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
-  cache_set_count_kernel<<<(unsigned)((d.batch + 255) / 256), 256, 0, stream>>>(view, counts, d.kv_heads,
-                                                                                d.batch);
+  return CURDKV_OK;
+}
+
+curdkv_status curdkv_cache_step(const curdkv_cache* cache, const void* K_new, const void* V_new,
+                                const float* G, int32_t g_per_head, const curdkv_desc* desc_new,
+                                int32_t budget, int32_t num_sink, int32_t window, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
+  if (!cache_ok(cache) || desc_new == nullptr || workspace == nullptr) return CURDKV_ERR_INVALID_ARG;
+  if (budget < 1 || num_sink < 0 || window < 0 || (int64_t)num_sink + window > budget)
+    return CURDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  CacheWorkspace L;
+  if (!layout(desc_new->batch, desc_new->kv_heads, desc_new->n_max, cache->capacity, budget, &L))
+    return CURDKV_ERR_INVALID_ARG;
+  if (workspace_bytes < L.total) return CURDKV_ERR_WORKSPACE;
+  const int64_t P = (int64_t)desc_new->batch * desc_new->kv_heads;
+  // the selection CTAs keep a head's keys and its candidate list in shared memory
+  const int list_cap = cache->capacity <= 4096 ? kSelListCap / 4 : (cache->capacity <= 16384 ? kSelListCap / 2 : kSelListCap);
+  const size_t stage_bytes = (((size_t)cache->capacity + 3) / 4) * sizeof(uint4);
+  const int64_t chunks = (desc_new->n_max + kAppendRowsPerCta - 1) / kAppendRowsPerCta;
+  if (stage_bytes > (size_t)kSelStageBytes || desc_new->n_max < 1 || P < 1 || P * (chunks + 1) > 0x7fffffffLL ||
+      desc_new->d % 8 != 0) {
+    // shapes the one-launch form does not cover: the two calls it stands for
+    curdkv_status st = curdkv_cache_append(cache, K_new, V_new, G, g_per_head, desc_new, workspace,
+                                           workspace_bytes, cuda_stream);
+    if (st != CURDKV_OK) return st;
+    curdkv_desc d = *desc_new;
+    return curdkv_cache_compress_inplace(cache, &d, budget, num_sink, window, workspace, workspace_bytes,
+                                         cuda_stream);
+  }
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  float* raw_new = reinterpret_cast<float*>(ws + L.raw_new);
+  curdkv_desc d = *desc_new;
+  d.raw_scores = 1;
+  d.score_mode = 0;
+  d.whiten = 0;
+  curdkv_status st = score_unnormalised(K_new, V_new, G, g_per_head, &d, raw_new, ws + L.score_ws,
+                                        L.raw_new - L.score_ws, cuda_stream);
+  if (st != CURDKV_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  StepArgs sa;
+  sa.append.cache = view_of(cache);
+  sa.append.K_new = KvView{static_cast<const __nv_bfloat16*>(K_new), d.k_stride_b, d.k_stride_h, d.k_stride_n};
+  sa.append.V_new = KvView{static_cast<const __nv_bfloat16*>(V_new), d.v_stride_b, d.v_stride_h, d.v_stride_n};
+  sa.append.raw_new = raw_new;
+  sa.append.t_new = d.seqlens;
+  sa.append.heads = d.kv_heads;
+  sa.append.t = d.n_max;
+  sa.append.d = d.d;
+  sa.append.status = reinterpret_cast<uint32_t*>(ws + L.score_ws);
+  sa.budget = budget;
+  sa.num_sink = num_sink;
+  sa.window = window;
+  sa.stage_quads = (int)(stage_bytes / sizeof(uint4));
+  sa.list_cap = list_cap;
+  sa.idx = reinterpret_cast<int32_t*>(ws + L.idx);
+  sa.counts = reinterpret_cast<int32_t*>(ws + L.counts);
+  const size_t smem = stage_bytes + (size_t)list_cap * 8;
+  if (cudaFuncSetAttribute(cache_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kSelStageBytes + kSelListBytes) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  cache_step_kernel<<<(unsigned)(P * (chunks + 1)), 256, smem, stream>>>(sa);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
+  if (cudaFuncSetAttribute(cache_fill_holes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           200 * 1024) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  cache_fill_holes_kernel<<<(unsigned)P, 256, (size_t)cache->capacity, stream>>>(
+      sa.append.cache, sa.idx, budget, sa.counts, d.kv_heads, d.d, reinterpret_cast<int32_t*>(ws + L.holes),
+      sa.append.status, 1, d.seqlens, d.n_max);
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
   return CURDKV_OK;

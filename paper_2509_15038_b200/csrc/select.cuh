@@ -668,7 +668,7 @@ __device__ __forceinline__ void select_fixed_row(RowKeys keys, const ForcedSet& 
 // (0: rows are read from global memory) followed by one candidate list of list_cap entries.
 // With norm.tile_sums the kernel first finishes Alg. 1 line 6 for its row (head sum, division on the
 // way into the staged keys) and `scores` is written.
-__global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
+static __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
     int budget, const int32_t* __restrict__ head_budgets, int num_sink, int window, int stage_quads,
     int list_cap, int32_t* __restrict__ idx, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,

@@ -76,10 +76,13 @@ def _whiten_segments(batch, heads, n, r=32):
 
 
 def test_whitened_segment_count_follows_the_cost_model():
-    """Segments per head minimise ceil(P s / 148) x (tiles per item + 10) over s (host logic only):
+    """Segments per head minimise ceil(P s / SMs) x (tiles per item + 10) over s (host logic only;
+    without a device the library plans for a B200's 148 SMs, which is also what a B200 reports):
     the three bench shapes, and a single long head, which must be cut up to feed all SMs."""
+    sms = 148
+
     def model(P, tiles):
-        cost = lambda s: -(-(P * s) // 148) * (-(-tiles // s) + 10)
+        cost = lambda s: -(-(P * s) // sms) * (-(-tiles // s) + 10)
         return min(range(1, min(tiles, 1024) + 1), key=lambda s: (cost(s), s))
     for batch, heads, n in [(32, 8, 8192), (128, 8, 32768), (32, 8, 131072), (1, 1, 131072), (1, 2, 1000)]:
         tiles = -(-n // 128)

@@ -176,6 +176,108 @@ def test_decode_in_place_keeps_the_same_rows(k, s, w):
             np.testing.assert_allclose(raw[b, h, :c][order][gi], ref.raw[b][h][ri], rtol=1e-3)
 
 
+def _cache_state(cache):
+    """Everything a cache holds, as host arrays cut to the rows in use."""
+    cnt = cache.count.cpu().numpy()
+    out = {"count": cnt, "total": cache.total.cpu().numpy()}
+    for name in ("K", "V"):
+        bits = synth.to_u16(getattr(cache, name))
+        out[name] = [bits[b, :, : cnt[b]] for b in range(len(cnt))]
+    for name in ("raw", "pos"):
+        arr = getattr(cache, name).cpu().numpy()
+        out[name] = [arr[b, :, : cnt[b]] for b in range(len(cnt))]
+    return out
+
+
+@pytest.mark.parametrize("k,s,w", [(64, 4, 0), (64, 0, 16), (100, 4, 8)])
+def test_decode_step_call_equals_append_then_in_place_compression(k, s, w):
+    """curdkv_cache_step (new rows copied and heads selected in one launch) leaves exactly the cache
+    that curdkv_cache_append + curdkv_cache_compress_inplace leave, step after step, with full and
+    with ragged blocks of new rows; and the kept rows are the oracle's, up to the tie band."""
+    B, H, d, r, t = 3, 2, 128, 32, 48
+    steps = 9
+    K, V = _history(B, H, steps * t, d, seed=41)
+    G = synth.make_G(d, r, seed=0)
+    Gd = torch.as_tensor(G, device=DEV)
+    rng = np.random.default_rng(k + s)
+    t_news = [None] * 3 + [rng.integers(0, t + 1, size=B).astype(np.int32) for _ in range(steps - 3)]
+    capacity = k + t
+    one = cur.DeviceCache(B, H, capacity, d, DEV)
+    two = cur.DeviceCache(B, H, capacity, d, DEV)
+    ws1 = cur.cache_workspace(B, H, t, capacity, k, DEV)
+    ws2 = cur.cache_workspace(B, H, t, capacity, k, DEV)
+    ref = dec.CacheOracle(B, H, d)
+    hist = _History(B, H)
+    Ku, Vu = synth.to_u16(K), synth.to_u16(V)
+    for i, tn in enumerate(t_news):
+        Kb, Vb = K[:, :, i * t:(i + 1) * t], V[:, :, i * t:(i + 1) * t]
+        tnd = None if tn is None else torch.as_tensor(tn, device=DEV)
+        cur.curdkv_cache_step(one, Kb, Vb, Gd, k, ws1, num_sink=s, window=w, t_new=tnd)
+        cur.curdkv_cache_append(two, Kb, Vb, Gd, ws2, t_new=tnd)
+        cur.curdkv_cache_compress_inplace(two, k, ws2, num_sink=s, window=w)
+        assert cur.curdkv_device_status(ws1) == 0 and cur.curdkv_device_status(ws2) == 0
+        a, b_ = _cache_state(one), _cache_state(two)
+        for name in ("count", "total"):
+            np.testing.assert_array_equal(a[name], b_[name], err_msg=f"step {i}: {name}")
+        for name in ("K", "V", "raw", "pos"):
+            for x, y in zip(a[name], b_[name]):
+                np.testing.assert_array_equal(x, y, err_msg=f"step {i}: {name}")
+        ref.append(Ku[:, :, i * t:(i + 1) * t], Vu[:, :, i * t:(i + 1) * t], G, tn)
+        hist.add(Ku[:, :, i * t:(i + 1) * t], Vu[:, :, i * t:(i + 1) * t], G, tn)
+        ref.compress(k, s, w)
+    st = _cache_state(one)
+    for b in range(B):
+        for h in range(H):
+            got = st["pos"][b][h]
+            assert len(got) == len(ref.pos[b][h])
+            _assert_kept_within_band(got, ref.pos[b][h], hist.raw[b][h], s, w, f"step call b={b} h={h}")
+            order = np.argsort(got)
+            both, gi, ri = np.intersect1d(got[order], ref.pos[b][h], return_indices=True)
+            np.testing.assert_array_equal(st["K"][b][h][order][gi], ref.K[b][h][ri])
+            np.testing.assert_array_equal(st["V"][b][h][order][gi], ref.V[b][h][ri])
+            np.testing.assert_allclose(st["raw"][b][h][order][gi], ref.raw[b][h][ri], rtol=1e-3)
+
+
+def test_ordered_compression_of_a_cache_left_unordered():
+    """append, in-place compression (which gives up the row order), append, then the ORDERED
+    compression: sinks and window are found by position, so the result is the oracle's."""
+    B, H, d, r = 2, 2, 128, 32
+    k, s, w = 48, 4, 8
+    K, V = _history(B, H, 200, d, seed=43)
+    G = synth.make_G(d, r, seed=0)
+    Gd = torch.as_tensor(G, device=DEV)
+    Ku, Vu = synth.to_u16(K), synth.to_u16(V)
+    capacity = 160
+    a, b_ = cur.DeviceCache(B, H, capacity, d, DEV), cur.DeviceCache(B, H, capacity, d, DEV)
+    ws = cur.cache_workspace(B, H, 100, capacity, k, DEV)
+    ref = dec.CacheOracle(B, H, d)
+    hist = _History(B, H)
+    hist.add(Ku, Vu, G)
+    cur.curdkv_cache_append(a, K[:, :, :100], V[:, :, :100], Gd, ws)
+    ref.append(Ku[:, :, :100], Vu[:, :, :100], G)
+    cur.curdkv_cache_compress_inplace(a, k, ws, num_sink=s, window=w)
+    ref.compress(k, s, w)
+    pos_now = a.pos.cpu().numpy()[:, :, :k]
+    assert np.any(np.diff(pos_now, axis=-1) < 0), "the in-place form is expected to leave rows unordered"
+    cur.curdkv_cache_append(a, K[:, :, 100:], V[:, :, 100:], Gd, ws)
+    ref.append(Ku[:, :, 100:], Vu[:, :, 100:], G)
+    cur.curdkv_cache_compress(a, b_, k, ws, num_sink=s, window=w)
+    ref.compress(k, s, w)
+    assert cur.curdkv_device_status(ws) == 0
+    st = _cache_state(b_)
+    np.testing.assert_array_equal(st["total"], ref.total)
+    for b in range(B):
+        for h in range(H):
+            got = st["pos"][b][h]
+            want = ref.pos[b][h]
+            assert len(got) == len(want) == k
+            assert set(range(s)) <= set(got.tolist()) and set(range(200 - w, 200)) <= set(got.tolist())
+            _assert_kept_within_band(got, want, hist.raw[b][h], s, w, f"ordered after in place b={b} h={h}")
+            for slot, token in enumerate(got):
+                np.testing.assert_array_equal(st["K"][b][h][slot], Ku[b, h, token])
+                np.testing.assert_array_equal(st["V"][b][h][slot], Vu[b, h, token])
+
+
 def test_decode_overflow_is_flagged_not_written():
     B, H, d = 1, 1, 128
     K, V = _history(B, H, 64, d, seed=23)
