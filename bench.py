@@ -672,9 +672,12 @@ def run_evict(args):
     cdesc = cur.make_desc(Kc, Vc, w.r)
     aws = torch.empty((1 << 20,), dtype=torch.uint8, device=dev)
 
+    split = not args.single_bf16_weights
+
     def step():
-        cur.curdkv_attention_out(Q, K, V, desc, scale=scale, O=O, workspace=aws)
-        cur.curdkv_attention_out(Q, Kc, Vc, cdesc, scale=scale, head_rows=rows, O=Oc, workspace=aws)
+        cur.curdkv_attention_out(Q, K, V, desc, scale=scale, O=O, workspace=aws, weight_split=split)
+        cur.curdkv_attention_out(Q, Kc, Vc, cdesc, scale=scale, head_rows=rows, O=Oc, workspace=aws,
+                                 weight_split=split)
         return cur.curdkv_eviction_loss(O, Oc)
 
     for _ in range(max(args.warmup, 3)):
@@ -698,7 +701,7 @@ def run_evict(args):
                      ("key_norm", dict(score_mode=1, use_projection=0)), ("random", dict(random=True))):
         Kx, Vx, rx = select(**kw)
         cur.curdkv_attention_out(Q, Kx, Vx, cur.make_desc(Kx, Vx, w.r), scale=scale, head_rows=rx, O=Oc,
-                                 workspace=aws)
+                                 workspace=aws, weight_split=split)
         lx, _ = cur.curdkv_eviction_loss(O, Oc)
         rel[name] = float((lx / ref).mean())
     P = LB * H
@@ -721,8 +724,9 @@ def run_evict(args):
         "roofline": {"bound": "tensor", "kernel": "attention_umma_kernel (full + compressed cache)",
                      "achieved": tf, "peak": peak, "peak_kind": peak_kind, "unit": "TFLOP/s",
                      "frac": tf / peak, "traffic": None,
-                     "note": "algorithmic flops = one QK^T and one PV; the kernel issues 1.5x that "
-                             "(PV for the hi and the lo half of the weights)"},
+                     "note": ("algorithmic flops = one QK^T and one PV; the kernel issues 1.5x that "
+                              "(PV for the hi and the lo half of the weights)") if split else
+                             "algorithmic flops = one QK^T and one PV, issued once (single bf16 weights)"},
     }), flush=True)
 
 
@@ -873,6 +877,8 @@ def main():
                     help="skip the other configurations (all_configs) and the three-call comparison")
     ap.add_argument("--dry-run", action="store_true",
                     help="host logic of the multi-rank path only (gloo, no CUDA): for tests on a CPU box")
+    ap.add_argument("--single-bf16-weights", action="store_true",
+                    help="--workload evict: softmax weights as single bf16 values (2e-3 instead of 1e-5 accuracy)")
     ap.add_argument("--decode-mode", choices=["inplace", "ordered"], default="inplace",
                     help="--workload decode: compress inside the cache (unordered) or copy in order")
     ap.add_argument("--whiten", action="store_true",

@@ -292,17 +292,21 @@ curdkv_status curdkv_cache_compress(const curdkv_cache* in, const curdkv_cache* 
  *                keep the evicted rows as zero rows; NULL drops them, which is what a
  *                compressed cache computes
  *   scale        multiplies the logits (the paper writes softmax(QK^T): scale = 1)
+ *   weight_split 1: the softmax weights enter the second product as bf16 pairs (hi + lo),
+ *                so O agrees with an fp64 evaluation to about 1e-5 of its largest entry;
+ *                0: as single bf16 values (a third fewer tensor-core products; O then
+ *                agrees to about 2e-3 of its largest entry, each row of weights still
+ *                sums to exactly the normaliser it is divided by)
  *   O            fp32 [batch][kv_heads][q_rows][128]; a head with no key rows gets 0
  * Online softmax in fp32 (exact up to rounding: no approximation of the maximum's
- * effect); the weights enter the second product as bf16 pairs (hi + lo), so O agrees
- * with an fp64 evaluation to about 1e-5 relative. */
+ * effect). */
 size_t curdkv_attention_workspace_bytes(const curdkv_desc* desc);
 curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stride_b, int64_t q_stride_h,
                                    int64_t q_stride_n, const void* K, const void* V,
                                    const curdkv_desc* desc, const int32_t* head_rows,
                                    const int32_t* head_offsets, int64_t packed_rows,
-                                   const int32_t* extra_zero_keys, float scale, float* O, void* workspace,
-                                   size_t workspace_bytes, void* cuda_stream);
+                                   const int32_t* extra_zero_keys, float scale, int32_t weight_split,
+                                   float* O, void* workspace, size_t workspace_bytes, void* cuda_stream);
 /* loss[p] = ||O_full[p] - O_compressed[p]||_F and (if not NULL) ref_norm[p] = ||O_full[p]||_F
  * over elems_per_problem floats per problem; fixed summation order. */
 curdkv_status curdkv_eviction_loss(const float* O_full, const float* O_compressed, int32_t problems,

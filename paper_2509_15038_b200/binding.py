@@ -120,7 +120,7 @@ def load():
     lib.curdkv_attention_workspace_bytes.argtypes = [dp]
     lib.curdkv_attention_out.restype = ctypes.c_int
     lib.curdkv_attention_out.argtypes = [vp, i32, i64, i64, i64, vp, vp, dp, vp, vp, i64, vp,
-                                         ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
+                                         ctypes.c_float, i32, vp, vp, ctypes.c_size_t, vp]
     lib.curdkv_eviction_loss.restype = ctypes.c_int
     lib.curdkv_eviction_loss.argtypes = [vp, vp, i32, i64, vp, vp, vp]
     lib.curdkv_selftest_bounded_wait.restype = ctypes.c_int
@@ -415,7 +415,8 @@ def curdkv_cache_step(cache: DeviceCache, K_new, V_new, G, budget: int, workspac
 
 
 def curdkv_attention_out(Q, K, V, desc: Desc, *, scale: float = 1.0, head_rows=None, head_offsets=None,
-                         extra_zero_keys=None, O=None, workspace: Optional[torch.Tensor] = None):
+                         extra_zero_keys=None, O=None, workspace: Optional[torch.Tensor] = None,
+                         weight_split: bool = True):
     """O = softmax(scale Q K^T) V per (b, h).  Q bf16 ``[B, Hkv, m, 128]``; K, V as described by
     ``desc``, or packed ``[rows, 128]`` arrays when ``head_offsets`` is given."""
     if Q.dtype != torch.bfloat16 or Q.dim() != 4 or Q.stride(3) != 1:
@@ -429,8 +430,8 @@ def curdkv_attention_out(Q, K, V, desc: Desc, *, scale: float = 1.0, head_rows=N
     packed_rows = K.shape[0] if head_offsets is not None else 0
     code = load().curdkv_attention_out(_ptr(Q), m, Q.stride(0), Q.stride(1), Q.stride(2), _ptr(K), _ptr(V),
                                        ctypes.byref(desc), _ptr(head_rows), _ptr(head_offsets),
-                                       packed_rows, _ptr(extra_zero_keys), float(scale), _ptr(O),
-                                       _ptr(workspace), workspace.numel(), _stream())
+                                       packed_rows, _ptr(extra_zero_keys), float(scale), int(weight_split),
+                                       _ptr(O), _ptr(workspace), workspace.numel(), _stream())
     _check(code, "curdkv_attention_out")
     return O, workspace
 

@@ -34,6 +34,7 @@ struct AttnArgs {
   const int32_t* extra_zero; // [problems] further keys with logit 0 and value 0 (Lemma 1), or nullptr
   int heads, m, packed;      // query rows per problem; packed: K, V are one [rows, d] array
   float scale;
+  int split;                 // 1: weights as bf16 pairs hi + lo; 0: single bf16 weights
   float* O;                  // [problems][m][128]
   uint32_t* status;
   unsigned long long wait_ns = kWaitLimitNs;   // limit of each pipeline wait
@@ -139,6 +140,10 @@ __device__ __forceinline__ void split_bf16x2(float w0, float w1, uint32_t& hi, u
   lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
+// SPLIT: the weights enter P V as bf16 pairs P_hi + P_lo (two products per tile, weights exact to
+// 2^-17); without it as single bf16 values (one product, weights exact to 2^-9, and the row sums are
+// taken over the rounded weights so that every row of P still sums to the normaliser it is divided by).
+template <bool SPLIT>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v, const AttnArgs a) {
@@ -281,7 +286,7 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         if (!(ok = mbar_wait(p_ready_bar(buf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status, a.wait_ns))) break;
         tc_fence_after();
         const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
-        for (int part = 0; part < 2; ++part) {             // P_hi, then P_lo
+        for (int part = 0; part < (SPLIT ? 2 : 1); ++part) {   // P_hi, then P_lo
           const uint32_t p_tmem = tmem_base + buf * 128u + part * 64u;
           for (int g = 0; g < groups; ++g)                 // 16 keys per MMA: 8 columns of P
             tc_mma_bf16_ts(tmem_base + 256u + buf * 128u, p_tmem + 8u * g,
@@ -377,18 +382,23 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             float x0, x1;
             unpack2(fma2(pack2(v[c], v[c + 1]), sc2, ntop2), x0, x1);
             const uint64_t w2 = pack2(fast_exp2(x0), fast_exp2(x1));
-            part[e & 3] = add2(part[e & 3], w2);           // equals the bf16 pairs to 2^-17
             float w0, w1;
             unpack2(w2, w0, w1);
             const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
             hi[e] = *reinterpret_cast<const uint32_t*>(&h);
-            float r0, r1;
-            unpack2(sub2(w2, pack2(__uint_as_float(hi[e] << 16), __uint_as_float(hi[e] & 0xffff0000u))), r0, r1);
-            const __nv_bfloat162 q = __floats2bfloat162_rn(r0, r1);
-            lo[e] = *reinterpret_cast<const uint32_t*>(&q);
+            const uint64_t h2 = pack2(__uint_as_float(hi[e] << 16), __uint_as_float(hi[e] & 0xffff0000u));
+            if (SPLIT) {
+              part[e & 3] = add2(part[e & 3], w2);         // equals the bf16 pairs to 2^-17
+              float r0, r1;
+              unpack2(sub2(w2, h2), r0, r1);
+              const __nv_bfloat162 q = __floats2bfloat162_rn(r0, r1);
+              lo[e] = *reinterpret_cast<const uint32_t*>(&q);
+            } else {
+              part[e & 3] = add2(part[e & 3], h2);         // the weights the product really uses
+            }
           }
           tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
-          tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
+          if (SPLIT) tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
         }
         float p0, p1;
         unpack2(add2(add2(part[0], part[1]), add2(part[2], part[3])), p0, p1);
@@ -403,11 +413,11 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             const int c = c0 + 2 * e;
             const float w0 = c < valid ? fast_exp2(fmaf(v[c], sc, -top)) : 0.f;
             const float w1 = c + 1 < valid ? fast_exp2(fmaf(v[c + 1], sc, -top)) : 0.f;
-            sum += w0 + w1;
             split_bf16x2(w0, w1, hi[e], lo[e]);
+            sum += SPLIT ? w0 + w1 : __uint_as_float(hi[e] << 16) + __uint_as_float(hi[e] & 0xffff0000u);
           }
           tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
-          tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
+          if (SPLIT) tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
         }
       }
       tmem_st_wait();

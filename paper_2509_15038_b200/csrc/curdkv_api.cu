@@ -782,9 +782,10 @@ curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stri
                                    int64_t q_stride_n, const void* K, const void* V,
                                    const curdkv_desc* desc, const int32_t* head_rows,
                                    const int32_t* head_offsets, int64_t packed_rows,
-                                   const int32_t* extra_zero_keys, float scale, float* O, void* workspace,
-                                   size_t workspace_bytes, void* cuda_stream) {
+                                   const int32_t* extra_zero_keys, float scale, int32_t weight_split,
+                                   float* O, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   curdkv_status st = check_desc(desc);
+  if (st == CURDKV_OK && weight_split != 0 && weight_split != 1) st = CURDKV_ERR_INVALID_ARG;
   if (st != CURDKV_OK) return st;
   if (Q == nullptr || K == nullptr || V == nullptr || O == nullptr || workspace == nullptr)
     return CURDKV_ERR_INVALID_ARG;
@@ -836,13 +837,18 @@ curdkv_status curdkv_attention_out(const void* Q, int32_t q_rows, int64_t q_stri
   a.m = q_rows;
   a.packed = packed ? 1 : 0;
   a.scale = scale;
+  a.split = weight_split;
   a.O = O;
   a.status = static_cast<uint32_t*>(workspace);
-  if (cudaFuncSetAttribute(umma::attention_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           umma::kAttnDynamic) != cudaSuccess)
+  auto launch = [&](auto kernel) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kAttnDynamic) !=
+        cudaSuccess)
+      return false;
+    kernel<<<(unsigned)(P * q_blocks), umma::kAttnThreads, umma::kAttnDynamic, stream>>>(mq, mk, mv, a);
+    return true;
+  };
+  if (!(weight_split ? launch(umma::attention_umma_kernel<true>) : launch(umma::attention_umma_kernel<false>)))
     return CURDKV_ERR_CUDA;
-  umma::attention_umma_kernel<<<(unsigned)(P * q_blocks), umma::kAttnThreads, umma::kAttnDynamic, stream>>>(
-      mq, mk, mv, a);
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }
