@@ -13,16 +13,23 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def run_path(w):
+def run_path(w, three_calls=False):
+    """The path as bench.py times it: one curdkv_compress call (three_calls: the separate calls)."""
     K, V, seqlens = synth.make_kv(w, DEV)
     G = synth.make_G(w.d, w.r, seed=0)
+    Gd = torch.as_tensor(G, device=DEV)
     sl = None if seqlens is None else torch.as_tensor(seqlens, device=DEV)
     desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads, seqlens=sl)
     ws = cur.alloc_workspace(desc, w.budget, w.adaptive)
-    scores, sums = cur.curdkv_score(K, V, torch.as_tensor(G, device=DEV), desc, ws)
-    idx, cnt, off = cur.curdkv_select(scores, desc, w.budget, num_sink=w.num_sink, window=w.window,
-                                      adaptive=w.adaptive, alpha=w.alpha, workspace=ws)
-    Ko, Vo = cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=w.adaptive, workspace=ws)
+    if three_calls:
+        scores, sums = cur.curdkv_score(K, V, Gd, desc, ws)
+        idx, cnt, off = cur.curdkv_select(scores, desc, w.budget, num_sink=w.num_sink, window=w.window,
+                                          adaptive=w.adaptive, alpha=w.alpha, workspace=ws)
+        Ko, Vo = cur.curdkv_compact(K, V, desc, idx, cnt, off, packed=w.adaptive, workspace=ws)
+    else:
+        scores, sums, idx, cnt, off, Ko, Vo = cur.curdkv_compress(
+            K, V, Gd, desc, w.budget, ws, num_sink=w.num_sink, window=w.window, adaptive=w.adaptive,
+            alpha=w.alpha)
     assert cur.curdkv_device_status(ws) == 0
     return K, V, G, seqlens, scores, sums, idx, cnt, off, Ko, Vo
 
@@ -75,6 +82,23 @@ def check_sampled_problems(w, K, V, G, seqlens, scores, idx, cnt, samples):
                                    w.budget, w.num_sink, w.window, seqlens=sl)
         np.testing.assert_array_equal(idx[lb, h].cpu().numpy(), eidx[0, 0])
     return worst
+
+
+def test_cfg3_full_size_three_calls_equal_the_single_call():
+    """At the headline size the single call (fused score + select kernel) and the three separate
+    calls give the same bits; run twice to catch anything that depends on timing."""
+    w = synth.CONFIGS["cfg3"]
+    a = run_path(w, three_calls=True)
+    want = [t.clone() for t in a[4:8]] + [a[9][::16].clone(), a[10][::16].clone()]
+    del a
+    torch.cuda.empty_cache()
+    for _ in range(2):
+        b = run_path(w)
+        got = list(b[4:8]) + [b[9][::16], b[10][::16]]
+        for name, x, y in zip(("scores", "head_sums", "idx", "head_counts", "K_out", "V_out"), got, want):
+            assert torch.equal(x, y), name
+        del b, got
+        torch.cuda.empty_cache()
 
 
 def test_cfg3_full_size():
