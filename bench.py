@@ -605,9 +605,11 @@ def run_decode(args):
     ms = t0.elapsed_time(t1) / args.steps
     P = LB * H
     rows = P * (k + t)                       # rows the compression looks at per step
-    # new rows read and stored, their scores; held scores read; then either every survivor read and
-    # written (ordered) or at most `chunk` moved rows per head read and written (in place)
-    counted = P * (t * 512 * 2 + (k + t) * 4 + (t if inplace else k) * 512 * 2)
+    # What a step has to move.  In place: the new rows read once for their scores, the scores of all
+    # rows looked at, and each surviving new row stored once (counted as all `chunk` of them: an upper
+    # bound; evicted new rows are never stored).  Ordered: new rows read and stored, scores, and every
+    # survivor read and written into the other cache.
+    counted = P * ((t * 512 + (k + t) * 4 + t * 512) if inplace else (t * 512 * 2 + (k + t) * 4 + k * 512 * 2))
     peak, peak_kind = measured_peak()
     gbs = counted / (ms * 1e-3) / 1e9
     print(json.dumps({
@@ -622,9 +624,11 @@ def run_decode(args):
                    "l2": "caches (%.1f GB) exceed the 126 MB L2" % (2 * 2 * P * cap * d * 2 / 1e9)},
         "gb_per_s": gbs, "counted_bytes_per_step": counted,
         "clocks": clocks, "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "whole step (append + select + gather)", "achieved": gbs,
-                     "peak": peak, "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s",
-                     "frac": gbs / peak, "traffic": None},
+        "roofline": {"bound": "hbm", "kernel": "whole step (score the new rows, select, place the survivors)",
+                     "achieved": gbs, "peak": peak, "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s",
+                     "frac": gbs / peak, "traffic": None,
+                     "note": "algorithmic bytes: every new row read once and stored at most once; the kernels "
+                             "read the surviving new rows a second time when they place them"},
     }), flush=True)
 
 

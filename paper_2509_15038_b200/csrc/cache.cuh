@@ -249,79 +249,61 @@ __global__ void __launch_bounds__(256) cache_fill_holes_kernel(const CacheView c
   }
 }
 
-// ---- one generation step: append the new rows AND select in place, in one launch -------------
-// The selection of a head only needs the scores and positions of its rows, not the rows
-// themselves, so it runs beside the copies of the new rows: of every (chunks + 1) consecutive CTAs
-// the first selects for one head (keys staged in shared memory from the held rows' scores and
-// positions and from the new rows' fresh scores; it also files the new rows' scores and
-// positions in the cache), the others copy 32 new rows of that head each.  The counters are
-// only read here; cache_fill_holes_kernel sets them afterwards.
+// ---- one generation step: append the new rows AND compress in place, in one launch ----------
+// One CTA per head.  The selection only needs scores and positions, so it runs first, over the
+// held rows' scores and positions and the new rows' fresh scores (keys staged in shared memory;
+// forced rows, found by position, carry the top key).  Only then are rows moved, and each at most
+// once: a surviving new row goes straight from the caller's block into its final slot (its own,
+// or a hole an evicted row leaves), a surviving old row beyond the new row count into a hole;
+// evicted new rows are never copied at all.  With s = slot of a row after a plain append (held
+// rows 0 .. held-1, new row i at held + i) the result is the cache curdkv_cache_append +
+// curdkv_cache_compress_inplace leave.  The last CTA of a sequence sets its counters (every CTA of
+// the sequence has read them by then: tickets, zero on entry).
 struct StepArgs {
   AppendArgs append;
   int budget, num_sink, window;
   int stage_quads, list_cap;       // shared-memory copy of a head's keys, candidate list
   int32_t* idx;                    // [batch*heads][budget]
   int32_t* counts;                 // [batch*heads]
+  int32_t* tickets;                // [batch], zero on entry
 };
 
 __global__ void __launch_bounds__(256) cache_step_kernel(const StepArgs s) {
   __shared__ SelectSmem sm;
+  __shared__ int s_first_mover, s_first_new, s_base, s_warp_tot[8];
   extern __shared__ uint4 step_keys[];                     // stage_quads quads, then the list
   const AppendArgs& a = s.append;
-  const int chunks_per_head = (a.t + kAppendRowsPerCta - 1) / kAppendRowsPerCta;
-  const int p = blockIdx.x / (chunks_per_head + 1), role = blockIdx.x % (chunks_per_head + 1);
-  const int b = p / a.heads, h = p % a.heads;
+  const int p = blockIdx.x, b = p / a.heads, h = p % a.heads;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cap = a.cache.capacity;
   int tb = a.t_new != nullptr ? a.t_new[b] : a.t;
   tb = tb < 0 ? 0 : (tb > a.t ? a.t : tb);
   int held = a.cache.count[b];
-  if (held < 0 || held > a.cache.capacity) {               // counters the caller never set up
-    if (threadIdx.x == 0 && role == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
-    held = held < 0 ? 0 : a.cache.capacity;
+  if (held < 0 || held > cap) {                            // counters the caller never set up
+    if (tid == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+    held = held < 0 ? 0 : cap;
   }
   const int first_pos = a.cache.total[b], offered = tb;
-  if (tb > a.cache.capacity - held) {
-    if (threadIdx.x == 0 && role == 0) flag_status(a.status, CURDKV_DEV_CACHE_FULL);
-    tb = a.cache.capacity - held;
+  if (tb > cap - held) {
+    if (tid == 0) flag_status(a.status, CURDKV_DEV_CACHE_FULL);
+    tb = cap - held;
   }
-  if (role > 0) {
-    // ------------------------------------------------------------ copy 32 new rows
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
-    const KvView& T = half ? a.V_new : a.K_new;
-    const __nv_bfloat16* src = T.base + b * T.stride_b + h * T.stride_h;
-    __nv_bfloat16* dst = (half ? a.cache.V : a.cache.K) + ((size_t)p * a.cache.capacity + held) * a.d;
-    const int chunks = a.d >> 3;
-    const int row0 = (role - 1) * kAppendRowsPerCta + warp;
-    for (int c = l16; c < chunks; c += 16) {
-      uint4 v[kAppendRowsPerCta / kAppendWarps];
-#pragma unroll
-      for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
-        const int i = row0 + j * kAppendWarps;
-        if (i < tb) v[j] = __ldg(reinterpret_cast<const uint4*>(src + i * T.stride_n) + c);
-      }
-#pragma unroll
-      for (int j = 0; j < kAppendRowsPerCta / kAppendWarps; ++j) {
-        const int i = row0 + j * kAppendWarps;
-        if (i < tb) reinterpret_cast<uint4*>(dst + (size_t)i * a.d)[c] = v[j];
-      }
-    }
-    return;
-  }
-  // -------------------------------------------------------------- select for head p (Alg. 1 lines 7-9)
+  // -------------------------------------------------------------- select (Alg. 1 lines 7-9)
   using G = WholeCta;
   const int n = held + tb;                                 // rows the head holds after the append
   const int k_eff = min(s.budget, n);
   const int recent = first_pos + offered - s.window;       // positions from here on are the window
-  float* raw_row = a.cache.raw + (size_t)p * a.cache.capacity;
-  int32_t* pos_row = a.cache.pos + (size_t)p * a.cache.capacity;
+  float* raw_row = a.cache.raw + (size_t)p * cap;
+  int32_t* pos_row = a.cache.pos + (size_t)p * cap;
   const float* raw_new = a.raw_new + (size_t)p * a.t;
   clear_hist<G>(sm.hist);
-  if (threadIdx.x == 0) sm.list_count[0] = 0;
+  if (tid == 0) sm.list_count[0] = 0;
   __syncthreads();
   {
     DigitRun run;
     uint32_t* keys32 = reinterpret_cast<uint32_t*>(step_keys);
     const int padded = ((n + 3) >> 2) << 2;
-    for (int j = threadIdx.x; j < padded; j += 256) {
+    for (int j = tid; j < padded; j += 256) {
       uint32_t key = 0u;                                   // beyond the rows held: never kept
       if (j < n) {
         float raw;
@@ -346,9 +328,99 @@ __global__ void __launch_bounds__(256) cache_step_kernel(const StepArgs s) {
   const ForcedSet F = forced_set(n, k_eff, 0, 0);          // forced rows carry the top key already
   RowKeys keys{nullptr, step_keys, n, 0, n, true, false};
   const KeyList list{reinterpret_cast<uint2*>(step_keys + s.stage_quads), &sm.list_count[0], (uint32_t)s.list_cap};
-  select_fixed_row<G>(keys, F, k_eff, s.budget, step_keys, s.stage_quads, list, true,
-                      s.idx + (size_t)p * s.budget, sm);
-  if (threadIdx.x == 0) s.counts[p] = k_eff;
+  int32_t* ix = s.idx + (size_t)p * s.budget;
+  select_fixed_row<G>(keys, F, k_eff, s.budget, step_keys, s.stage_quads, list, true, ix, sm);
+  if (tid == 0) s.counts[p] = k_eff;
+
+  // -------------------------------------------------------------- place the survivors (Alg. 1 line 10)
+  // ix is ascending: [0, first_new) old rows that stay, [first_new, first_mover) new rows whose
+  // own slot lies below k_eff, [first_mover, k_eff) movers (slot >= k_eff) that go into the holes.
+  // The staged keys are done with: their space takes the slot flags and the list of holes.
+  unsigned char* slot_kept = reinterpret_cast<unsigned char*>(step_keys);
+  int32_t* holes = reinterpret_cast<int32_t*>(slot_kept + ((cap + 15) & ~15));
+  __syncthreads();                                         // ix (global) and the end of the key sweeps
+  if (tid == 0) {
+    int lo = 0, hi = k_eff;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (ix[mid] < k_eff) lo = mid + 1; else hi = mid; }
+    s_first_mover = lo;
+    lo = 0, hi = k_eff;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (ix[mid] < held) lo = mid + 1; else hi = mid; }
+    s_first_new = lo;
+    s_base = 0;
+  }
+  for (int t = tid; t < k_eff; t += 256) slot_kept[t] = 0;
+  __syncthreads();
+  const int first_mover = s_first_mover, first_new = min(s_first_new, first_mover);
+  const int movers = k_eff - first_mover;
+  for (int t = tid; t < first_mover; t += 256) slot_kept[ix[t]] = 1;
+  __syncthreads();
+  for (int s0 = 0; s0 < k_eff; s0 += 256) {                // holes in ascending slot order
+    const int sl = s0 + tid;
+    const bool hole = sl < k_eff && slot_kept[sl] == 0;
+    const uint32_t bal = __ballot_sync(0xffffffffu, hole);
+    if (lane == 0) s_warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int before = s_base;
+    for (int w = 0; w < warp; ++w) before += s_warp_tot[w];
+    if (hole) holes[before + __popc(bal & ((1u << lane) - 1u))] = sl;
+    __syncthreads();
+    if (tid == 0) {
+      int tot = 0;
+      for (int w = 0; w < 8; ++w) tot += s_warp_tot[w];
+      s_base += tot;
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && s_base != movers) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+  const int moves = min(s_base, movers);
+  // jobs: natural-slot new rows first, then mover i -> hole i.  A half-warp per tensor row (K in
+  // lanes 0-15, V in lanes 16-31), four rows per warp in flight; sources and destinations are
+  // disjoint (sources: slots >= k_eff or the caller's block), so the order is free.
+  const int half = lane >> 4, l16 = lane & 15, chunks = a.d >> 3;
+  const int jobs = (first_mover - first_new) + moves;
+  __nv_bfloat16* cache_rows = (half ? a.cache.V : a.cache.K) + (size_t)p * cap * a.d;
+  const KvView& T = half ? a.V_new : a.K_new;
+  const __nv_bfloat16* new_rows = T.base + b * T.stride_b + h * T.stride_h;
+  for (int j0 = warp; j0 < jobs; j0 += 32) {
+    const __nv_bfloat16* src[4];
+    int dst[4], from[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int j = min(j0 + 8 * q, jobs - 1);
+      if (j < first_mover - first_new) {                   // new row, own slot
+        from[q] = dst[q] = ix[first_new + j];
+      } else {
+        from[q] = ix[first_mover + (j - (first_mover - first_new))];
+        dst[q] = holes[j - (first_mover - first_new)];
+      }
+      src[q] = from[q] < held ? cache_rows + (size_t)from[q] * a.d
+                              : new_rows + (int64_t)(from[q] - held) * T.stride_n;
+    }
+    for (int c = l16; c < chunks; c += 16) {
+      uint4 v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const uint4*>(src[q] + c * 8);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (j0 + 8 * q < jobs) reinterpret_cast<uint4*>(cache_rows + (size_t)dst[q] * a.d)[c] = v[q];
+    }
+    if (lane < 4 && j0 + 8 * lane < jobs && from[lane] != dst[lane]) {   // a mover's score and position
+      int f = from[0], t2 = dst[0];
+#pragma unroll
+      for (int q = 1; q < 4; ++q)
+        if (lane == q) { f = from[q]; t2 = dst[q]; }
+      raw_row[t2] = raw_row[f];
+      pos_row[t2] = pos_row[f];
+    }
+  }
+  // -------------------------------------------------------------- counters, by the sequence's last CTA
+  __threadfence();
+  __syncthreads();
+  if (tid == 0 && atomicAdd(s.tickets + b, 1) == a.heads - 1) {
+    a.cache.count[b] = k_eff;
+    a.cache.total[b] = first_pos + offered;
+    s.tickets[b] = 0;
+  }
 }
 
 }  // namespace curdkv

@@ -13,7 +13,7 @@ using namespace curdkv;
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct CacheWorkspace {     // byte offsets from the workspace base
-  size_t score_ws, raw_new, sums, idx, counts, keyed, holes, total;
+  size_t score_ws, raw_new, sums, idx, counts, keyed, holes, tickets, total;
 };
 
 bool layout(int32_t batch, int32_t heads, int32_t t_max, int32_t capacity, int32_t budget,
@@ -38,6 +38,7 @@ bool layout(int32_t batch, int32_t heads, int32_t t_max, int32_t capacity, int32
   L->counts = take(P * 4);
   L->keyed = take(P * (size_t)capacity * 4);    // in-place compression only
   L->holes = take(P * (size_t)capacity * 4);
+  L->tickets = take((size_t)batch * 4);         // curdkv_cache_step only
   L->total = o;
   return true;
 }
@@ -227,8 +228,7 @@ curdkv_status curdkv_cache_step(const curdkv_cache* cache, const void* K_new, co
   // the selection CTAs keep a head's keys and its candidate list in shared memory
   const int list_cap = cache->capacity <= 4096 ? kSelListCap / 4 : (cache->capacity <= 16384 ? kSelListCap / 2 : kSelListCap);
   const size_t stage_bytes = (((size_t)cache->capacity + 3) / 4) * sizeof(uint4);
-  const int64_t chunks = (desc_new->n_max + kAppendRowsPerCta - 1) / kAppendRowsPerCta;
-  if (stage_bytes > (size_t)kSelStageBytes || desc_new->n_max < 1 || P < 1 || P * (chunks + 1) > 0x7fffffffLL ||
+  if (stage_bytes > (size_t)kSelStageBytes || desc_new->n_max < 1 || P < 1 || P > 0x7fffffffLL ||
       desc_new->d % 8 != 0) {
     // shapes the one-launch form does not cover: the two calls it stands for
     curdkv_status st = curdkv_cache_append(cache, K_new, V_new, G, g_per_head, desc_new, workspace,
@@ -265,19 +265,16 @@ curdkv_status curdkv_cache_step(const curdkv_cache* cache, const void* K_new, co
   sa.list_cap = list_cap;
   sa.idx = reinterpret_cast<int32_t*>(ws + L.idx);
   sa.counts = reinterpret_cast<int32_t*>(ws + L.counts);
-  const size_t smem = stage_bytes + (size_t)list_cap * 8;
+  sa.tickets = reinterpret_cast<int32_t*>(ws + L.tickets);
+  if (cudaMemsetAsync(sa.tickets, 0, (size_t)d.batch * sizeof(int32_t), stream) != cudaSuccess)
+    return CURDKV_ERR_CUDA;
+  // after the selection the staged keys' space takes a flag per slot and the list of holes
+  const size_t place_bytes = (((size_t)cache->capacity + 15) & ~size_t(15)) + ((size_t)cache->capacity / 2 + 1) * 4;
+  const size_t smem = (stage_bytes > place_bytes ? stage_bytes : place_bytes) + (size_t)list_cap * 8;
   if (cudaFuncSetAttribute(cache_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kSelStageBytes + kSelListBytes) != cudaSuccess)
     return CURDKV_ERR_CUDA;
-  cache_step_kernel<<<(unsigned)(P * (chunks + 1)), 256, smem, stream>>>(sa);
-  count_launch();
-  if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
-  if (cudaFuncSetAttribute(cache_fill_holes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           200 * 1024) != cudaSuccess)
-    return CURDKV_ERR_CUDA;
-  cache_fill_holes_kernel<<<(unsigned)P, 256, (size_t)cache->capacity, stream>>>(
-      sa.append.cache, sa.idx, budget, sa.counts, d.kv_heads, d.d, reinterpret_cast<int32_t*>(ws + L.holes),
-      sa.append.status, 1, d.seqlens, d.n_max);
+  cache_step_kernel<<<(unsigned)P, 256, smem, stream>>>(sa);
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
