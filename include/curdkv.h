@@ -325,13 +325,14 @@ curdkv_status curdkv_cache_compress_inplace(const curdkv_cache* cache, const cur
                                             int32_t budget, int32_t num_sink, int32_t window,
                                             void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* One generation step in two launches after the scoring of the new rows: what
- * curdkv_cache_append followed by curdkv_cache_compress_inplace does (same arguments, same
- * resulting cache bit for bit, same status flags).  The selection needs only scores and
- * positions, so one kernel copies the new rows into the cache and, beside those copies,
- * selects for every head from the held rows' scores and the new rows' fresh ones; a second
- * kernel moves the survivors into the holes and sets the counters.  Requires budget >= 1 and
- * num_sink + window <= budget; capacities above 36,864 rows run as the two calls. */
+/* One generation step: what curdkv_cache_append followed by curdkv_cache_compress_inplace
+ * does (same arguments, same resulting cache bit for bit, same status flags), in one kernel
+ * after the scoring of the new rows.  The selection needs only scores and positions, so every
+ * head first selects over its held rows' scores and the new rows' fresh ones; only then are
+ * rows moved, each at most once: a surviving new row goes straight from K_new / V_new into its
+ * final slot, a surviving held row beyond the new row count into a hole, and evicted new rows
+ * are never copied.  Requires budget >= 1 and num_sink + window <= budget; capacities above
+ * 36,864 rows run as the two calls. */
 curdkv_status curdkv_cache_step(const curdkv_cache* cache, const void* K_new, const void* V_new,
                                 const float* G, int32_t g_per_head, const curdkv_desc* desc_new,
                                 int32_t budget, int32_t num_sink, int32_t window, void* workspace,
