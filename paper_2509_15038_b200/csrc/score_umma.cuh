@@ -68,6 +68,10 @@ struct Args {
   // Tiles are dealt to the CTAs in chunks of this many consecutive tiles (1: tile t goes to CTA
   // t mod grid).  The fused kernel counts a head's tiles once per chunk instead of once per tile.
   int chunk_tiles = 1;
+  // L2 policy of the K/V tile loads: 1 = evict-first (the tiles are read once), 0 = the default
+  // policy.  Measured: on caches of many GB the default is ~0.5 % faster, on a 1 GB cache
+  // evict-first is (the launcher picks by size).
+  int evict_first = 1;
 };
 
 // The tiles of one CTA in the order every role walks them: chunks first, first + stride, ... of
@@ -465,7 +469,8 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint64_t policy;
-      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      if (a.evict_first) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(policy));
       uint32_t it = 0;
       bool ok = true;
       for (TileWalk w(first, stride, (uint32_t)a.chunk_tiles, total_tiles); ok && w.valid(); w.next()) {
