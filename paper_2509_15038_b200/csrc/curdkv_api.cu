@@ -8,7 +8,7 @@
 #include "compact.cuh"
 #include "score_simt.cuh"
 #include "score_umma.cuh"
-#include "select.cuh"
+#include "select_kernels.cuh"
 #include "whiten_factor.cuh"
 #include "whiten_umma.cuh"
 #include "attn_umma.cuh"
