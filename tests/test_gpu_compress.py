@@ -142,3 +142,37 @@ def test_compress_shapes_that_take_the_three_step_route():
     _both_ways(K, V, None, 120, 4, 16, use_projection=0, what="no projection")
     _both_ways(K, V, G, 120, 4, 16, whiten=1, ridge=1e-4, what="whitened")
     _both_ways(K[:, :, :100], V[:, :, :100], G, 30, 2, 4, what="n_max < 128")
+
+
+def test_compress_replays_from_a_cuda_graph():
+    """The single call on a shape that takes the one-kernel route (a cooperative launch) can be captured
+    once and replayed; the replay reproduces the eager results bit for bit."""
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=76, n_max=1024, budget=200)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=DEV)
+    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads)
+    ws = cur.alloc_workspace(desc, w.budget)
+    out = cur.curdkv_compress(K, V, G, desc, w.budget, ws, num_sink=4, window=32)
+    torch.cuda.synchronize()
+    want = [t.clone() for t in out]
+    names = ("scores", "head_sums", "idx", "head_counts", "head_offsets", "K_out", "V_out")
+    bufs = dict(zip(names, out))
+
+    def step():
+        cur.curdkv_compress(K, V, G, desc, w.budget, ws, num_sink=4, window=32, **bufs)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in out:
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert cur.curdkv_device_status(ws) == 0
+    for name, a, b in zip(names, want, out):
+        assert torch.equal(a, b), name
