@@ -238,6 +238,38 @@ def test_decode_step_call_equals_append_then_in_place_compression(k, s, w):
             np.testing.assert_allclose(st["raw"][b][h][order][gi], ref.raw[b][h][ri], rtol=1e-3)
 
 
+def test_decode_step_call_with_a_cache_that_overflows_and_one_that_is_still_filling():
+    """The step call on the edges: a cache still below its budget (every new row keeps its own slot),
+    a block that does not fit under the capacity (the rows that fit are taken, the flag is raised),
+    and a sequence that brings no rows.  Same cache and same flags as append + in-place compression."""
+    B, H, d, r, t = 3, 2, 128, 32, 40
+    K, V = _history(B, H, 4 * t, d, seed=47)
+    Gd = torch.as_tensor(synth.make_G(d, r, seed=0), device=DEV)
+    for k, capacity in ((100, 140), (60, 70)):              # filling for two steps / overflowing at once
+        one = cur.DeviceCache(B, H, capacity, d, DEV)
+        two = cur.DeviceCache(B, H, capacity, d, DEV)
+        ws1 = cur.cache_workspace(B, H, t, capacity, k, DEV)
+        ws2 = cur.cache_workspace(B, H, t, capacity, k, DEV)
+        saw_full = False
+        for i in range(4):
+            Kb, Vb = K[:, :, i * t:(i + 1) * t], V[:, :, i * t:(i + 1) * t]
+            tn = torch.as_tensor(np.array([t, 0, 17], dtype=np.int32), device=DEV) if i == 2 else None
+            cur.curdkv_cache_step(one, Kb, Vb, Gd, k, ws1, num_sink=2, window=5, t_new=tn)
+            cur.curdkv_cache_append(two, Kb, Vb, Gd, ws2, t_new=tn)
+            f_append = cur.curdkv_device_status(ws2)
+            cur.curdkv_cache_compress_inplace(two, k, ws2, num_sink=2, window=5)
+            f1, f2 = cur.curdkv_device_status(ws1), f_append | cur.curdkv_device_status(ws2)
+            assert f1 == f2, (k, i, f1, f2)
+            saw_full |= bool(f1 & cur.DEV_CACHE_FULL)
+            a, b_ = _cache_state(one), _cache_state(two)
+            for name in ("count", "total"):
+                np.testing.assert_array_equal(a[name], b_[name], err_msg=f"k={k} step {i}: {name}")
+            for name in ("K", "V", "raw", "pos"):
+                for x, y in zip(a[name], b_[name]):
+                    np.testing.assert_array_equal(x, y, err_msg=f"k={k} step {i}: {name}")
+        assert saw_full == (capacity == 70)                 # 40 held + 40 offered > 70; never above 140
+
+
 def test_ordered_compression_of_a_cache_left_unordered():
     """append, in-place compression (which gives up the row order), append, then the ORDERED
     compression: sinks and window are found by position, so the result is the oracle's."""
