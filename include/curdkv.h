@@ -189,10 +189,13 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
  * gathered rows) and the default output layouts (adaptive = 0: idx
  * [batch][kv_heads][budget], K_out / V_out [batch][kv_heads][budget][d]; adaptive = 1:
  * packed).  With a fixed budget, one shared G, projection on, whiten off, d = 128,
- * r <= 32 and n_max >= 128 the scoring kernel also normalises and selects: the CTA
- * that writes the last tile of a head runs Alg. 1 lines 6-9 for that head on extra
- * warps while the stream of K and V goes on, so the selection costs no time of its
- * own.  Other shapes run the three steps in sequence.
+ * r <= 32, n_max >= 128, no per-sequence lengths and at least four heads per SM of the
+ * device, the scoring kernel also normalises and selects: the heads whose last tile has been
+ * written are handed, through one list served by all CTAs, to extra warps that run Alg. 1
+ * lines 6-9 for them while the stream of K and V goes on, so the selection costs almost no
+ * time of its own (a cooperative launch; it can still be captured into a CUDA graph).  Other
+ * shapes run the three steps in sequence, the selection kernel forming the head sums and
+ * dividing on its first sweep instead of a separate normalisation pass.
  *   workspace   curdkv_workspace_bytes(desc, budget > 0 ? budget : 1, adaptive) bytes
  *   head_offsets  may be NULL when adaptive = 0
  * Enqueues kernels and memsets on the stream only. */
