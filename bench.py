@@ -547,7 +547,7 @@ DECODE = dict(layers=32, batch=16, kv_heads=8, d=128, r=32, budget=2048, num_sin
 
 def run_decode(args):
     """Generation-phase workload (Sec. 3.2): every step appends `chunk` new rows per head to a cache
-    that holds `budget` rows and compresses it back to `budget` (Alg. 1 lines 2-10 on the cache)."""
+    that holds `budget` rows and compresses it back to `budget` (Alg. 1 (all steps) on the cache)."""
     from paper_2509_15038_b200 import binding as cur
 
     c = DECODE

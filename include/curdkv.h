@@ -5,12 +5,13 @@
  *
  * For every (batch element, KV head) the library
  *   1. sketches the bf16 key and value matrices with a caller-supplied Gaussian
- *      matrix G and takes squared sketch-row norms (Alg. 1 lines 2-4),
- *   2. multiplies key and value scores and normalises them per head (lines 5-6),
+ *      matrix G and takes squared sketch-row norms (Alg. 1 (sketch and row norms)),
+ *   2. multiplies key and value scores and normalises them per head (product and
+ *      normalisation steps),
  *   3. keeps the sink and recent-window tokens and the top-scoring rest
- *      (lines 7-9), with a fixed budget per head or AdaCurDKV's layer-wide
+ *      (sink, top-k and union steps), with a fixed budget per head or AdaCurDKV's layer-wide
  *      adaptive budgets (Sec. 3.2, "Adaptive budget allocation"),
- *   4. gathers the surviving rows into a compacted cache (line 10).
+ *   4. gathers the surviving rows into a compacted cache (gather step).
  *
  * General conventions
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned
@@ -73,10 +74,10 @@ typedef struct curdkv_desc {
   int64_t v_stride_b, v_stride_h, v_stride_n;
   const int32_t* seqlens; /* device int32 [batch]: valid rows n_b (clamped to [0, n_max]),
                              or NULL when every sequence has n_max rows                     */
-  int32_t score_mode;     /* 0: l = lK * lV (Alg. 1 line 5)  1: key only  2: value only
+  int32_t score_mode;     /* 0: l = lK * lV (Alg. 1 (product step))  1: key only  2: value only
                              (ablation of App. C.3)                                         */
-  int32_t use_projection; /* 1: sketch with G (Alg. 1 lines 2-3); 0: raw squared row norms  */
-  int32_t raw_scores;     /* 0: normalise per head (Alg. 1 line 6); 1: leave l^KV of line 5 as
+  int32_t use_projection; /* 1: sketch with G (Alg. 1 (sample G, project)); 0: raw squared row norms  */
+  int32_t raw_scores;     /* 0: normalise per head (Alg. 1 (normalisation step)); 1: leave l^KV of the product step as
                              it is (head_sums is still written) -- what the generation-phase
                              cache stores, since a row's l^KV does not depend on other rows  */
   int32_t whiten;         /* 0: Alg. 1 as printed (||a_j G||^2 follows the row norms).
@@ -98,7 +99,7 @@ typedef struct curdkv_desc {
  * descriptor. */
 size_t curdkv_workspace_bytes(const curdkv_desc* desc, int32_t max_budget, int32_t adaptive);
 
-/* Alg. 1 lines 2-6: scores[b][h][j] = lK_j * lV_j / sum_j(lK_j * lV_j) with
+/* Alg. 1 (scoring steps): scores[b][h][j] = lK_j * lV_j / sum_j(lK_j * lV_j) with
  * lK_j = ||K[b][h][j] G||^2, lV_j = ||V[b][h][j] G||^2 (fp32 accumulation).
  *   G          fp32 [d][r] row-major shared by all heads (g_per_head = 0) or
  *              [kv_heads][d][r] (g_per_head = 1); the same G for K and V.
@@ -142,7 +143,7 @@ curdkv_status curdkv_score_static(const void* K, const void* V, const float* G, 
                                   const curdkv_desc* desc, float* scores, float* head_sums,
                                   uint32_t* status_flags, void* cuda_stream);
 
-/* Alg. 1 lines 7-9 (adaptive = 0) or AdaCurDKV (adaptive = 1).
+/* Alg. 1 (sinks, top-k, union) (adaptive = 0) or AdaCurDKV (adaptive = 1).
  * Forced set of a sequence of n_b rows: the last `window` rows and the first
  * `num_sink` rows; if the budget cannot hold them all, the most recent window
  * rows come first, then sinks in index order.  Ties between equal scores go
@@ -170,7 +171,7 @@ curdkv_status curdkv_select(const float* scores, const curdkv_desc* desc, int32_
                             int32_t* head_offsets, void* workspace, size_t workspace_bytes,
                             void* cuda_stream);
 
-/* Alg. 1 line 10: K_out[row] = K[b][h][idx[...]], V_out likewise (byte copies).
+/* Alg. 1 (gather step): K_out[row] = K[b][h][idx[...]], V_out likewise (byte copies).
  *   out_stride_h > 0  fixed layout: idx is [batch][kv_heads][idx_stride]; row t of
  *                     head (b,h) goes to output row (b*kv_heads+h)*out_stride_h + t
  *   out_stride_h = 0  packed layout: head (b,h) starts at row head_offsets[b*kv_heads+h]
@@ -183,7 +184,7 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
                              const int32_t* head_offsets, void* K_out, void* V_out,
                              int64_t out_stride_h, void* workspace, void* cuda_stream);
 
-/* Alg. 1 lines 2-10 (or AdaCurDKV) in one call on device buffers: what curdkv_score,
+/* Alg. 1 (all steps) (or AdaCurDKV) in one call on device buffers: what curdkv_score,
  * curdkv_select and curdkv_compact do one after the other, with the same arguments,
  * the same outputs bit for bit (scores, head_sums, idx, head_counts, head_offsets,
  * gathered rows) and the default output layouts (adaptive = 0: idx
@@ -192,7 +193,7 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
  * r <= 32, n_max >= 128, no per-sequence lengths and at least four heads per SM of the
  * device, the scoring kernel also normalises and selects: the heads whose last tile has been
  * written are handed, through one list served by all CTAs, to extra warps that run Alg. 1
- * lines 6-9 for them while the stream of K and V goes on, so the selection costs almost no
+ * normalisation and selection steps for them while the stream of K and V goes on, so the selection costs almost no
  * time of its own (a cooperative launch; it can still be captured into a CUDA graph).  Other
  * shapes run the three steps in sequence, the selection kernel forming the head sums and
  * dividing on its first sweep instead of a separate normalisation pass.
@@ -206,7 +207,7 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
                               int32_t* head_offsets, void* K_out, void* V_out, void* workspace,
                               size_t workspace_bytes, void* cuda_stream);
 
-/* The whole path (Alg. 1 lines 2-10, or AdaCurDKV) for a cache that lives in HOST
+/* The whole path (Alg. 1 (all steps), or AdaCurDKV) for a cache that lives in HOST
  * memory: chunks of `chunk_batch` batch elements are copied to the device,
  * scored, selected and gathered, and the results copied back, double-buffered on
  * two internal streams so that copies overlap kernels.  Synchronous: returns when
@@ -232,9 +233,9 @@ curdkv_status curdkv_compress_host(const void* K_host, const void* V_host, const
 /* ---- Generation phase.  Sec. 3.2 notes that the method also applies while tokens are
  * generated, not only at prefill, and gives no procedure for it.  Reading used:
  * a cache holds, per (sequence, KV head), up to `capacity` rows of K and V with their
- * original token positions and their unnormalised scores l^KV (Alg. 1 lines 2-5).
+ * original token positions and their unnormalised scores l^KV (Alg. 1 (sketch, row norms, product)).
  * curdkv_cache_append scores newly generated rows and appends them;
- * curdkv_cache_compress applies Alg. 1 lines 6-10 to the rows held at that moment
+ * curdkv_cache_compress applies Alg. 1 (normalisation, selection, gather) to the rows held at that moment
  * (sinks = positions < num_sink, window = the most recent `window` rows, the
  * best-scoring rest up to `budget`, ascending position order).  Incremental
  * compression keeps exactly the tokens a single application of Alg. 1 to the whole
@@ -264,7 +265,7 @@ curdkv_status curdkv_cache_append(const curdkv_cache* cache, const void* K_new, 
                                   const float* G, int32_t g_per_head, const curdkv_desc* desc_new,
                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Alg. 1 lines 6-10 on the rows held in `in`; the kept rows, scores and positions go
+/* Alg. 1 (normalisation, selection, gather) on the rows held in `in`; the kept rows, scores and positions go
  * to `out` (a different cache with capacity >= min(budget, in->capacity); the two
  * must not overlap), which also receives the counters.  Sequences holding at most
  * `budget` rows are copied unchanged.  desc supplies batch, kv_heads and d.

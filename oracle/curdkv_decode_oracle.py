@@ -7,9 +7,9 @@ Sec. 3.2 states that the method applies while tokens are generated as well as at
 prefill, without spelling the procedure out.  The reading restated here: a cache
 holds, per (sequence, KV head), rows of K and V with their original token
 positions and their unnormalised combined scores l^KV_j = l^K_j * l^V_j
-(Alg. 1 lines 2-5; a row's score depends only on that row and on G).  Newly
+(Alg. 1 (sketch, row norms, product); a row's score depends only on that row and on G).  Newly
 generated rows are appended with their scores.  A compression step applies
-Alg. 1 lines 6-10 to the rows held at that moment: normalise over them, keep the
+Alg. 1 (normalisation, selection, gather) to the rows held at that moment: normalise over them, keep the
 sinks (positions < s), the most recent `window` positions and the best-scoring
 rest up to the budget k, in ascending position order.
 
@@ -26,7 +26,7 @@ from oracle import curdkv_oracle as orc
 
 
 def raw_scores(K, V, G):
-    """l^K_j * l^V_j in fp64 for bf16 bit patterns K, V [B,H,n,d] (Alg. 1 lines 2-5)."""
+    """l^K_j * l^V_j in fp64 for bf16 bit patterns K, V [B,H,n,d] (Alg. 1 (sketch, row norms, product))."""
     _, _, lK, lV = orc.score(K, V, G, return_factors=True)
     return lK * lV
 
@@ -57,7 +57,7 @@ class CacheOracle:
             self.total[b] += tb
 
     def compress(self, budget, num_sink, window):
-        """Alg. 1 lines 6-10 on the held rows of every (b, h)."""
+        """Alg. 1 (normalisation, selection, gather) on the held rows of every (b, h)."""
         for b in range(self.B):
             for h in range(self.H):
                 raw = self.raw[b][h]
@@ -65,10 +65,10 @@ class CacheOracle:
                 if n == 0:
                     continue
                 S = raw.sum()
-                norm = raw / S if S > 0 else np.zeros_like(raw)          # line 6
-                idx, cnt = orc.select_fixed(norm[None, None, :], budget, num_sink, window)  # lines 7-9
+                norm = raw / S if S > 0 else np.zeros_like(raw)          # normalise
+                idx, cnt = orc.select_fixed(norm[None, None, :], budget, num_sink, window)  # sinks, top-k, union
                 keep = idx[0, 0, : cnt[0, 0]]
-                self.pos[b][h] = self.pos[b][h][keep]                     # line 10 (+ bookkeeping)
+                self.pos[b][h] = self.pos[b][h][keep]                     # gather (+ bookkeeping)
                 self.raw[b][h] = raw[keep]
                 self.K[b][h] = self.K[b][h][keep]
                 self.V[b][h] = self.V[b][h][keep]

@@ -43,7 +43,7 @@ static int seq_len(const int32_t *seqlens, int b, int n_max) {
 }
 
 /* ------------------------------------------------------------------------
- * Algorithm 1, lines 2-6: sketch, squared row norms, product, normalise.
+ * Algorithm 1, scoring steps: sketch, squared row norms, product, normalise.
  *   score_mode 0: l = lK * lV (paper default)   1: l = lK   2: l = lV
  *   use_projection 0: rows are used as they are (ablation of App. C.3)
  * Optional outputs lK, lV (fp64 [B][H][n_max]) may be NULL.
@@ -102,7 +102,7 @@ void oracle_score(const uint16_t *K, const uint16_t *V, int B, int H, int n_max,
 }
 
 /* ------------------------------------------------------------------------
- * Forced-keep set (Algorithm 1 line 7, extended by the recent window):
+ * Forced-keep set (the sink step of Algorithm 1, extended by the recent window):
  *   F = {0..s-1}  U  {n-w..n-1}, clipped to the sequence.  If the budget
  * cannot hold all of F, the window's most recent tokens come first, then the
  * sinks in index order.  flag[j] = 1 for forced tokens; returns |F| kept.
@@ -132,7 +132,7 @@ static int cand_cmp(const void *pa, const void *pb) {
 static double key_of(double s) { return (s == s && s > 0.0) ? s : 0.0; }
 
 /* ------------------------------------------------------------------------
- * Algorithm 1, lines 7-9, fixed budget per head.
+ * Algorithm 1, selection steps (sinks, top-k, union), fixed budget per head.
  *   budget        k: rows kept per head, forced tokens included
  *   head_budgets  NULL, or int32 [B][H] caller-fixed k per head (<= budget)
  *   idx           int32 [B][H][budget], ascending token index, tail = -1
@@ -234,7 +234,7 @@ void oracle_select_adaptive(const double *scores, int B, int H, int n_max,
 }
 
 /* ------------------------------------------------------------------------
- * Algorithm 1 line 10: K'_i = K_i[S_i], V'_i = V_i[S_i] -- byte copies of the
+ * Algorithm 1, gather step: K'_i = K_i[S_i], V'_i = V_i[S_i] -- byte copies of the
  * original (unprojected) rows.  out_stride_h > 0: row t of head (b,h) goes to
  * ((b*H+h)*out_stride_h + t) * d (idx row stride idx_stride); out_stride_h = 0:
  * packed, head (b,h) starts at row offsets[b*H+h] in both idx and the output.

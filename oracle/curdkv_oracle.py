@@ -59,7 +59,7 @@ def num_threads() -> int:
 
 
 def score(K, V, G, seqlens=None, score_mode=0, use_projection=1, return_factors=False):
-    """Alg. 1 lines 2-6.  Returns (scores [B,H,n] f64, head_sums [B,H] f64[, lK, lV])."""
+    """Alg. 1 (scoring steps).  Returns (scores [B,H,n] f64, head_sums [B,H] f64[, lK, lV])."""
     K = np.ascontiguousarray(K, dtype=np.uint16)
     V = np.ascontiguousarray(V, dtype=np.uint16)
     G = np.ascontiguousarray(G, dtype=np.float32)
@@ -89,7 +89,7 @@ def score(K, V, G, seqlens=None, score_mode=0, use_projection=1, return_factors=
 
 
 def select_fixed(scores, budget, num_sink=0, window=0, seqlens=None, head_budgets=None):
-    """Alg. 1 lines 7-9.  Returns (idx [B,H,budget] int32 ascending, tail -1; counts [B,H])."""
+    """Alg. 1 (sinks, top-k, union).  Returns (idx [B,H,budget] int32 ascending, tail -1; counts [B,H])."""
     scores = np.ascontiguousarray(scores, dtype=np.float64)
     B, H, n = scores.shape
     seqlens = _i32(seqlens)
@@ -121,7 +121,7 @@ def select_adaptive(scores, budget, num_sink=0, window=0, alpha=0.2, seqlens=Non
 
 
 def compact(K, V, idx, counts, offsets=None):
-    """Alg. 1 line 10.  Fixed layout (idx [B,H,budget]) -> [B,H,budget,d] (unused rows 0);
+    """Alg. 1 (gather step).  Fixed layout (idx [B,H,budget]) -> [B,H,budget,d] (unused rows 0);
     packed layout (idx [total] with offsets) -> [total, d]."""
     K = np.ascontiguousarray(K, dtype=np.uint16)
     V = np.ascontiguousarray(V, dtype=np.uint16)

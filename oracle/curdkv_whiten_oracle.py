@@ -16,7 +16,7 @@ construction for the d x d Gram matrix:
 
 With G = I_d and ridge = 0, l_j = a_j (A^T A)^{-1} a_j^T = ||U(j,:)||^2 exactly
 (full column rank); a Gaussian G ~ N(0, 1/r) gives an unbiased estimate of it.
-The remaining steps are Alg. 1 lines 5-6 unchanged: l^KV = l^K l^V, normalise.
+The remaining steps are Alg. 1 (product and normalisation) unchanged: l^KV = l^K l^V, normalise.
 Rows at or beyond a sequence's length take no part (not in M, score 0).
 """
 from __future__ import annotations
@@ -59,7 +59,7 @@ def score_whitened(K, V, G, ridge, seqlens=None):
         for h in range(H):
             lK[b, h, :nb] = whitened_row_scores(K[b, h, :nb], G, ridge)
             lV[b, h, :nb] = whitened_row_scores(V[b, h, :nb], G, ridge)
-            l = lK[b, h, :nb] * lV[b, h, :nb]                    # Alg. 1 line 5
+            l = lK[b, h, :nb] * lV[b, h, :nb]                    # Alg. 1 (product step)
             sums[b, h] = l.sum()
-            scores[b, h, :nb] = l / sums[b, h] if sums[b, h] > 0 else 0.0   # line 6
+            scores[b, h, :nb] = l / sums[b, h] if sums[b, h] > 0 else 0.0   # normalise
     return scores, sums, lK, lV

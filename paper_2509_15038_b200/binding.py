@@ -188,7 +188,7 @@ def alloc_workspace(desc: Desc, max_budget: int = 1, adaptive: bool = False, dev
 
 
 def curdkv_score(K, V, G, desc: Desc, workspace: torch.Tensor, scores=None, head_sums=None):
-    """Alg. 1 lines 2-6.  G: fp32 device tensor [d, r] or [Hkv, d, r].  Returns (scores, head_sums)."""
+    """Alg. 1 (scoring steps).  G: fp32 device tensor [d, r] or [Hkv, d, r].  Returns (scores, head_sums)."""
     dev = K.device
     if scores is None:
         scores = torch.empty((desc.batch, desc.kv_heads, desc.n_max), dtype=torch.float32, device=dev)
@@ -224,7 +224,7 @@ def curdkv_select(scores, desc: Desc, budget: int, *, num_sink: int = 0, window:
                   head_budgets=None, adaptive: bool = False, alpha: float = 0.2,
                   workspace: Optional[torch.Tensor] = None, idx=None, head_counts=None,
                   head_offsets=None):
-    """Alg. 1 lines 7-9 / AdaCurDKV.  Returns (idx, head_counts, head_offsets)."""
+    """Alg. 1 (sinks, top-k, union) / AdaCurDKV.  Returns (idx, head_counts, head_offsets)."""
     dev = scores.device
     P = desc.batch * desc.kv_heads
     if idx is None:
@@ -247,7 +247,7 @@ def curdkv_select(scores, desc: Desc, budget: int, *, num_sink: int = 0, window:
 
 def curdkv_compact(K, V, desc: Desc, idx, head_counts, head_offsets=None, *, packed: bool = False,
                    K_out=None, V_out=None, workspace: Optional[torch.Tensor] = None):
-    """Alg. 1 line 10.  Fixed layout -> [B, Hkv, budget, d]; packed -> [capacity, d]."""
+    """Alg. 1 (gather step).  Fixed layout -> [B, Hkv, budget, d]; packed -> [capacity, d]."""
     dev = K.device
     if packed:
         rows = idx.numel()
@@ -272,7 +272,7 @@ def curdkv_compress(K, V, G, desc: Desc, budget: int, workspace: torch.Tensor, *
                     window: int = 0, head_budgets=None, adaptive: bool = False, alpha: float = 0.2,
                     scores=None, head_sums=None, idx=None, head_counts=None, head_offsets=None,
                     K_out=None, V_out=None):
-    """Alg. 1 lines 2-10 (or AdaCurDKV) in one call; the workspace must come from
+    """Alg. 1 (all steps) (or AdaCurDKV) in one call; the workspace must come from
     ``alloc_workspace(desc, budget, adaptive)``.  Returns (scores, head_sums, idx, head_counts,
     head_offsets, K_out, V_out) with the layouts of the three separate calls."""
     dev = K.device
@@ -384,7 +384,7 @@ def curdkv_cache_append(cache: DeviceCache, K_new, V_new, G, workspace: torch.Te
 
 def curdkv_cache_compress(src: DeviceCache, dst: DeviceCache, budget: int, workspace: torch.Tensor, *,
                           num_sink: int = 0, window: int = 0) -> None:
-    """Alg. 1 lines 6-10 on the rows held in ``src``; survivors go to ``dst``."""
+    """Alg. 1 (normalisation, selection, gather) on the rows held in ``src``; survivors go to ``dst``."""
     desc = Desc(src.batch, src.kv_heads, src.kv_heads, src.capacity, src.d, 1)
     desc.use_projection = 1
     code = load().curdkv_cache_compress(ctypes.byref(src.c), ctypes.byref(dst.c), ctypes.byref(desc),
@@ -395,7 +395,7 @@ def curdkv_cache_compress(src: DeviceCache, dst: DeviceCache, budget: int, works
 
 def curdkv_cache_compress_inplace(cache: DeviceCache, budget: int, workspace: torch.Tensor, *,
                                   num_sink: int = 0, window: int = 0) -> None:
-    """Alg. 1 lines 6-10 on the rows held in ``cache``, in place (the row order is given up)."""
+    """Alg. 1 (normalisation, selection, gather) on the rows held in ``cache``, in place (the row order is given up)."""
     desc = Desc(cache.batch, cache.kv_heads, cache.kv_heads, cache.capacity, cache.d, 1)
     desc.use_projection = 1
     code = load().curdkv_cache_compress_inplace(ctypes.byref(cache.c), ctypes.byref(desc), int(budget),

@@ -1,6 +1,6 @@
 // Bookkeeping kernels of the generation-phase cache (Sec. 3.2: the method also
 // applies while tokens are generated): rows are appended with their
-// unnormalised scores l^KV (Alg. 1 lines 2-5) and original positions, and a
+// unnormalised scores l^KV (Alg. 1 (sketch, row norms, product)) and original positions, and a
 // compression step carries scores and positions along with the gathered rows.
 #pragma once
 #include "common.cuh"
@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(256) cache_step_kernel(const StepArgs s) {
     if (tid == 0) flag_status(a.status, CURDKV_DEV_CACHE_FULL);
     tb = cap - held;
   }
-  // -------------------------------------------------------------- select (Alg. 1 lines 7-9)
+  // -------------------------------------------------------------- select (Alg. 1 (sinks, top-k, union))
   using G = WholeCta;
   const int n = held + tb;                                 // rows the head holds after the append
   const int k_eff = min(s.budget, n);
@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(256) cache_step_kernel(const StepArgs s) {
   select_fixed_row<G>(keys, F, k_eff, s.budget, step_keys, s.stage_quads, list, true, ix, sm);
   if (tid == 0) s.counts[p] = k_eff;
 
-  // -------------------------------------------------------------- place the survivors (Alg. 1 line 10)
+  // -------------------------------------------------------------- place the survivors (Alg. 1 (gather step))
   // ix is ascending: [0, first_new) old rows that stay, [first_new, first_mover) new rows whose
   // own slot lies below k_eff, [first_mover, k_eff) movers (slot >= k_eff) that go into the holes.
   // The staged keys are done with: their space takes the slot flags and the list of holes.

@@ -18,7 +18,7 @@ constexpr size_t kStatusBytes = 256;
 // Adds one to the library's launch counter (defined beside the C ABI).
 void count_launch();
 
-// curdkv_score without its last step: `scores` receive l^K l^V (Alg. 1 line 5) as the score
+// curdkv_score without its last step: `scores` receive l^K l^V (Alg. 1 (product step)) as the score
 // kernels leave them, entries at or beyond a sequence's length are unspecified, head sums are not
 // formed.  For callers that read the valid entries only (defined beside the C ABI).
 curdkv_status score_unnormalised(const void* K, const void* V, const float* G, int32_t g_per_head,

@@ -1,4 +1,4 @@
-// Gather of the selected rows into the compacted cache (Alg. 1 line 10):
+// Gather of the selected rows into the compacted cache (Alg. 1 (gather step)):
 // byte copies with 16-byte vectors, a half-warp per row (K in lanes 0-15, V in
 // lanes 16-31), eight rows in flight per warp.
 #pragma once

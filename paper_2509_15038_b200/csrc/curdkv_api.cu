@@ -267,7 +267,7 @@ namespace {
 
 // curdkv_score; with normalise = false the scores stay as the score kernels leave them
 // (unnormalised, one or four partial sums per tile in the workspace: *parts_per_tile) for a
-// selection kernel that finishes Alg. 1 line 6 itself.
+// selection kernel that finishes Alg. 1 (normalisation step) itself.
 curdkv_status score_impl(const void* K, const void* V, const float* G, int32_t g_per_head,
                          const curdkv_desc* desc, float* scores, float* head_sums, void* workspace,
                          size_t workspace_bytes, void* cuda_stream, bool normalise, int* parts_per_tile) {

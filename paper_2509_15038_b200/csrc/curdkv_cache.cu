@@ -1,5 +1,5 @@
 // Generation-phase cache (Sec. 3.2): append newly generated rows with their
-// l^KV, compress the held rows with Alg. 1 lines 6-10.  Built on the public
+// l^KV, compress the held rows with Alg. 1 (normalisation, selection, gather).  Built on the public
 // entry points of curdkv.h plus the bookkeeping kernels of cache.cuh.
 #include <cstdint>
 

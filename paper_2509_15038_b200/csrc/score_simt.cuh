@@ -1,13 +1,13 @@
 // Score kernels that run on the plain fp32 pipes.
 //
-//   row_norm_kernel    Alg. 1 without lines 2-3 (the "no projection" ablation of
+//   row_norm_kernel    Alg. 1 without its sampling and projection steps (the "no projection" ablation of
 //                      App. C.3): l_j = ||a_j||^2.  Pure streaming, HBM bound.
-//   sketch_fma_kernel  Alg. 1 lines 2-5 with fp32 FMAs: y = a_j G, l_j = ||y||^2.
+//   sketch_fma_kernel  Alg. 1 (sketch, row norms, product) with fp32 FMAs: y = a_j G, l_j = ||y||^2.
 //                      Kept for sketch shapes the tensor-core kernel does not
 //                      cover; fp32 G is used as it is (no splitting).
 //
 // Both write UNNORMALISED scores and one partial sum per 128-row tile; the
-// normalise kernel finishes Alg. 1 line 6.
+// normalise kernel finishes Alg. 1 (normalisation step).
 #pragma once
 #include "common.cuh"
 
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(256) sketch_fma_kernel(const ScoreArgs a, cons
 }
 
 // ---------------------------------------------------------------------------
-// Alg. 1 line 6: S = sum of the partial sums of the head's valid tiles in a
+// Alg. 1 (normalisation step): S = sum of the partial sums of the head's valid tiles in a
 // fixed order, scores /= S; scores at or beyond the sequence length become 0.
 // With `raw` the division is left out (S is still reported).
 // grid = batch*heads*ceil(n_max / 4096) (chunk fastest), block = 256.

@@ -1,5 +1,5 @@
 // Fused sketch + squared-norm + combine kernel on the 5th-gen tensor cores
-// (Alg. 1 lines 2-5) for d = 128 and r <= 64.
+// (Alg. 1 (sketch, row norms, product)) for d = 128 and r <= 64.
 //
 // Per 128-token tile and tensor (K, then V):  Y = A G  with A the bf16 tile
 // [128 x 128] brought in by TMA (128-byte swizzle) and G held in shared memory
@@ -29,7 +29,7 @@ namespace umma {
 constexpr int kThreads = 192;
 // The fused form adds a group of selection warps behind the six pipeline warps: whenever this CTA
 // writes the last tile of a head, they normalise that head's scores and select its tokens (Alg. 1
-// lines 6-9) while the pipeline goes on streaming.
+// normalisation and selection steps) while the pipeline goes on streaming.
 constexpr int kFusedSelThreads = 256;
 constexpr int kFusedSelFirst = kThreads + 32;              // one publisher warp sits between the two groups
 constexpr int kFusedThreads = kFusedSelFirst + kFusedSelThreads;
@@ -310,7 +310,7 @@ __device__ __forceinline__ int fused_pop(const Args& a, int nonempty_heads, vola
   }
 }
 
-// Alg. 1 lines 6-9 for head p by the selection warps (group G of kFusedSelThreads threads): the head
+// Alg. 1 (normalisation and selection) for head p by the selection warps (group G of kFusedSelThreads threads): the head
 // sum in the order normalise_kernel forms it, the division on the way into the leading-digit
 // histogram, then the fixed-budget selection of select_fixed_kernel on the normalised scores.
 template <class G>
@@ -660,7 +660,7 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       }
     }
   } else if constexpr (FUSED) {
-    // ------------------------------------------------------------ selection (Alg. 1 lines 6-9)
+    // ------------------------------------------------------------ selection (Alg. 1 (normalisation and selection))
     using G = WarpRange<kFusedSelFirst, kFusedSelThreads, 1>;
     const KeyList list{reinterpret_cast<uint2*>(base_ptr + L::kList), &fused.s.sel.list_count[0],
                        (uint32_t)kFusedListCap};

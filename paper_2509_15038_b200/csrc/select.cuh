@@ -1,4 +1,4 @@
-// Token selection (Alg. 1 lines 7-9 and AdaCurDKV, Sec. 3.2): forced sinks +
+// Token selection (Alg. 1 (sinks, top-k, union) and AdaCurDKV, Sec. 3.2): forced sinks +
 // window, then an exact top-k of the remaining scores by radix select on the
 // fp32 bit patterns (scores are >= 0, so the patterns order like the values),
 // ties to the lower token index, output in ascending token order.
@@ -545,7 +545,7 @@ __device__ __forceinline__ float head_sum_fixed_order(const float* partials, int
   return S;
 }
 
-// Alg. 1 line 6 for one row, on the way to the selection: row[j] <- row[j] / S for j < n (0 when the
+// Alg. 1 (normalisation step) for one row, on the way to the selection: row[j] <- row[j] / S for j < n (0 when the
 // sum is not positive; left as it is with `raw`), row[j] <- 0 for first_unwritten <= j < n_max, and
 // the leading-digit histogram of the resulting rank keys in `hist` (zero on entry).  With `staged`
 // (16-byte aligned rows only) the rank keys are also left there, a quad per four tokens.  The row
@@ -602,7 +602,7 @@ __device__ __forceinline__ void scale_row_and_histogram(float* row, const RowKey
   for (int j = first_unwritten + G::tid(); j < n_max; j += step) row[j] = 0.f;
 }
 
-// What a selection kernel needs to finish Alg. 1 line 6 itself (the scores then arrive as the
+// What a selection kernel needs to finish Alg. 1 (normalisation step) itself (the scores then arrive as the
 // score kernels leave them: unnormalised, with per-tile partial sums).  tile_sums = nullptr: the
 // scores are final already.
 struct Normaliser {
@@ -612,7 +612,7 @@ struct Normaliser {
 };
 
 // ---------------------------------------------------------------------------
-// Fixed per-head budget, one row, by the group G: Alg. 1 lines 7-9 on the scores `keys` describes.
+// Fixed per-head budget, one row, by the group G: Alg. 1 (sinks, top-k, union) on the scores `keys` describes.
 // k_eff = min(k, n) rows are kept; their ascending indices go to out[0, k_eff), -1 to
 // out[k_eff, budget).  `staged` (stage_quads quads, or nothing) may hold a copy of the keys;
 // `hist_ready` says that sm.hist already holds the leading-digit histogram of the row's keys (the

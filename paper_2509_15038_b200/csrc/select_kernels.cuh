@@ -1,4 +1,4 @@
-// The two selection kernels (Alg. 1 lines 7-9 with a fixed budget per head, and AdaCurDKV of
+// The two selection kernels (Alg. 1 (sinks, top-k, union) with a fixed budget per head, and AdaCurDKV of
 // Sec. 3.2), built from the per-row routines of select.cuh.
 #pragma once
 #include "select.cuh"
@@ -7,7 +7,7 @@ namespace curdkv {
 
 // grid = batch*heads, block = 1024, 512 or 256, dynamic shared memory = 16 * stage_quads bytes
 // (0: rows are read from global memory) followed by one candidate list of list_cap entries.
-// With norm.tile_sums the kernel first finishes Alg. 1 line 6 for its row (head sum, division on the
+// With norm.tile_sums the kernel first finishes Alg. 1 (normalisation step) for its row (head sum, division on the
 // way into the staged keys) and `scores` is written.
 __global__ void __launch_bounds__(kSelThreads) select_fixed_kernel(
     float* __restrict__ scores, const int32_t* __restrict__ seqlens, int heads, int n_max,
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS) select_adaptive_kerne
   clear_hist<G>(hist_all);
   if (tid == 0) sm.s.list_count[0] = sm.s.list_count[1] = 0;
   if (norm.tile_sums != nullptr) {
-    // Alg. 1 line 6 first: the scores arrive unnormalised, with per-tile partial sums
+    // Alg. 1 (normalisation step) first: the scores arrive unnormalised, with per-tile partial sums
     const int tiles = (n + kTileRows - 1) / kTileRows;
     const float S = head_sum_fixed_order<G>(
         norm.tile_sums + (size_t)p * norm.tiles_per_head * norm.parts_per_tile, tiles * norm.parts_per_tile, sm.s);

@@ -6,7 +6,7 @@
 //   M = A^T A + lambda I            gram_umma_kernel (tensor cores, one pass over K, V)
 //   M = L L^T,  W = L^{-T} G        whiten_factor_kernel (fp64, one CTA per matrix)
 //   l_j = ||a_j W||^2               sketch_items_kernel (second pass, W staged per head)
-// after which Alg. 1 lines 5-6 run unchanged.
+// after which Alg. 1 (product and normalisation) run unchanged.
 //
 // Both streaming kernels walk "items": a head cut into `segments` runs of
 // consecutive 128-row tiles, so that a CTA stays on one head long enough to
@@ -234,7 +234,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------
-// Sketch + norms + combine (Alg. 1 lines 2-5) with a projection that changes
+// Sketch + norms + combine (Alg. 1 (sketch, row norms, product)) with a projection that changes
 // from head to head (the whitened W of each head and tensor, or a caller's
 // per-head G) instead of one shared G.  Same pipeline as sketch_umma_kernel;
 // the epilogue warps restage [W_hi | W_lo] for K and for V at the start of

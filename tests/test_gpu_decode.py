@@ -22,7 +22,7 @@ def _history(B, H, N, d, seed):
 
 
 class _History:
-    """fp64 scores l^K l^V (Alg. 1 lines 2-5) of every real row a sequence has been fed, by position:
+    """fp64 scores l^K l^V (Alg. 1 (sketch, row norms, product)) of every real row a sequence has been fed, by position:
     what the tie-band rule measures a differing token against."""
 
     def __init__(self, B, H):

@@ -28,7 +28,7 @@ def rand_kv(rng, B, H, n, d, scale=1.0):
 # ---------------------------------------------------------------- sketch + norms
 
 def test_hand_worked_example():
-    """Alg. 1 lines 2-9 on the exact-arithmetic example in tests/golden/hand_example.txt."""
+    """Alg. 1 (scoring and selection) on the exact-arithmetic example in tests/golden/hand_example.txt."""
     vals = {}
     with open(os.path.join(GOLDEN, "hand_example.txt")) as f:
         for line in f:
