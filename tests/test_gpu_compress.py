@@ -124,6 +124,8 @@ def test_compress_options_and_layouts():
     _both_ways(K, V, G, 300, 0, 9, what="per-head budgets",
                head_budgets=np.tile(np.array([[300, 0, 13], [5000, 77, 1]], dtype=np.int32), (100, 1)))
     _both_ways(K, V, G, 0, 0, 0, what="budget 0")
+    _both_ways(K, V, G, 2000, 4, 32, what="budget above the row count")      # keeps every row
+    _both_ways(K, V, G, 40, 30, 30, what="forced rows beyond the budget")   # window first, then sinks
     _both_ways(torch.zeros_like(K), V, G, 100, 2, 4, what="all-zero keys")       # head sums of 0
     # token-major storage viewed as [B, H, n, d]
     g = torch.Generator(device=DEV).manual_seed(7)
