@@ -250,16 +250,21 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       uint32_t it = 0;
       bool ok = mbar_wait(q_full_bar, 0, abort_flag, a.status, a.wait_ns);
       tc_fence_after();
+      // The issuing thread shares its scheduler with two softmax warps, so what it executes per
+      // MMA counts: descriptors are formed once per tile and stepped by constants (the address
+      // field counts 16-byte units and cannot carry out of its 14 bits inside shared memory).
+      const uint64_t q_desc = smem_desc_sw128(base + kAttnQ);
       auto issue_s = [&](uint32_t buf) {                   // S[buf] = Q K^T for the next K tile of the ring
         const int slot = it % kAttnRing;
         if (!(ok = mbar_wait(full_bar(slot), (it / kAttnRing) & 1u, abort_flag, a.status, a.wait_ns))) return;
         tc_fence_after();
-        const uint32_t k_base = base + kAttnSlot0 + slot * kSlotBytes;
+        const uint64_t k_desc = smem_desc_sw128(base + kAttnSlot0 + slot * kSlotBytes);
+        const uint32_t d_tmem = tmem_base + buf * 128u;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          tc_mma_bf16(tmem_base + buf * 128u, smem_desc_sw128(base + kAttnQ + off),
-                      smem_desc_sw128(k_base + off), idesc_s, k > 0);
+          constexpr uint32_t kHalfUnits = kHalfBytes >> 4;
+          const uint32_t off = (uint32_t)(k >> 2) * kHalfUnits + (uint32_t)(k & 3) * 2u;   // 16-byte units
+          tc_mma_bf16(d_tmem, q_desc + off, k_desc + off, idesc_s, k > 0);
         }
         tc_commit(empty_bar(slot));
         tc_commit(s_full_bar(buf));
@@ -285,13 +290,21 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         const uint32_t buf = (uint32_t)t & 1u;             // the group that owns this tile, its P and O
         if (!(ok = mbar_wait(p_ready_bar(buf), (uint32_t)(t >> 1) & 1u, abort_flag, a.status, a.wait_ns))) break;
         tc_fence_after();
-        const uint32_t v_base = base + kAttnSlot0 + slot * kSlotBytes;
+        const uint64_t v_desc = smem_desc_mn_sw128(base + kAttnSlot0 + slot * kSlotBytes);
+        const uint32_t o_tmem = tmem_base + 256u + buf * 128u;
+#pragma unroll
         for (int part = 0; part < (SPLIT ? 2 : 1); ++part) {   // P_hi, then P_lo
           const uint32_t p_tmem = tmem_base + buf * 128u + part * 64u;
-          for (int g = 0; g < groups; ++g)                 // 16 keys per MMA: 8 columns of P
-            tc_mma_bf16_ts(tmem_base + 256u + buf * 128u, p_tmem + 8u * g,
-                           smem_desc_mn_sw128(v_base + g * 2048), idesc_pv,
-                           (t > 1 || part > 0 || g > 0) ? 1u : 0u);
+          // 16 keys per MMA: 8 columns of P, 2048 bytes (128 units) of the V tile
+          if (groups == 8) {
+            tc_mma_bf16_ts(o_tmem, p_tmem, v_desc, idesc_pv, (t > 1 || part > 0) ? 1u : 0u);
+#pragma unroll
+            for (int g = 1; g < 8; ++g) tc_mma_bf16_ts(o_tmem, p_tmem + 8u * g, v_desc + 128u * g, idesc_pv, 1u);
+          } else {
+            for (int g = 0; g < groups; ++g)
+              tc_mma_bf16_ts(o_tmem, p_tmem + 8u * g, v_desc + 128u * g, idesc_pv,
+                             (t > 1 || part > 0 || g > 0) ? 1u : 0u);
+          }
         }
         tc_commit(empty_bar(slot));
         ++it;
