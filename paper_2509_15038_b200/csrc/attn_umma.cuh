@@ -46,10 +46,16 @@ constexpr int kAttnQ = 0;
 constexpr int kAttnSlot0 = kSlotBytes;
 constexpr int kAttnBar = kAttnSlot0 + kAttnRing * kSlotBytes;
 constexpr int kAttnDynamic = kAttnBar + 256 + 1024;
-// TMEM columns: S of group g at 128 g, overwritten in place by its P (bf16 pairs: P_hi in the
-// first 64 columns, P_lo in the last 64); O of group g at 256 + 128 g
+// TMEM columns: S of group g at 128 g, overwritten in place by its P (bf16 pairs, see
+// attn_p_column); O of group g at 256 + 128 g
 constexpr int kAttnTmemCols = 512;
 constexpr float kAttnMaxSlack = 8.f;                       // log2 units a tile may exceed the running maximum
+
+// Where the weights of a tile sit inside the 128 columns its logits came in: the weights of keys
+// 32c .. 32c+31 stay inside the columns of those keys' logits, P_hi (16 columns of bf16 pairs) at
+// 32c and P_lo at 32c + 16, so that a softmax thread can turn the row over 32 keys at a time.
+// Column of P_hi for the g-th group of 16 keys:
+__host__ __device__ constexpr uint32_t attn_p_column(int g) { return 32u * (uint32_t)(g >> 1) + 8u * (uint32_t)(g & 1); }
 
 // P V: A = P K-major, B = V tile MN-major (contraction over the keys)
 __host__ __device__ constexpr uint32_t instr_desc_pv() { return instr_desc_bf16(128) | (1u << 16); }
@@ -294,15 +300,16 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         const uint32_t o_tmem = tmem_base + 256u + buf * 128u;
 #pragma unroll
         for (int part = 0; part < (SPLIT ? 2 : 1); ++part) {   // P_hi, then P_lo
-          const uint32_t p_tmem = tmem_base + buf * 128u + part * 64u;
-          // 16 keys per MMA: 8 columns of P, 2048 bytes (128 units) of the V tile
+          const uint32_t p_tmem = tmem_base + buf * 128u + part * 16u;
+          // 16 keys per MMA: 8 columns of P (attn_p_column), 2048 bytes (128 units) of the V tile
           if (groups == 8) {
             tc_mma_bf16_ts(o_tmem, p_tmem, v_desc, idesc_pv, (t > 1 || part > 0) ? 1u : 0u);
 #pragma unroll
-            for (int g = 1; g < 8; ++g) tc_mma_bf16_ts(o_tmem, p_tmem + 8u * g, v_desc + 128u * g, idesc_pv, 1u);
+            for (int g = 1; g < 8; ++g)
+              tc_mma_bf16_ts(o_tmem, p_tmem + attn_p_column(g), v_desc + 128u * g, idesc_pv, 1u);
           } else {
             for (int g = 0; g < groups; ++g)
-              tc_mma_bf16_ts(o_tmem, p_tmem + 8u * g, v_desc + 128u * g, idesc_pv,
+              tc_mma_bf16_ts(o_tmem, p_tmem + attn_p_column(g), v_desc + 128u * g, idesc_pv,
                              (t > 1 || part > 0 || g > 0) ? 1u : 0u);
           }
         }
@@ -336,32 +343,44 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       if (!(ok = __all_sync(0xffffffffu, ok))) break;
       tc_fence_after();
       const int valid = n - t * kTileRows;                 // keys of this tile that exist
-      // the whole row of S into registers: its columns are about to take P
-      float v[128];
-#pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) tmem_ld32(s_addr + c0, *reinterpret_cast<float(*)[32]>(v + c0));
-      tmem_ld_wait();
+      // First pass over the row: its maximum.  The row is read from TMEM 64 columns at a time here
+      // and again below (a thread that held all 128 logits left the compiler no room).
       float tile_top = -INFINITY;
       if (valid >= kTileRows) {
         // max_c (v_c * sc) = sc * max_c v_c or sc * min_c v_c; four independent chains
-        float ext[4] = {v[0], v[1], v[2], v[3]};
-        if (sc >= 0.f) {
+        float ext[4];
 #pragma unroll
-          for (int c = 4; c < 128; c += 8)
+        for (int c0 = 0; c0 < 128; c0 += 64) {
+          float v[64];
+          tmem_ld32(s_addr + c0, *reinterpret_cast<float(*)[32]>(v));
+          tmem_ld32(s_addr + c0 + 32, *reinterpret_cast<float(*)[32]>(v + 32));
+          tmem_ld_wait();
+          if (c0 == 0) { ext[0] = v[0]; ext[1] = v[1]; ext[2] = v[2]; ext[3] = v[3]; }
+          if (sc >= 0.f) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) ext[j] = c + 2 * j + 1 < 128 ? max3(ext[j], v[c + 2 * j], v[c + 2 * j + 1]) : ext[j];
-          tile_top = fmaxf(fmaxf(ext[0], ext[1]), fmaxf(ext[2], ext[3])) * sc;
-        } else {
+            for (int c = 0; c < 64; c += 8)
 #pragma unroll
-          for (int c = 4; c < 128; c += 8)
+              for (int j = 0; j < 4; ++j) ext[j] = max3(ext[j], v[c + 2 * j], v[c + 2 * j + 1]);
+          } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) ext[j] = c + 2 * j + 1 < 128 ? min3(ext[j], v[c + 2 * j], v[c + 2 * j + 1]) : ext[j];
-          tile_top = fminf(fminf(ext[0], ext[1]), fminf(ext[2], ext[3])) * sc;
+            for (int c = 0; c < 64; c += 8)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) ext[j] = min3(ext[j], v[c + 2 * j], v[c + 2 * j + 1]);
+          }
         }
+        tile_top = (sc >= 0.f ? fmaxf(fmaxf(ext[0], ext[1]), fmaxf(ext[2], ext[3]))
+                              : fminf(fminf(ext[0], ext[1]), fminf(ext[2], ext[3]))) * sc;
       } else {
 #pragma unroll
-        for (int c = 0; c < 128; ++c)
-          if (c < valid) tile_top = fmaxf(tile_top, v[c] * sc);
+        for (int c0 = 0; c0 < 128; c0 += 64) {
+          float v[64];
+          tmem_ld32(s_addr + c0, *reinterpret_cast<float(*)[32]>(v));
+          tmem_ld32(s_addr + c0 + 32, *reinterpret_cast<float(*)[32]>(v + 32));
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 64; ++c)
+            if (c0 + c < valid) tile_top = fmaxf(tile_top, v[c] * sc);
+        }
       }
       // move the running maximum only when the tile exceeds it by more than the slack
       const bool move = tile_top > top + kAttnMaxSlack || top == -INFINITY;
@@ -382,36 +401,44 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       }
       sum *= alpha;
       top = new_top;
+      // Second pass: the weights of 64 keys take the place of those keys' logits.
       if (valid >= kTileRows) {
         // full tile: the arithmetic runs on packed pairs of keys
         const uint64_t sc2 = pack2(sc, sc), ntop2 = pack2(-top, -top);
         uint64_t part[4] = {0ull, 0ull, 0ull, 0ull};       // eight partial row sums
 #pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {             // 32 keys -> 16 columns of P_hi and of P_lo
-          uint32_t hi[16], lo[16];
+        for (int c0 = 0; c0 < 128; c0 += 64) {
+          float v[64];
+          tmem_ld32(s_addr + c0, *reinterpret_cast<float(*)[32]>(v));
+          tmem_ld32(s_addr + c0 + 32, *reinterpret_cast<float(*)[32]>(v + 32));
+          tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int c = c0 + 2 * e;
-            float x0, x1;
-            unpack2(fma2(pack2(v[c], v[c + 1]), sc2, ntop2), x0, x1);
-            const uint64_t w2 = pack2(fast_exp2(x0), fast_exp2(x1));
-            float w0, w1;
-            unpack2(w2, w0, w1);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
-            hi[e] = *reinterpret_cast<const uint32_t*>(&h);
-            const uint64_t h2 = pack2(__uint_as_float(hi[e] << 16), __uint_as_float(hi[e] & 0xffff0000u));
-            if (SPLIT) {
-              part[e & 3] = add2(part[e & 3], w2);         // equals the bf16 pairs to 2^-17
-              float r0, r1;
-              unpack2(sub2(w2, h2), r0, r1);
-              const __nv_bfloat162 q = __floats2bfloat162_rn(r0, r1);
-              lo[e] = *reinterpret_cast<const uint32_t*>(&q);
-            } else {
-              part[e & 3] = add2(part[e & 3], h2);         // the weights the product really uses
+          for (int c1 = 0; c1 < 64; c1 += 32) {            // 32 keys -> 16 columns of P_hi and of P_lo
+            uint32_t hi[16], lo[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const int c = c1 + 2 * e;
+              float x0, x1;
+              unpack2(fma2(pack2(v[c], v[c + 1]), sc2, ntop2), x0, x1);
+              const uint64_t w2 = pack2(fast_exp2(x0), fast_exp2(x1));
+              float w0, w1;
+              unpack2(w2, w0, w1);
+              const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
+              hi[e] = *reinterpret_cast<const uint32_t*>(&h);
+              const uint64_t h2 = pack2(__uint_as_float(hi[e] << 16), __uint_as_float(hi[e] & 0xffff0000u));
+              if (SPLIT) {
+                part[e & 3] = add2(part[e & 3], w2);       // equals the bf16 pairs to 2^-17
+                float r0, r1;
+                unpack2(sub2(w2, h2), r0, r1);
+                const __nv_bfloat162 q = __floats2bfloat162_rn(r0, r1);
+                lo[e] = *reinterpret_cast<const uint32_t*>(&q);
+              } else {
+                part[e & 3] = add2(part[e & 3], h2);       // the weights the product really uses
+              }
             }
+            tmem_st16(s_addr + (uint32_t)(c0 + c1), hi);
+            if (SPLIT) tmem_st16(s_addr + (uint32_t)(c0 + c1) + 16u, lo);
           }
-          tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
-          if (SPLIT) tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
         }
         float p0, p1;
         unpack2(add2(add2(part[0], part[1]), add2(part[2], part[3])), p0, p1);
@@ -419,18 +446,25 @@ attention_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
       } else {
         // last tile of the cache: keys beyond its end are masked by index
 #pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t hi[16], lo[16];
+        for (int c0 = 0; c0 < 128; c0 += 64) {
+          float v[64];
+          tmem_ld32(s_addr + c0, *reinterpret_cast<float(*)[32]>(v));
+          tmem_ld32(s_addr + c0 + 32, *reinterpret_cast<float(*)[32]>(v + 32));
+          tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int c = c0 + 2 * e;
-            const float w0 = c < valid ? fast_exp2(fmaf(v[c], sc, -top)) : 0.f;
-            const float w1 = c + 1 < valid ? fast_exp2(fmaf(v[c + 1], sc, -top)) : 0.f;
-            split_bf16x2(w0, w1, hi[e], lo[e]);
-            sum += SPLIT ? w0 + w1 : __uint_as_float(hi[e] << 16) + __uint_as_float(hi[e] & 0xffff0000u);
+          for (int c1 = 0; c1 < 64; c1 += 32) {
+            uint32_t hi[16], lo[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const int c = c1 + 2 * e;
+              const float w0 = c0 + c < valid ? fast_exp2(fmaf(v[c], sc, -top)) : 0.f;
+              const float w1 = c0 + c + 1 < valid ? fast_exp2(fmaf(v[c + 1], sc, -top)) : 0.f;
+              split_bf16x2(w0, w1, hi[e], lo[e]);
+              sum += SPLIT ? w0 + w1 : __uint_as_float(hi[e] << 16) + __uint_as_float(hi[e] & 0xffff0000u);
+            }
+            tmem_st16(s_addr + (uint32_t)(c0 + c1), hi);
+            if (SPLIT) tmem_st16(s_addr + (uint32_t)(c0 + c1) + 16u, lo);
           }
-          tmem_st16(s_addr + (uint32_t)(c0 >> 1), hi);
-          if (SPLIT) tmem_st16(s_addr + 64u + (uint32_t)(c0 >> 1), lo);
         }
       }
       tmem_st_wait();
