@@ -170,9 +170,15 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             const uint32_t d_tmem = tmem_base + acc * 256u + tensor * 128u;
-            for (int g = 0; g < groups; ++g) {
-              const uint64_t desc = smem_desc_mn_sw128(tile + g * 2048);
-              tc_mma_bf16(d_tmem, desc, desc, idesc, (t > w.t_lo || g > 0) ? 1u : 0u);
+            // one descriptor per tile, stepped by 2048 bytes (128 units of 16 bytes) per 16 rows
+            const uint64_t desc0 = smem_desc_mn_sw128(tile);
+            if (groups == 8) {
+              tc_mma_bf16(d_tmem, desc0, desc0, idesc, t > w.t_lo ? 1u : 0u);
+#pragma unroll
+              for (int g = 1; g < 8; ++g) tc_mma_bf16(d_tmem, desc0 + 128u * g, desc0 + 128u * g, idesc, 1u);
+            } else {
+              for (int g = 0; g < groups; ++g)
+                tc_mma_bf16(d_tmem, desc0 + 128u * g, desc0 + 128u * g, idesc, (t > w.t_lo || g > 0) ? 1u : 0u);
             }
             tc_commit(empty_bar(slot));
           }
