@@ -93,7 +93,7 @@ typedef struct curdkv_desc {
 
 /* Bytes of device workspace the calls below need for this shape (256-byte
  * aligned base required).  max_budget > 0 includes what curdkv_compress needs on
- * top of curdkv_score (one counter per head); max_budget = 0 sizes a workspace
+ * top of curdkv_score (three counters per head); max_budget = 0 sizes a workspace
  * for curdkv_score / curdkv_select / curdkv_compact alone.  `adaptive` is
  * reserved (it does not change the size today).  Returns 0 for an invalid
  * descriptor. */
@@ -377,7 +377,9 @@ curdkv_status curdkv_selftest_bounded_wait(uint64_t limit_ns, void* workspace, v
  * before and after its sketch kernel -- the kernel that streams K and V -- so
  * that a benchmark can time that kernel alone without a profiler.  The request
  * is cleared by that call.  With projection off or n_max < 128 the scores come
- * from a plain streaming kernel and nothing is recorded. */
+ * from a plain streaming kernel and nothing is recorded.  (Inside curdkv_compress
+ * an event behind the kernel that scores and selects keeps the gather from
+ * starting before that kernel has ended, which costs the call about 1 %.) */
 curdkv_status curdkv_profile_next_score(void* start_event, void* stop_event);
 
 /* Number of kernels this library has launched in this process so far. */

@@ -40,6 +40,13 @@ __device__ __forceinline__ void flag_status(uint32_t* status, uint32_t bits) {
   if (status != nullptr) atomicOr(status, bits);
 }
 
+// Nanoseconds of the device-wide timer (the clock every bounded wait is measured on).
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
 // Eight bf16 values packed in a 16-byte vector -> fp32.
 __device__ __forceinline__ void unpack_bf16x8(const uint4& v, float (&f)[8]) {
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};

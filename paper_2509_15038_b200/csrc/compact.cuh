@@ -18,6 +18,11 @@ struct CompactArgs {
   __nv_bfloat16* V_out;
   int64_t out_stride_h;     // > 0: fixed layout, 0: packed
   uint32_t* status;
+  // Set when the launch may start before the kernel that selects has finished (programmatic
+  // dependent launch behind the fused score + select kernel): ready[p] becomes non-zero once
+  // head p's indices and count are written and fenced; a CTA waits for its head's entry.
+  const int32_t* ready = nullptr;
+  unsigned long long wait_ns = 2000000000ull;
 };
 
 constexpr int kCompactWarps = 8;
@@ -32,9 +37,32 @@ __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const Compa
   const int n = seq_len_of(a.seqlens, b, a.n_max);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
   const bool fixed = a.out_stride_h > 0;
+  if (a.ready != nullptr) {
+    __shared__ int head_missing;
+    if (threadIdx.x == 0) {
+      head_missing = 0;
+      unsigned long long t0 = 0;
+      for (uint32_t spin = 1; *(volatile const int32_t*)(a.ready + p) == 0; ++spin) {
+        __nanosleep(500);
+        if ((spin & 0x3fu) == 0) {
+          const unsigned long long now = global_ns();
+          if (t0 == 0) t0 = now;
+          // the selecting kernel flags its own failures; here the head simply never arrived
+          if ((*(volatile uint32_t*)a.status & CURDKV_DEV_TIMEOUT) != 0 || now - t0 > a.wait_ns) {
+            flag_status(a.status, CURDKV_DEV_TIMEOUT);
+            head_missing = 1;
+            break;
+          }
+        }
+      }
+      __threadfence();                                     // the head's indices were written by another CTA
+    }
+    __syncthreads();
+    if (head_missing) return;
+  }
   // a count the layout cannot hold (a stale or unwritten counts buffer) is cut to what it can
   // hold and flagged, so that neither the index row nor the output rows of a neighbour are touched
-  int count = a.counts[p];
+  int count = __ldcg(a.counts + p);                        // (written by a kernel that may still run)
   const int64_t room = fixed ? (a.idx_stride < a.out_stride_h ? a.idx_stride : a.out_stride_h)
                              : (int64_t)a.offsets[p + 1] - a.offsets[p];
   if (count < 0 || count > room) {
@@ -53,7 +81,7 @@ __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const Compa
     int j[kCompactRowsPerWarp];
 #pragma unroll
     for (int i = 0; i < kCompactRowsPerWarp; ++i) {
-      j[i] = t0 + i < count ? __ldg(ix + t0 + i) : -1;
+      j[i] = t0 + i < count ? __ldcg(ix + t0 + i) : -1;
       if (t0 + i < count && (j[i] < 0 || j[i] >= n)) {
         if (lane == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
         j[i] = -1;

@@ -62,9 +62,9 @@ inline int stream_evict_first(const curdkv_desc* d) {
 }
 
 // What curdkv_compress keeps next to the status words: per head a tile counter and an entry of
-// the list of finished heads, and two queue counters.
+// the list of finished heads and a selected flag, and two queue counters.
 inline size_t head_counter_bytes(const curdkv_desc* d) {
-  return round256((size_t)d->batch * d->kv_heads * 2 * sizeof(int32_t)) + 256;
+  return round256((size_t)d->batch * d->kv_heads * 3 * sizeof(int32_t)) + 256;
 }
 
 // ---- TMA descriptors for the tensor-core sketch kernel ---------------------
@@ -235,6 +235,10 @@ namespace {
 curdkv_status score_impl(const void* K, const void* V, const float* G, int32_t g_per_head,
                          const curdkv_desc* desc, float* scores, float* head_sums, void* workspace,
                          size_t workspace_bytes, void* cuda_stream, bool normalise, int* parts_per_tile);
+curdkv_status compact_impl(const void* K, const void* V, const curdkv_desc* desc, const int32_t* idx,
+                           int64_t idx_stride, const int32_t* head_counts, const int32_t* head_offsets,
+                           void* K_out, void* V_out, int64_t out_stride_h, void* workspace,
+                           void* cuda_stream, const int32_t* ready);
 }  // namespace
 
 namespace curdkv {
@@ -582,6 +586,20 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
                              const int32_t* idx, int64_t idx_stride, const int32_t* head_counts,
                              const int32_t* head_offsets, void* K_out, void* V_out,
                              int64_t out_stride_h, void* workspace, void* cuda_stream) {
+  return compact_impl(K, V, desc, idx, idx_stride, head_counts, head_offsets, K_out, V_out, out_stride_h,
+                      workspace, cuda_stream, nullptr);
+}
+
+}  // extern "C"
+
+namespace {
+
+// curdkv_compact; with `ready` the launch is a programmatic dependent of the kernel before it
+// in the stream (the fused score + select kernel), whose selection groups set ready[p] per head.
+curdkv_status compact_impl(const void* K, const void* V, const curdkv_desc* desc, const int32_t* idx,
+                           int64_t idx_stride, const int32_t* head_counts, const int32_t* head_offsets,
+                           void* K_out, void* V_out, int64_t out_stride_h, void* workspace,
+                           void* cuda_stream, const int32_t* ready) {
   curdkv_status st = check_desc(desc);
   if (st != CURDKV_OK) return st;
   if ((st = check_kv(K, V, desc)) != CURDKV_OK) return st;
@@ -610,17 +628,38 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
   a.V_out = static_cast<__nv_bfloat16*>(V_out);
   a.out_stride_h = out_stride_h;
   a.status = static_cast<uint32_t*>(workspace);
+  a.ready = ready;
 
   // enough CTAs per head to cover a typical head in one sweep; larger heads loop
   const int64_t rows_hint = out_stride_h > 0 ? out_stride_h : (idx_stride > 0 ? idx_stride : 1024);
   int64_t ctas = (rows_hint + kCompactRowsPerCta - 1) / kCompactRowsPerCta;
+  // (a CTA that first has to wait for its head's flag pays a round trip to L2 for it: eight
+  // sweeps per CTA then)
+  if (ready != nullptr) ctas = (ctas + 7) / 8;
   if (ctas < 1) ctas = 1;
   if (ctas > 256) ctas = 256;
   while (P * ctas > 0x7fffffffLL) ctas >>= 1;
-  compact_kernel<<<(unsigned)(P * ctas), kCompactWarps * 32, 0, stream>>>(a, (int)ctas);
+  if (ready == nullptr) {
+    compact_kernel<<<(unsigned)(P * ctas), kCompactWarps * 32, 0, stream>>>(a, (int)ctas);
+  } else {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(P * ctas));
+    cfg.blockDim = dim3(kCompactWarps * 32);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, compact_kernel, a, (int)ctas) != cudaSuccess) return CURDKV_ERR_CUDA;
+  }
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int32_t g_per_head,
                               const curdkv_desc* desc, int32_t budget, const int32_t* head_budgets,
@@ -676,7 +715,8 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
     if (cudaMemsetAsync(ws, 0, kStatusBytes + counters, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
     int32_t* head_done = reinterpret_cast<int32_t*>(ws + kStatusBytes);
     int32_t* done_list = head_done + P;
-    int32_t* queue_ctr = reinterpret_cast<int32_t*>(ws + kStatusBytes + round256((size_t)P * 2 * sizeof(int32_t)));
+    int32_t* head_ready = done_list + P;
+    int32_t* queue_ctr = reinterpret_cast<int32_t*>(ws + kStatusBytes + round256((size_t)P * 3 * sizeof(int32_t)));
     float* tile_sums = reinterpret_cast<float*>(ws + kStatusBytes + counters);
     CUtensorMap mk, mv;
     if (!make_tile_map(&mk, K, desc, desc->k_stride_b, desc->k_stride_h, desc->k_stride_n) ||
@@ -698,6 +738,7 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
     u.head_done = head_done;
     u.done_list = done_list;
     u.queue_ctr = queue_ctr;
+    u.head_ready = head_ready;
     u.head_budgets = head_budgets;
     u.idx = idx;
     u.counts = head_counts;
@@ -720,8 +761,14 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
   }
   if (st != CURDKV_OK) return st;
   if (!adaptive && budget == 0) return CURDKV_OK;          // nothing is kept, nothing to gather
-  return curdkv_compact(K, V, desc, idx, adaptive ? 0 : budget, head_counts, head_offsets, K_out, V_out,
-                        adaptive ? 0 : budget, workspace, cuda_stream);
+  // Behind the fused kernel the gather is launched as its programmatic dependent: its CTAs move in
+  // as that kernel's CTAs finish and copy the heads already selected while the last heads'
+  // selection, which only starts when the stream ends, is still running.
+  const int32_t* ready = nullptr;
+  if (fused)
+    ready = reinterpret_cast<const int32_t*>(static_cast<unsigned char*>(workspace) + kStatusBytes) + 2 * P;
+  return compact_impl(K, V, desc, idx, adaptive ? 0 : budget, head_counts, head_offsets, K_out, V_out,
+                      adaptive ? 0 : budget, workspace, cuda_stream, ready);
 }
 
 curdkv_status curdkv_gqa_map(const curdkv_desc* desc, int32_t* kv_head_of_q, void* cuda_stream) {

@@ -59,6 +59,7 @@ struct Args {
   int32_t* head_done = nullptr;        // [batch*heads] tiles written so far, zero on entry
   int32_t* done_list = nullptr;        // [batch*heads] finished heads (index + 1) in the order they finished; zero on entry
   int32_t* queue_ctr = nullptr;        // [2] heads entered into done_list / tickets handed to selection groups; zero on entry
+  int32_t* head_ready = nullptr;       // [batch*heads] or nullptr: set to 1 once a head's indices and count are written; zero on entry
   const int32_t* head_budgets = nullptr;
   int32_t* idx = nullptr;              // [batch*heads][budget]
   int32_t* counts = nullptr;
@@ -137,11 +138,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
 }
 // Bounded wait.  Gives up when another role has aborted or after limit_ns;
 // then raises the CTA's abort flag and the device status bit.
@@ -436,6 +432,12 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  if constexpr (FUSED) {
+    // A gather launched as a programmatic dependent of this kernel may be scheduled from here on;
+    // its CTAs find room as CTAs of this launch finish, and wait per head on head_ready.  (Without
+    // such a dependent the instruction does nothing.)
+    if (tid == 0 && a.head_ready != nullptr) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
 
   // ---- tile schedule: running tile number -> (problem p, first row, valid rows n)
   const uint32_t* prefix = reinterpret_cast<const uint32_t*>(base_ptr + L::kPrefix);
@@ -674,6 +676,13 @@ sketch_umma_kernel(const __grid_constant__ CUtensorMap map_k,
       G::sync();
       if (p < 0) break;
       fused_select_head<G>(a, p, list, fused.s.sel);
+      if (a.head_ready != nullptr) {
+        G::sync();                                         // every thread's indices are written
+        if (G::tid() == 0) {
+          __threadfence();
+          *(volatile int32_t*)(a.head_ready + p) = 1;
+        }
+      }
     }
   }
 
