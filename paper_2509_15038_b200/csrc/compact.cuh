@@ -30,6 +30,8 @@ constexpr int kCompactRowsPerWarp = 8;
 constexpr int kCompactRowsPerCta = kCompactWarps * kCompactRowsPerWarp;
 
 // grid = batch*heads*ctas_per_head; the CTAs of a head stride over its rows.
+// BEHIND: the launch is a programmatic dependent of the kernel that selects (a.ready is set).
+template <bool BEHIND>
 __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const CompactArgs a,
                                                                      const int ctas_per_head) {
   const int p = blockIdx.x / ctas_per_head, part = blockIdx.x % ctas_per_head;
@@ -37,7 +39,7 @@ __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const Compa
   const int n = seq_len_of(a.seqlens, b, a.n_max);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
   const bool fixed = a.out_stride_h > 0;
-  if (a.ready != nullptr) {
+  if constexpr (BEHIND) {
     __shared__ int head_missing;
     if (threadIdx.x == 0) {
       head_missing = 0;
@@ -62,7 +64,9 @@ __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const Compa
   }
   // a count the layout cannot hold (a stale or unwritten counts buffer) is cut to what it can
   // hold and flagged, so that neither the index row nor the output rows of a neighbour are touched
-  int count = __ldcg(a.counts + p);                        // (written by a kernel that may still run)
+  // (behind a kernel that may still be running, what it wrote is read from L2, not through the
+  // read-only path)
+  int count = BEHIND ? __ldcg(a.counts + p) : a.counts[p];
   const int64_t room = fixed ? (a.idx_stride < a.out_stride_h ? a.idx_stride : a.out_stride_h)
                              : (int64_t)a.offsets[p + 1] - a.offsets[p];
   if (count < 0 || count > room) {
@@ -78,15 +82,18 @@ __global__ void __launch_bounds__(kCompactWarps * 32) compact_kernel(const Compa
 
   for (int t0 = (part * kCompactWarps + warp) * kCompactRowsPerWarp; t0 < count;
        t0 += ctas_per_head * kCompactRowsPerCta) {
-    int j[kCompactRowsPerWarp];
-#pragma unroll
-    for (int i = 0; i < kCompactRowsPerWarp; ++i) {
-      j[i] = t0 + i < count ? __ldcg(ix + t0 + i) : -1;
-      if (t0 + i < count && (j[i] < 0 || j[i] >= n)) {
-        if (lane == 0) flag_status(a.status, CURDKV_DEV_BAD_INDEX);
-        j[i] = -1;
+    // the warp's eight indices in one request (lane i holds the i-th), then handed round
+    int mine = -1;
+    if (lane < kCompactRowsPerWarp && t0 + lane < count) {
+      mine = BEHIND ? __ldcg(ix + t0 + lane) : __ldg(ix + t0 + lane);
+      if (mine < 0 || mine >= n) {
+        flag_status(a.status, CURDKV_DEV_BAD_INDEX);
+        mine = -1;
       }
     }
+    int j[kCompactRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kCompactRowsPerWarp; ++i) j[i] = __shfl_sync(0xffffffffu, mine, i);
     for (int c = l16; c < chunks; c += 16) {
       uint4 v[kCompactRowsPerWarp];
 #pragma unroll

@@ -640,7 +640,7 @@ curdkv_status compact_impl(const void* K, const void* V, const curdkv_desc* desc
   if (ctas > 256) ctas = 256;
   while (P * ctas > 0x7fffffffLL) ctas >>= 1;
   if (ready == nullptr) {
-    compact_kernel<<<(unsigned)(P * ctas), kCompactWarps * 32, 0, stream>>>(a, (int)ctas);
+    compact_kernel<false><<<(unsigned)(P * ctas), kCompactWarps * 32, 0, stream>>>(a, (int)ctas);
   } else {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(P * ctas));
@@ -651,7 +651,7 @@ curdkv_status compact_impl(const void* K, const void* V, const curdkv_desc* desc
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, compact_kernel, a, (int)ctas) != cudaSuccess) return CURDKV_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, compact_kernel<true>, a, (int)ctas) != cudaSuccess) return CURDKV_ERR_CUDA;
   }
   if (!launch_ok()) return CURDKV_ERR_CUDA;
   return CURDKV_OK;
