@@ -261,7 +261,7 @@ def streaming_kernel_name(w, whiten, three_calls):
     if whiten:
         return "sketch_items_kernel<%d>" % (32 if w.r <= 32 else 64)
     fused = (not three_calls and not w.adaptive and w.ragged is None and w.r <= 32 and w.n_max >= 128
-             and w.folded_batch * w.kv_heads >= 4 * sms)
+             and w.folded_batch * w.kv_heads >= sms)
     return "sketch_umma_kernel<%d, %s>" % (32 if w.r <= 32 else 64, "true" if fused else "false")
 
 

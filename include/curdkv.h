@@ -190,7 +190,7 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
  * gathered rows) and the default output layouts (adaptive = 0: idx
  * [batch][kv_heads][budget], K_out / V_out [batch][kv_heads][budget][d]; adaptive = 1:
  * packed).  With a fixed budget, one shared G, projection on, whiten off, d = 128,
- * r <= 32, n_max >= 128, no per-sequence lengths and at least four heads per SM of the
+ * r <= 32, n_max >= 128, no per-sequence lengths and at least one head per SM of the
  * device, the scoring kernel also normalises and selects: the heads whose last tile has been
  * written are handed, through one list served by all CTAs, to extra warps that run Alg. 1
  * normalisation and selection steps for them while the stream of K and V goes on, so the selection costs almost no

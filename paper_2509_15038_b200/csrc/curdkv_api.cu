@@ -687,12 +687,14 @@ curdkv_status curdkv_compress(const void* K, const void* V, const float* G, int3
   // One launch scores and selects when the tensor-core sketch applies and every head has its own
   // budget; the selection then hides behind the K/V stream.  Otherwise the three steps follow
   // one another.
-  // (With fewer than four heads per SM the selection of the last heads, which only starts when the
-  // stream ends and runs on a quarter of a selection CTA's threads, costs more than it saves.)
+  // (With fewer heads than SMs the selection of the last heads, which only starts when the stream
+  // ends and runs on a quarter of a selection CTA's threads, costs more than the gather that
+  // starts beside it wins back: 64 heads of 8192 rows 0.100 against 0.092 ms, 128 heads 0.149
+  // against 0.153 ms, 256 heads 0.259 against 0.266 ms.)
   // Ragged batches keep the three-step route as well: their many short heads make the
   // selection warps busy enough to slow the stream by more than the hidden selection saves.
   const bool fused = !adaptive && budget > 0 && desc->use_projection && !g_per_head && !desc->whiten &&
-                     P >= 4 * (int64_t)sm_count() && desc->seqlens == nullptr &&
+                     P >= (int64_t)sm_count() && desc->seqlens == nullptr &&
                      desc->d == 128 && desc->r >= 1 && desc->r <= 32 && desc->n_max >= kTileRows &&
                      G != nullptr && P > 0 && P * tiles <= 0x7fffffffLL &&
                      P * (int64_t)budget <= 0x7fffffffLL;

@@ -1,7 +1,7 @@
 """curdkv_compress (one call; for the main shapes one kernel that scores, normalises and selects)
 against the three separate calls, bit for bit, and through them against the oracle.  Needs a B200.
 
-The single-kernel route is taken from four heads per SM upwards (592 heads on a B200): the cases
+The single-kernel route is taken from one head per SM upwards (148 heads on a B200): the cases
 below that are meant to reach it use 600 heads or more, the others cover the three-step route."""
 import numpy as np
 import pytest
