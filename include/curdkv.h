@@ -194,7 +194,9 @@ curdkv_status curdkv_compact(const void* K, const void* V, const curdkv_desc* de
  * device, the scoring kernel also normalises and selects: the heads whose last tile has been
  * written are handed, through one list served by all CTAs, to extra warps that run Alg. 1
  * normalisation and selection steps for them while the stream of K and V goes on, so the selection costs almost no
- * time of its own (a cooperative launch; it can still be captured into a CUDA graph).  Other
+ * time of its own (a cooperative launch; it can still be captured into a CUDA graph), and the
+ * gather is launched as that kernel's programmatic dependent: it copies the heads that are
+ * already selected while the last heads, which finish streaming last, are being selected.  Other
  * shapes run the three steps in sequence, the selection kernel forming the head sums and
  * dividing on its first sweep instead of a separate normalisation pass.
  *   workspace   curdkv_workspace_bytes(desc, budget > 0 ? budget : 1, adaptive) bytes
