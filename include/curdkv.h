@@ -373,6 +373,15 @@ curdkv_status curdkv_device_status(const void* workspace, uint32_t* host_flags, 
  * stream stays usable: read the word with curdkv_device_status(). */
 curdkv_status curdkv_selftest_bounded_wait(uint64_t limit_ns, void* workspace, void* cuda_stream);
 
+/* The same for the one wait outside those kernels (no counterpart in the paper): inside
+ * curdkv_compress the gather may start before the kernel that selects has ended, and each
+ * of its CTAs then waits, bounded, for its head's ready flag.  This call launches that
+ * gather for one head whose flag nothing ever sets, with `limit_ns` (1 .. 10^9) as the
+ * limit: the kernel comes back after about limit_ns with CURDKV_DEV_TIMEOUT in the status
+ * word of `workspace` (at least 512 bytes, 256-byte aligned; cleared first) and has read
+ * and written nothing else. */
+curdkv_status curdkv_selftest_gather_wait(uint64_t limit_ns, void* workspace, void* cuda_stream);
+
 /* Profiling aid (no counterpart in the paper): asks the next curdkv_score or
  * curdkv_score_static call of THIS host thread to record the two cudaEvent_t
  * handles (passed as void*, either may be NULL) on its stream immediately

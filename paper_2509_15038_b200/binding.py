@@ -29,7 +29,7 @@ EXPORTS = (
     "curdkv_profile_next_score", "curdkv_cache_workspace_bytes", "curdkv_cache_append",
     "curdkv_cache_compress", "curdkv_attention_workspace_bytes", "curdkv_attention_out",
     "curdkv_eviction_loss", "curdkv_gqa_expand", "curdkv_cache_compress_inplace",
-    "curdkv_selftest_bounded_wait", "curdkv_compress", "curdkv_cache_step",
+    "curdkv_selftest_bounded_wait", "curdkv_selftest_gather_wait", "curdkv_compress", "curdkv_cache_step",
 )
 
 
@@ -125,6 +125,8 @@ def load():
     lib.curdkv_eviction_loss.argtypes = [vp, vp, i32, i64, vp, vp, vp]
     lib.curdkv_selftest_bounded_wait.restype = ctypes.c_int
     lib.curdkv_selftest_bounded_wait.argtypes = [ctypes.c_uint64, vp, vp]
+    lib.curdkv_selftest_gather_wait.restype = ctypes.c_int
+    lib.curdkv_selftest_gather_wait.argtypes = [ctypes.c_uint64, vp, vp]
     lib.curdkv_profile_next_score.restype = ctypes.c_int
     lib.curdkv_profile_next_score.argtypes = [vp, vp]
     lib.curdkv_launch_count.restype = ctypes.c_uint64
@@ -459,6 +461,12 @@ def curdkv_selftest_bounded_wait(limit_ns: int, workspace: torch.Tensor) -> None
     """Runs the kernels' bounded wait on a barrier nobody completes; leaves DEV_TIMEOUT in the status word."""
     _check(load().curdkv_selftest_bounded_wait(int(limit_ns), _ptr(workspace), _stream()),
            "curdkv_selftest_bounded_wait")
+
+
+def curdkv_selftest_gather_wait(limit_ns: int, workspace: torch.Tensor) -> None:
+    """Runs the gather's bounded wait for a head that is never announced; leaves DEV_TIMEOUT in the status word."""
+    _check(load().curdkv_selftest_gather_wait(int(limit_ns), _ptr(workspace), _stream()),
+           "curdkv_selftest_gather_wait")
 
 
 def curdkv_gqa_map(desc: Desc, device="cuda") -> torch.Tensor:

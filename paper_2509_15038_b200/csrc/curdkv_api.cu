@@ -933,6 +933,22 @@ curdkv_status curdkv_selftest_bounded_wait(uint64_t limit_ns, void* workspace, v
   return CURDKV_OK;
 }
 
+curdkv_status curdkv_selftest_gather_wait(uint64_t limit_ns, void* workspace, void* cuda_stream) {
+  if (workspace == nullptr || limit_ns == 0 || limit_ns > 1000000000ull) return CURDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return CURDKV_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, 2 * kStatusBytes, stream) != cudaSuccess) return CURDKV_ERR_CUDA;
+  CompactArgs a = {};                                      // one head; the kernel leaves before it reads any of the rest
+  a.heads = 1;
+  a.d = 128;
+  a.status = static_cast<uint32_t*>(workspace);
+  a.ready = reinterpret_cast<const int32_t*>(static_cast<unsigned char*>(workspace) + kStatusBytes);
+  a.wait_ns = limit_ns;
+  compact_kernel<true><<<1, kCompactWarps * 32, 0, stream>>>(a, 1);
+  if (!launch_ok()) return CURDKV_ERR_CUDA;
+  return CURDKV_OK;
+}
+
 curdkv_status curdkv_profile_next_score(void* start_event, void* stop_event) {
   g_profile_start = static_cast<cudaEvent_t>(start_event);
   g_profile_stop = static_cast<cudaEvent_t>(stop_event);

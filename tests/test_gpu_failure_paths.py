@@ -40,6 +40,33 @@ def test_bounded_wait_runs_out_and_the_stream_stays_usable():
     assert torch.equal(after_scores, before_scores) and torch.equal(after_sums, before_sums)
 
 
+def test_gather_wait_for_a_head_that_never_arrives_runs_out():
+    """The gather that curdkv_compress starts beside the last selections waits per head for a ready
+    flag.  With a flag that nothing sets, the wait ends at its limit with CURDKV_DEV_TIMEOUT, nothing
+    else in the workspace is touched, and the next call on the stream works as before."""
+    w = synth.shrink(synth.CONFIGS["cfg2"], layers=1, n_max=2048)
+    K, V, _ = synth.make_kv(w, DEV)
+    G = torch.as_tensor(synth.make_G(w.d, w.r, seed=0), device=DEV)
+    desc = cur.make_desc(K, V, w.r, q_heads=w.q_heads)
+    ws = cur.alloc_workspace(desc, w.budget)
+    before = [t.clone() for t in cur.curdkv_compress(K, V, G, desc, w.budget, ws, window=w.window)]
+    ws[512:] = 0x5a
+    t0 = time.perf_counter()
+    cur.curdkv_selftest_gather_wait(2_000_000, ws)
+    code, flags = cur.curdkv_device_status(ws, with_code=True)
+    waited = time.perf_counter() - t0
+    assert flags & cur.DEV_TIMEOUT and code == 5
+    assert 0.002 <= waited < 1.0
+    assert bool((ws[512:] == 0x5a).all())
+    after = cur.curdkv_compress(K, V, G, desc, w.budget, ws, window=w.window)
+    assert cur.curdkv_device_status(ws, with_code=True) == (0, 0)
+    assert all(torch.equal(x, y) for x, y in zip(before, after))
+    for bad in (0, 2_000_000_000):
+        with pytest.raises(cur.CurdkvError) as e:
+            cur.curdkv_selftest_gather_wait(bad, ws)
+        assert e.value.code == 1
+
+
 def test_bounded_wait_limit_is_validated_on_the_host():
     ws = torch.zeros((256,), dtype=torch.uint8, device=DEV)
     before = cur.launch_count()
